@@ -1,0 +1,149 @@
+/*
+ * resq.h -- C ABI of the ResQ mixed-precision linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer (paper, Section 4.1): activations are expressed in an orthogonal basis U = P·R
+ * (Eq. 5); the first r coefficients of every token are quantized to symmetric per-token INT8,
+ * the remaining K - r to symmetric per-token INT4 (Eq. 1, Eq. 2); the weights, projected offline
+ * by U^T, are quantized the same way per output channel (Eq. 3); the output is the sum of the
+ * two same-precision integer products, each rescaled by its token scale and channel scale (Eq. 4):
+ *
+ *     Y[t][n] = s_x8[t]·s_w8[n]·sum_{j<r}  x8[t][j]·w8[n][j]
+ *             + s_x4[t]·s_w4[n]·sum_{j<K-r} x4[t][j]·w4[n][j]
+ *
+ * Conventions shared by every entry point
+ *  - All data pointers are DEVICE pointers to caller-owned memory unless a parameter says "host".
+ *    The library allocates no device memory, keeps no reference to any buffer after the call
+ *    returns, and never synchronizes the stream: work is enqueued on `stream` (a cudaStream_t
+ *    passed as void*, NULL = default stream).
+ *  - Descriptor structs are read on the host during the call.
+ *  - Matrices are row-major with the K (reduction) dimension contiguous.  The high-precision
+ *    coefficients come first in a row: columns [0, r) are the INT8 segment, [r, K) the INT4 one.
+ *  - INT4 packing: byte i of a row holds code 2i in bits 0..3 and code 2i+1 in bits 4..7, two's
+ *    complement.  Codes produced here lie in [-127,127] and [-7,7]; consumers accept the full
+ *    [-128,127] and [-8,7].
+ *  - Quantizer arithmetic (fixed so that results are reproducible bit for bit): absmax a over the
+ *    segment; s = a / qmax as an IEEE fp32 division (qmax = 127 or 7); if the scale is stored as
+ *    fp16 it is rounded to fp16 first and the rounded value is the one used; code =
+ *    clamp(round-half-even(x / s)) with an IEEE fp32 division; a == 0 gives s = 0 and codes 0.
+ *  - Shape rules: r % 32 == 0, (K - r) % 32 == 0, 0 < r < K, n_out % 8 == 0, T >= 1.
+ *    Data pointers must be 16-byte aligned.
+ *  - Every function returns a resq_status_t (0 = success).  Arguments are validated on the host
+ *    before anything is launched; on a non-zero return nothing was enqueued.  Waits inside the
+ *    kernels are bounded; a wait that runs out sets a device status word (see resq_device_status)
+ *    and the kernel drains and returns.
+ *  - Inputs must be finite; NaN/Inf are not checked.
+ */
+#ifndef RESQ_H_
+#define RESQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum resq_status {
+    RESQ_OK = 0,
+    RESQ_ERR_NULL = 1,       /* a required pointer is NULL */
+    RESQ_ERR_SHAPE = 2,      /* a shape rule above is violated */
+    RESQ_ERR_ALIGN = 3,      /* a pointer is not 16-byte aligned */
+    RESQ_ERR_WORKSPACE = 4,  /* workspace missing or smaller than resq_workspace_bytes() */
+    RESQ_ERR_ARCH = 5,       /* current device is not compute capability 10.x */
+    RESQ_ERR_CUDA = 6,       /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+    RESQ_ERR_TIMEOUT = 7     /* reported by resq_device_status: a bounded device wait ran out */
+} resq_status_t;
+
+/* Weight-scale storage type. */
+enum { RESQ_SCALE_FP32 = 0, RESQ_SCALE_FP16 = 1 };
+/* Output type of Y. */
+enum { RESQ_Y_BF16 = 0, RESQ_Y_FP32 = 1 };
+
+/* One linear layer: K input features (coefficients), n_out output channels, r high-precision
+ * coefficients (the paper uses r = K/8, Section 4.1). */
+typedef struct resq_layer_desc {
+    int32_t K;
+    int32_t n_out;
+    int32_t r;
+    int32_t w_scale_dtype; /* RESQ_SCALE_FP32 or RESQ_SCALE_FP16 */
+} resq_layer_desc_t;
+
+/* Quantized weights of one layer, as written by resq_pack_weights (Eq. 3). */
+typedef struct resq_weights {
+    const int8_t* w8;    /* [n_out][r]        INT8 codes                                   */
+    const uint8_t* w4;   /* [n_out][(K-r)/2]  INT4 codes, packed                            */
+    const void* s_w8;    /* [n_out]           fp32 or fp16 per w_scale_dtype                */
+    const void* s_w4;    /* [n_out]                                                          */
+    const int8_t* w4_i8; /* [n_out][K-r] optional: the INT4 codes one per byte (sign-extended),
+                            a layout for the compute-bound many-token kernel; NULL = absent, the
+                            kernel then expands `w4` itself into the workspace */
+} resq_weights_t;
+
+/* Byte sizes of the packed buffers of a layer. */
+size_t resq_w8_bytes(const resq_layer_desc_t* desc);    /* n_out * r          */
+size_t resq_w4_bytes(const resq_layer_desc_t* desc);    /* n_out * (K-r) / 2  */
+size_t resq_w4_i8_bytes(const resq_layer_desc_t* desc); /* n_out * (K-r)      */
+size_t resq_scale_bytes(const resq_layer_desc_t* desc); /* n_out * 4 or * 2   */
+
+/* Scratch bytes that resq_project_quantize / resq_mixed_gemm / resq_linear need for T tokens.
+ * has_P != 0: the online projection is used.  has_w4_i8 != 0: weights carry the w4_i8 layout.
+ * Returns 0 on an invalid descriptor. */
+size_t resq_workspace_bytes(const resq_layer_desc_t* desc, int T, int has_P, int has_w4_i8);
+
+/*
+ * Eq. 3: quantize projected weights.  W_proj is (U^T W)^T as fp32 [n_out][K]; each output channel is
+ * split at r and quantized per segment (round to nearest; the paper's experiments use GPTQ instead,
+ * which is out of scope).  Outputs w8, w4, s_w8, s_w4 as in resq_weights_t; w4_i8 may be NULL.
+ */
+int resq_pack_weights(const resq_layer_desc_t* desc, const float* W_proj, int8_t* w8, uint8_t* w4,
+                      void* s_w8, void* s_w4, int8_t* w4_i8, void* stream);
+
+/*
+ * Eq. 2: per-token split quantization of the coefficients.
+ *   P == NULL: the rows of X (bf16 [T][K]) already are the coefficients -- the projection was
+ *              folded into the preceding layer's weights (Section 4.3, U_A/U_B).
+ *   P != NULL: bf16 [K][K], row i = input feature, column j = coefficient; C = X·P is formed online
+ *              on the tensor cores with fp32 accumulation (Section 4.3, U_D for the down_proj input)
+ *              and quantized from fp32 without an intermediate bf16 rounding.  Needs workspace.
+ * Outputs: x8 int8 [T][r]; x4 packed uint8 [T][(K-r)/2]; s_x8, s_x4 fp32 [T].
+ * x4_i8 (optional, may be NULL): the INT4 codes one per byte, int8 [T][K-r].
+ */
+int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int8_t* x8, uint8_t* x4,
+                          float* s_x8, float* s_x4, int8_t* x4_i8, void* workspace,
+                          size_t workspace_bytes, void* stream);
+
+/*
+ * Eq. 4 with the dequantizing epilogue: Y = diag(s_x8)(x8·w8^T)diag(s_w8) + diag(s_x4)(x4·w4^T)diag(s_w4).
+ * Integer products accumulate exactly in int32; the epilogue is fp32:
+ *     y = (float)acc8 * (s_x8[t] * s_w8[n]) + (float)acc4 * (s_x4[t] * s_w4[n])
+ * rounded to bf16 (nearest even) when y_dtype == RESQ_Y_BF16.  Y is [T][n_out].
+ * T <= 16 runs the weight-streaming split-K kernel, larger T the tensor-core tile kernel.
+ * dbg_acc8 / dbg_acc4: optional int32 [T][n_out] dumps of the two accumulators (NULL = off).
+ */
+int resq_mixed_gemm(const resq_layer_desc_t* desc, int T, const int8_t* x8, const uint8_t* x4,
+                    const float* s_x8, const float* s_x4, const resq_weights_t* W, void* Y, int y_dtype,
+                    int32_t* dbg_acc8, int32_t* dbg_acc4, void* workspace, size_t workspace_bytes,
+                    void* stream);
+
+/*
+ * The whole layer: resq_project_quantize followed by resq_mixed_gemm, with the quantized
+ * activations held in the workspace.  X bf16 [T][K]; P bf16 [K][K] or NULL; Y [T][n_out].
+ */
+int resq_linear(const resq_layer_desc_t* desc, int T, const void* X, const void* P,
+                const resq_weights_t* W, void* Y, int y_dtype, void* workspace, size_t workspace_bytes,
+                void* stream);
+
+/* Inverse of the INT4 packing, for inspection: packed [rows][cols/2] -> int8 [rows][cols]. */
+int resq_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, void* stream);
+
+/* Synchronizes `stream`, then reads and clears the device status word of the current device:
+ * RESQ_OK, RESQ_ERR_TIMEOUT, or RESQ_ERR_CUDA if the stream reported an error. */
+int resq_device_status(void* stream);
+
+/* Static, human-readable name of a status code. */
+const char* resq_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RESQ_H_ */

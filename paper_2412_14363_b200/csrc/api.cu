@@ -1,0 +1,268 @@
+// C ABI of the library: argument validation, workspace carving and dispatch.  No arithmetic here.
+#include <cstdio>
+#include <cstdlib>
+#include <cuda_runtime.h>
+
+#include "internal.h"
+
+namespace resq {
+
+__device__ int g_status_word = 0;
+
+int* device_status_ptr() {
+    static int* cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cache[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        cache[dev] = static_cast<int*>(p);
+    }
+    return cache[dev];
+}
+
+void* tensor_map_encode_fn() {
+    static void* fn = nullptr;
+    if (!fn) {
+        cudaDriverEntryPointQueryResult q;
+        void* f = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = f;
+    }
+    return fn;
+}
+
+namespace {
+
+constexpr int kDecodeMaxT = 0;  // TODO(decode): 16 once the streaming kernel lands
+constexpr int kPanelRows = 512;  // token rows of fp32 coefficients staged per projection panel
+
+inline size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int check_shape(int K, int n_out, int r) {
+    if (K <= 0 || r <= 0 || r >= K || n_out <= 0) return RESQ_ERR_SHAPE;
+    if (r % 32 != 0 || (K - r) % 32 != 0 || n_out % 8 != 0) return RESQ_ERR_SHAPE;
+    return RESQ_OK;
+}
+int check_desc(const resq_layer_desc_t* d) {
+    if (!d) return RESQ_ERR_NULL;
+    if (d->w_scale_dtype != RESQ_SCALE_FP32 && d->w_scale_dtype != RESQ_SCALE_FP16) return RESQ_ERR_SHAPE;
+    return check_shape(d->K, d->n_out, d->r);
+}
+int check_arch() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RESQ_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return RESQ_ERR_CUDA;
+    return major == 10 ? RESQ_OK : RESQ_ERR_ARCH;
+}
+
+// Carving of the caller's workspace.  Every entry point uses the same map (and its own subset).
+struct Workspace {
+    size_t x8, x4, sx8, sx4, x4e, w4e, panel, decode, total;
+};
+Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
+    Workspace w{};
+    const size_t K4 = static_cast<size_t>(K - r), Tz = static_cast<size_t>(T), N = static_cast<size_t>(n_out);
+    size_t o = 0;
+    w.x8 = o;  o += align_up(Tz * r);
+    w.x4 = o;  o += align_up(Tz * K4 / 2);
+    w.sx8 = o; o += align_up(Tz * 4);
+    w.sx4 = o; o += align_up(Tz * 4);
+    const bool tiles = T > kDecodeMaxT;
+    w.x4e = o;    o += tiles ? align_up(Tz * K4) : 0;
+    w.w4e = o;    o += (tiles && !has_w4_i8) ? align_up(N * K4) : 0;
+    w.panel = o;  o += has_P ? align_up(static_cast<size_t>(T < kPanelRows ? T : kPanelRows) * K * 4) : 0;
+    w.decode = o; o += tiles ? 0 : align_up(decode_scratch_bytes(T, n_out));
+    w.total = o;
+    return w;
+}
+
+int cuda_status(cudaError_t e) { return e == cudaSuccess ? RESQ_OK : RESQ_ERR_CUDA; }
+
+}  // namespace
+}  // namespace resq
+
+using namespace resq;
+
+extern "C" {
+
+size_t resq_w8_bytes(const resq_layer_desc_t* d) {
+    return check_desc(d) ? 0 : static_cast<size_t>(d->n_out) * d->r;
+}
+size_t resq_w4_bytes(const resq_layer_desc_t* d) {
+    return check_desc(d) ? 0 : static_cast<size_t>(d->n_out) * (d->K - d->r) / 2;
+}
+size_t resq_w4_i8_bytes(const resq_layer_desc_t* d) {
+    return check_desc(d) ? 0 : static_cast<size_t>(d->n_out) * (d->K - d->r);
+}
+size_t resq_scale_bytes(const resq_layer_desc_t* d) {
+    return check_desc(d) ? 0 : static_cast<size_t>(d->n_out) * (d->w_scale_dtype == RESQ_SCALE_FP16 ? 2 : 4);
+}
+
+size_t resq_workspace_bytes(const resq_layer_desc_t* d, int T, int has_P, int has_w4_i8) {
+    if (check_desc(d) || T < 1) return 0;
+    return carve(d->K, d->n_out, d->r, T, has_P != 0, has_w4_i8 != 0).total;
+}
+
+int resq_pack_weights(const resq_layer_desc_t* d, const float* W_proj, int8_t* w8, uint8_t* w4, void* s_w8,
+                      void* s_w4, int8_t* w4_i8, void* stream) {
+    if (int e = check_desc(d)) return e;
+    if (!W_proj || !w8 || !w4 || !s_w8 || !s_w4) return RESQ_ERR_NULL;
+    if (!aligned16(W_proj) || !aligned16(w8) || !aligned16(w4) || !aligned16(s_w8) || !aligned16(s_w4) ||
+        !aligned16(w4_i8))
+        return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_split_quantize(W_proj, true, d->n_out, d->K, d->r, w8, w4, s_w8, s_w4,
+                                             d->w_scale_dtype == RESQ_SCALE_FP16, w4_i8,
+                                             static_cast<size_t>(d->K) * 4, static_cast<cudaStream_t>(stream)));
+}
+
+int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int8_t* x8, uint8_t* x4, float* s_x8,
+                          float* s_x4, int8_t* x4_i8, void* workspace, size_t workspace_bytes, void* stream) {
+    if (T < 1) return RESQ_ERR_SHAPE;
+    if (int e = check_shape(K, 8, r)) return e;
+    if (!X || !x8 || !s_x8 || !s_x4 || (!x4 && !x4_i8)) return RESQ_ERR_NULL;
+    if (!aligned16(X) || !aligned16(P) || !aligned16(x8) || !aligned16(x4) || !aligned16(s_x8) ||
+        !aligned16(s_x4) || !aligned16(x4_i8) || !aligned16(workspace))
+        return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!P)
+        return cuda_status(launch_split_quantize(X, false, T, K, r, x8, x4, s_x8, s_x4, false, x4_i8,
+                                                 static_cast<size_t>(K) * 2, st));
+    // Online projection: panels of token rows, fp32 coefficients staged in the workspace.
+    const int rows_max = T < kPanelRows ? T : kPanelRows;
+    const size_t need = align_up(static_cast<size_t>(rows_max) * K * 4);
+    if (!workspace || workspace_bytes < need) return RESQ_ERR_WORKSPACE;
+    float* panel = static_cast<float*>(workspace);
+    const size_t K4 = static_cast<size_t>(K - r);
+    for (int t0 = 0; t0 < T; t0 += kPanelRows) {
+        const int rows = T - t0 < kPanelRows ? T - t0 : kPanelRows;
+        const char* Xp = static_cast<const char*>(X) + static_cast<size_t>(t0) * K * 2;
+        if (cudaError_t e = launch_project_gemm(Xp, P, rows, K, panel, st); e != cudaSuccess) return RESQ_ERR_CUDA;
+        if (cudaError_t e = launch_split_quantize(panel, true, rows, K, r, x8 + static_cast<size_t>(t0) * r,
+                                                  x4 ? x4 + static_cast<size_t>(t0) * K4 / 2 : nullptr, s_x8 + t0,
+                                                  s_x4 + t0, false,
+                                                  x4_i8 ? x4_i8 + static_cast<size_t>(t0) * K4 : nullptr,
+                                                  static_cast<size_t>(K) * 4, st);
+            e != cudaSuccess)
+            return RESQ_ERR_CUDA;
+    }
+    return RESQ_OK;
+}
+
+static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, const uint8_t* x4,
+                           const int8_t* x4e_ready, const float* s_x8, const float* s_x4, const resq_weights_t* W,
+                           void* Y, int y_dtype, int32_t* dbg8, int32_t* dbg4, char* ws, const Workspace& map,
+                           cudaStream_t st) {
+    const bool fp16 = d->w_scale_dtype == RESQ_SCALE_FP16;
+    const size_t K4 = static_cast<size_t>(d->K - d->r);
+    if (T <= kDecodeMaxT)
+        return cuda_status(launch_mixed_gemm_decode(T, d->n_out, d->K, d->r, x8, x4, s_x8, s_x4, W->w8, W->w4,
+                                                    W->s_w8, W->s_w4, fp16, Y, y_dtype, dbg8, dbg4,
+                                                    ws + map.decode, st));
+    const int8_t* x4e = x4e_ready;
+    if (!x4e) {
+        int8_t* buf = reinterpret_cast<int8_t*>(ws + map.x4e);
+        if (cudaError_t e = launch_unpack_int4(x4, buf, T, K4, st); e != cudaSuccess) return RESQ_ERR_CUDA;
+        x4e = buf;
+    }
+    const int8_t* w4e = W->w4_i8;
+    if (!w4e) {
+        int8_t* buf = reinterpret_cast<int8_t*>(ws + map.w4e);
+        if (cudaError_t e = launch_unpack_int4(W->w4, buf, d->n_out, K4, st); e != cudaSuccess) return RESQ_ERR_CUDA;
+        w4e = buf;
+    }
+    return cuda_status(launch_mixed_gemm_tiles(T, d->n_out, d->K, d->r, x8, x4e, s_x8, s_x4, W->w8, w4e, W->s_w8,
+                                               W->s_w4, fp16, Y, y_dtype, dbg8, dbg4, st));
+}
+
+static int check_weights(const resq_weights_t* W) {
+    if (!W || !W->w8 || !W->w4 || !W->s_w8 || !W->s_w4) return RESQ_ERR_NULL;
+    if (!aligned16(W->w8) || !aligned16(W->w4) || !aligned16(W->s_w8) || !aligned16(W->s_w4) ||
+        !aligned16(W->w4_i8))
+        return RESQ_ERR_ALIGN;
+    return RESQ_OK;
+}
+
+int resq_mixed_gemm(const resq_layer_desc_t* d, int T, const int8_t* x8, const uint8_t* x4, const float* s_x8,
+                    const float* s_x4, const resq_weights_t* W, void* Y, int y_dtype, int32_t* dbg_acc8,
+                    int32_t* dbg_acc4, void* workspace, size_t workspace_bytes, void* stream) {
+    if (int e = check_desc(d)) return e;
+    if (T < 1 || (y_dtype != RESQ_Y_BF16 && y_dtype != RESQ_Y_FP32)) return RESQ_ERR_SHAPE;
+    if (!x8 || !x4 || !s_x8 || !s_x4 || !Y) return RESQ_ERR_NULL;
+    if ((dbg_acc8 == nullptr) != (dbg_acc4 == nullptr)) return RESQ_ERR_NULL;
+    if (int e = check_weights(W)) return e;
+    if (!aligned16(x8) || !aligned16(x4) || !aligned16(s_x8) || !aligned16(s_x4) || !aligned16(Y) ||
+        !aligned16(dbg_acc8) || !aligned16(dbg_acc4) || !aligned16(workspace))
+        return RESQ_ERR_ALIGN;
+    const Workspace map = carve(d->K, d->n_out, d->r, T, false, W->w4_i8 != nullptr);
+    if (!workspace || workspace_bytes < map.total) return RESQ_ERR_WORKSPACE;
+    if (int e = check_arch()) return e;
+    return mixed_gemm_impl(d, T, x8, x4, nullptr, s_x8, s_x4, W, Y, y_dtype, dbg_acc8, dbg_acc4,
+                           static_cast<char*>(workspace), map, static_cast<cudaStream_t>(stream));
+}
+
+int resq_linear(const resq_layer_desc_t* d, int T, const void* X, const void* P, const resq_weights_t* W, void* Y,
+                int y_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    if (int e = check_desc(d)) return e;
+    if (T < 1 || (y_dtype != RESQ_Y_BF16 && y_dtype != RESQ_Y_FP32)) return RESQ_ERR_SHAPE;
+    if (!X || !Y) return RESQ_ERR_NULL;
+    if (int e = check_weights(W)) return e;
+    if (!aligned16(X) || !aligned16(P) || !aligned16(Y) || !aligned16(workspace)) return RESQ_ERR_ALIGN;
+    const Workspace map = carve(d->K, d->n_out, d->r, T, P != nullptr, W->w4_i8 != nullptr);
+    if (!workspace || workspace_bytes < map.total) return RESQ_ERR_WORKSPACE;
+    if (int e = check_arch()) return e;
+    char* ws = static_cast<char*>(workspace);
+    int8_t* x8 = reinterpret_cast<int8_t*>(ws + map.x8);
+    uint8_t* x4 = reinterpret_cast<uint8_t*>(ws + map.x4);
+    float* s_x8 = reinterpret_cast<float*>(ws + map.sx8);
+    float* s_x4 = reinterpret_cast<float*>(ws + map.sx4);
+    const bool tiles = T > kDecodeMaxT;
+    int8_t* x4e = tiles ? reinterpret_cast<int8_t*>(ws + map.x4e) : nullptr;
+    // The tile kernel consumes the one-code-per-byte layout, the streaming kernel the packed one.
+    if (int e = resq_project_quantize(X, P, T, d->K, d->r, x8, tiles ? nullptr : x4, s_x8, s_x4, x4e, ws + map.panel,
+                                      workspace_bytes - map.panel, stream))
+        return e;
+    return mixed_gemm_impl(d, T, x8, x4, x4e, s_x8, s_x4, W, Y, y_dtype, nullptr, nullptr, ws, map,
+                           static_cast<cudaStream_t>(stream));
+}
+
+int resq_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, void* stream) {
+    if (!packed || !out) return RESQ_ERR_NULL;
+    if (cols % 8 != 0) return RESQ_ERR_SHAPE;
+    if (!aligned16(packed) || !aligned16(out)) return RESQ_ERR_ALIGN;
+    return cuda_status(launch_unpack_int4(packed, out, rows, cols, static_cast<cudaStream_t>(stream)));
+}
+
+int resq_device_status(void* stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return RESQ_ERR_CUDA;
+    int* p = device_status_ptr();
+    if (!p) return RESQ_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, p, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RESQ_ERR_CUDA;
+    if (v != 0) {
+        int zero = 0;
+        cudaMemcpy(p, &zero, sizeof(int), cudaMemcpyHostToDevice);
+        return RESQ_ERR_TIMEOUT;
+    }
+    return RESQ_OK;
+}
+
+const char* resq_status_string(int s) {
+    switch (s) {
+        case RESQ_OK: return "ok";
+        case RESQ_ERR_NULL: return "null pointer";
+        case RESQ_ERR_SHAPE: return "invalid shape";
+        case RESQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case RESQ_ERR_WORKSPACE: return "workspace missing or too small";
+        case RESQ_ERR_ARCH: return "device is not compute capability 10.x";
+        case RESQ_ERR_CUDA: return "CUDA call failed";
+        case RESQ_ERR_TIMEOUT: return "bounded device wait ran out";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,45 @@
+// Internal declarations shared by the translation units of the library (host side).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/resq.h"
+
+namespace resq {
+
+// Device status word (one per device that loaded the library); kernels OR an error code into it.
+int* device_status_ptr();  // device address of the status word of the current device, or nullptr
+
+// ---- kernels (launch wrappers; return cudaGetLastError()) ----------------------------------
+// Split quantization of the rows of a [rows][K] matrix (Eq. 2 for activations, Eq. 3 for weights).
+//   in_is_f32: rows are fp32 (weights, projected coefficients) instead of bf16.
+//   scale_fp16: scales are rounded to and stored as fp16 (weights only).
+//   absmax_bits: optional [rows][2] uint32 bit patterns of the precomputed per-segment absmax
+//                (written by the projection GEMM's epilogue); NULL = compute here.
+cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, int K, int r, int8_t* q8,
+                                  uint8_t* q4, void* s8, void* s4, bool scale_fp16, int8_t* q4_i8,
+                                  size_t in_row_stride, cudaStream_t st);
+
+cudaError_t launch_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, cudaStream_t st);
+
+// Many-token tile kernel on tcgen05 kind::i8.  x4e / w4e are the INT4 codes one per byte.
+cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8, const int8_t* x4e,
+                                    const float* s_x8, const float* s_x4, const int8_t* w8, const int8_t* w4e,
+                                    const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
+                                    int32_t* dbg8, int32_t* dbg4, cudaStream_t st);
+
+// Few-token (T <= 16) weight-streaming split-K kernel.  scratch: see decode_scratch_bytes().
+size_t decode_scratch_bytes(int T, int N);
+cudaError_t launch_mixed_gemm_decode(int T, int N, int K, int r, const int8_t* x8, const uint8_t* x4,
+                                     const float* s_x8, const float* s_x4, const int8_t* w8, const uint8_t* w4,
+                                     const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
+                                     int32_t* dbg8, int32_t* dbg4, void* scratch, cudaStream_t st);
+
+// Online projection C = X·P (bf16 x bf16 -> fp32) on tcgen05 kind::f16; writes fp32 C [T][K].
+cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, float* C, cudaStream_t st);
+
+// Driver entry point for tensor-map encoding (resolved once, without linking libcuda).
+void* tensor_map_encode_fn();
+
+}  // namespace resq

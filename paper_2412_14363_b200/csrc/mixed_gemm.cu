@@ -1,0 +1,319 @@
+// Many-token mixed-precision GEMM (Eq. 4 + dequantizing epilogue) on tcgen05 kind::i8.
+//
+// Persistent, warp-specialised kernel, one CTA per SM, 128 x 256 output tiles:
+//   warp 0     TMA producer: streams 128-byte-wide K blocks of the activation and weight codes
+//              into a 4-stage shared-memory ring (128-byte swizzle), first the INT8 segment, then
+//              the INT4 segment (codes one per byte, so both run on the i8 tensor path exactly);
+//   warp 1     owns TMEM (512 columns) and issues tcgen05.mma: the INT8 segment accumulates into
+//              columns [0,256), the INT4 segment into [256,512) -- two int32 accumulators per output
+//              because the two segments carry different (token, channel) scales;
+//   warps 2-5  epilogue: tcgen05.ld both accumulators, y = acc8*(sx8*sw8) + acc4*(sx4*sw4) in fp32,
+//              convert and store.
+// Out-of-range rows/columns/K are zero-filled by TMA and masked at the store.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace resq {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 128;  // BK in bytes == int8 elements
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK;
+constexpr int kThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr uint32_t kTmemCols = 512;
+
+struct Params {
+    int T, N, r, K4;
+    int m_tiles, n_tiles, kb8, kb4;
+    const float* s_x8;
+    const float* s_x4;
+    const void* s_w8;
+    const void* s_w4;
+    int w_fp16;
+    void* Y;
+    int y_dtype;
+    int32_t* dbg8;
+    int32_t* dbg4;
+    int* status;
+};
+
+struct __align__(8) Shared {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t acc_full;
+    uint64_t acc_empty;
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    int epi_stop;
+    float sw8[BN];
+    float sw4[BN];
+};
+
+constexpr size_t kSmemBytes = 1024 + STAGES * (A_BYTES + B_BYTES) + sizeof(Shared);
+
+__device__ __forceinline__ float load_scale(const void* p, int i, int fp16) {
+    return fp16 ? __half2float(reinterpret_cast<const __half*>(p)[i]) : reinterpret_cast<const float*>(p)[i];
+}
+
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constant__ CUtensorMap tmA4,
+                  const __grid_constant__ CUtensorMap tmB8, const __grid_constant__ CUtensorMap tmB4,
+                  const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + STAGES * A_BYTES;
+    Shared* sh = reinterpret_cast<Shared*>(smem + STAGES * (A_BYTES + B_BYTES));
+    volatile int* abort_flag = &sh->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_tiles = p.m_tiles * p.n_tiles;
+    const int kb_total = p.kb8 + p.kb4;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&sh->full[s], 1);
+            mbar_init(&sh->empty[s], 1);
+        }
+        mbar_init(&sh->acc_full, 1);
+        mbar_init(&sh->acc_empty, kEpiThreads);
+        mbar_init(&sh->drain, 1);
+        sh->abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tmA8);
+        tma_prefetch_desc(&tmA4);
+        tma_prefetch_desc(&tmB8);
+        tma_prefetch_desc(&tmB4);
+    }
+    if (warp == 1) {
+        tmem_alloc(&sh->tmem_base, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int issued = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * BN;
+                for (int kb = 0; kb < kb_total; ++kb) {
+                    if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+                    mbar_arrive_expect_tx(&sh->full[stage], A_BYTES + B_BYTES);
+                    if (kb < p.kb8) {
+                        tma_load_2d(sA + stage * A_BYTES, &tmA8, &sh->full[stage], kb * BK, m0);
+                        tma_load_2d(sB + stage * B_BYTES, &tmB8, &sh->full[stage], kb * BK, n0);
+                    } else {
+                        tma_load_2d(sA + stage * A_BYTES, &tmA4, &sh->full[stage], (kb - p.kb8) * BK, m0);
+                        tma_load_2d(sB + stage * B_BYTES, &tmB4, &sh->full[stage], (kb - p.kb8) * BK, n0);
+                    }
+                    ++issued;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+            if (!ok) {
+                // Let the copies already in flight land before the CTA gives up its shared memory.
+                int n = issued < STAGES ? issued : STAGES;
+                for (int i = 0; i < n; ++i) {
+                    if (stage == 0) { stage = STAGES; phase ^= 1; }
+                    --stage;
+                    const uint64_t t0 = global_timer_ns();
+                    while (!mbar_try_wait(&sh->full[stage], phase) && global_timer_ns() - t0 < 100000000ull) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_i8(BM, BN);
+            int stage = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                if (!mbar_wait(&sh->acc_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                for (int kb = 0; kb < kb_total; ++kb) {
+                    if (!mbar_wait(&sh->full[stage], phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t a_desc = make_smem_desc_k128(smem_u32(sA + stage * A_BYTES));
+                    const uint64_t b_desc = make_smem_desc_k128(smem_u32(sB + stage * B_BYTES));
+                    const bool seg8 = kb < p.kb8;
+                    const uint32_t d = tmem_base + (seg8 ? 0u : static_cast<uint32_t>(BN));
+                    const bool first = seg8 ? (kb == 0) : (kb == p.kb8);
+#pragma unroll
+                    for (int k = 0; k < BK / 32; ++k)
+                        mma_i8_ss(d, a_desc + 2 * k, b_desc + 2 * k, idesc, (first && k == 0) ? 0u : 1u);
+                    tc_commit(&sh->empty[stage]);  // frees the ring slot once these MMAs have read it
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                tc_commit(&sh->acc_full);
+                acc_phase ^= 1;
+            }
+            if (!ok) {
+                tc_commit(&sh->drain);
+                const uint64_t t0 = global_timer_ns();
+                while (!mbar_try_wait(&sh->drain, 0) && global_timer_ns() - t0 < 100000000ull) {}
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int quad = warp & 3;  // TMEM lane quadrant this warp may access
+        const int et = threadIdx.x - 64;
+        uint32_t acc_phase = 0;
+        // The 128 epilogue threads meet at named barriers, so they must leave the loop together:
+        // one thread samples the abort flag and the others take its reading.
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+            const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * BN;
+            epi_barrier();  // previous tile's readers of sw8/sw4/epi_stop are done
+            if (et == 0) sh->epi_stop = *abort_flag;
+            for (int j = et; j < BN; j += kEpiThreads) {
+                const int n = n0 + j;
+                sh->sw8[j] = n < p.N ? load_scale(p.s_w8, n, p.w_fp16) : 0.f;
+                sh->sw4[j] = n < p.N ? load_scale(p.s_w4, n, p.w_fp16) : 0.f;
+            }
+            epi_barrier();
+            if (sh->epi_stop) break;
+            const int row = m0 + quad * 32 + lane;
+            const bool row_ok = row < p.T;
+            const float sx8 = row_ok ? __ldg(p.s_x8 + row) : 0.f;
+            const float sx4 = row_ok ? __ldg(p.s_x4 + row) : 0.f;
+            if (!mbar_wait(&sh->acc_full, acc_phase, abort_flag)) continue;  // flag is set; leave at the next sample
+            acc_phase ^= 1;
+            tc_fence_after();
+            const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t a8[32], a4[32];
+                tmem_ld32(lane_addr + c * 32, a8);
+                tmem_ld32(lane_addr + BN + c * 32, a4);
+                tmem_ld_wait();
+                const int nb = n0 + c * 32;
+                if (row_ok) {
+                    const size_t off = static_cast<size_t>(row) * p.N + nb;
+                    if (p.dbg8) {
+#pragma unroll
+                        for (int g = 0; g < 8; ++g)
+                            if (nb + g * 4 < p.N) {
+                                reinterpret_cast<uint4*>(p.dbg8 + off)[g] =
+                                    make_uint4(a8[4 * g], a8[4 * g + 1], a8[4 * g + 2], a8[4 * g + 3]);
+                                reinterpret_cast<uint4*>(p.dbg4 + off)[g] =
+                                    make_uint4(a4[4 * g], a4[4 * g + 1], a4[4 * g + 2], a4[4 * g + 3]);
+                            }
+                    }
+                    float y[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float t8 = static_cast<float>(static_cast<int>(a8[j])) * (sx8 * sh->sw8[c * 32 + j]);
+                        const float t4 = static_cast<float>(static_cast<int>(a4[j])) * (sx4 * sh->sw4[c * 32 + j]);
+                        y[j] = t8 + t4;
+                    }
+                    if (p.y_dtype == RESQ_Y_BF16) {
+                        __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.Y) + off;
+#pragma unroll
+                        for (int g = 0; g < 4; ++g)
+                            if (nb + g * 8 < p.N) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    __nv_bfloat162 h = __floats2bfloat162_rn(y[g * 8 + 2 * q], y[g * 8 + 2 * q + 1]);
+                                    w[q] = *reinterpret_cast<uint32_t*>(&h);
+                                }
+                                reinterpret_cast<uint4*>(yp)[g] = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                    } else {
+                        float* yp = reinterpret_cast<float*>(p.Y) + off;
+#pragma unroll
+                        for (int g = 0; g < 8; ++g)
+                            if (nb + g * 4 < p.N)
+                                reinterpret_cast<float4*>(yp)[g] =
+                                    make_float4(y[4 * g], y[4 * g + 1], y[4 * g + 2], y[4 * g + 3]);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&sh->acc_empty);
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && sh->abort_flag) atomicOr(p.status, RESQ_ERR_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// [rows][kbytes] uint8 matrix, box = 128 bytes x box_rows, 128-byte swizzle, zero fill out of range.
+bool make_map_u8(CUtensorMap* m, const void* base, uint64_t rows, uint64_t kbytes, uint32_t box_rows) {
+    EncodeFn enc = reinterpret_cast<EncodeFn>(tensor_map_encode_fn());
+    if (!enc) return false;
+    cuuint64_t dims[2] = {kbytes, rows};
+    cuuint64_t strides[1] = {kbytes};
+    cuuint32_t box[2] = {128, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8, const int8_t* x4e,
+                                    const float* s_x8, const float* s_x4, const int8_t* w8, const int8_t* w4e,
+                                    const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
+                                    int32_t* dbg8, int32_t* dbg4, cudaStream_t st) {
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 64 && !attr_set[dev]) {
+        e = cudaFuncSetAttribute(mixed_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kSmemBytes));
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    const int K4 = K - r;
+    CUtensorMap tA8, tA4, tB8, tB4;
+    if (!make_map_u8(&tA8, x8, T, r, BM) || !make_map_u8(&tA4, x4e, T, K4, BM) ||
+        !make_map_u8(&tB8, w8, N, r, BN) || !make_map_u8(&tB4, w4e, N, K4, BN))
+        return cudaErrorInvalidValue;
+    Params p;
+    p.T = T; p.N = N; p.r = r; p.K4 = K4;
+    p.m_tiles = (T + BM - 1) / BM;
+    p.n_tiles = (N + BN - 1) / BN;
+    p.kb8 = (r + BK - 1) / BK;
+    p.kb4 = (K4 + BK - 1) / BK;
+    p.s_x8 = s_x8; p.s_x4 = s_x4; p.s_w8 = s_w8; p.s_w4 = s_w4;
+    p.w_fp16 = w_scale_fp16 ? 1 : 0;
+    p.Y = Y; p.y_dtype = y_dtype; p.dbg8 = dbg8; p.dbg4 = dbg8 ? dbg4 : nullptr;
+    p.status = device_status_ptr();
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int tiles = p.m_tiles * p.n_tiles;
+    const int grid = tiles < sms ? tiles : sms;
+    mixed_gemm_kernel<<<grid, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
+    return cudaGetLastError();
+}
+
+}  // namespace resq

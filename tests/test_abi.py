@@ -1,0 +1,91 @@
+"""CPU-side checks of the C ABI: the library loads, exports what the header declares, and validates
+arguments on the host before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def resq():
+    import __graft_entry__
+    __graft_entry__.build()
+    import paper_2412_14363_b200 as m
+    return m
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "resq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(resq_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(resq):
+    names = _declared_functions()
+    assert {"resq_pack_weights", "resq_project_quantize", "resq_mixed_gemm", "resq_linear"} <= set(names)
+    for n in names:
+        assert hasattr(resq.lib, n), n
+    assert sorted(resq.EXPORTS) == names
+
+
+def test_status_strings(resq):
+    assert resq.status_string(0) == "ok"
+    assert "workspace" in resq.status_string(resq.ERR_WORKSPACE)
+    assert resq.status_string(99) == "unknown status"
+
+
+def test_size_queries(resq):
+    d = resq.layer_desc(4096, 4096, 512)
+    assert resq.lib.resq_w8_bytes(ctypes.byref(d)) == 4096 * 512
+    assert resq.lib.resq_w4_bytes(ctypes.byref(d)) == 4096 * 3584 // 2
+    assert resq.lib.resq_w4_i8_bytes(ctypes.byref(d)) == 4096 * 3584
+    assert resq.lib.resq_scale_bytes(ctypes.byref(d)) == 4096 * 4
+    d16 = resq.layer_desc(4096, 4096, 512, resq.SCALE_FP16)
+    assert resq.lib.resq_scale_bytes(ctypes.byref(d16)) == 4096 * 2
+    # one block of the 8B-shaped model packs to 122.9 MB (0.5625 bytes per weight)
+    total = 0
+    for K, N in ((4096, 4096), (4096, 1024), (4096, 1024), (4096, 4096), (4096, 14336), (4096, 14336), (14336, 4096)):
+        dd = resq.layer_desc(K, N, K // 8)
+        total += resq.lib.resq_w8_bytes(ctypes.byref(dd)) + resq.lib.resq_w4_bytes(ctypes.byref(dd))
+    assert abs(total / 1e6 - 122.7) < 0.5
+    assert resq.resq_workspace_bytes(d, 4096, False, True) > 4096 * 3584
+    assert resq.resq_workspace_bytes(d, 4096, True, True) > resq.resq_workspace_bytes(d, 4096, False, True)
+    assert resq.resq_workspace_bytes(resq.layer_desc(4096, 4096, 500), 16, False, True) == 0
+
+
+def test_host_validation_happens_before_any_launch(resq):
+    """Bad arguments are rejected with their status code; none of these calls needs a device."""
+    L = resq.lib
+    good = resq.layer_desc(512, 512, 64)
+    fake = 0x10000  # 16-byte aligned, never dereferenced on the host
+    ws = resq.WeightsStruct(fake, fake, fake, fake, None)
+    W = ctypes.byref(ws)
+    # shape rules
+    for K, N, r in ((512, 512, 0), (512, 512, 512), (512, 512, 48), (500, 512, 64), (512, 508, 64), (0, 8, 0)):
+        bad = resq.layer_desc(K, N, r)
+        assert L.resq_mixed_gemm(ctypes.byref(bad), 16, fake, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
+        assert L.resq_pack_weights(ctypes.byref(bad), fake, fake, fake, fake, fake, None, None) == resq.ERR_SHAPE
+    assert L.resq_mixed_gemm(ctypes.byref(good), 0, fake, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
+    assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake, fake, fake, fake, W, fake, 7, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
+    assert L.resq_project_quantize(fake, None, 16, 512, 60, fake, fake, fake, fake, None, None, 0, None) == resq.ERR_SHAPE
+    # null pointers
+    assert L.resq_mixed_gemm(None, 16, fake, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_NULL
+    assert L.resq_mixed_gemm(ctypes.byref(good), 16, None, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_NULL
+    assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake, fake, fake, fake, W, fake, 0, fake, None, fake, 1 << 30, None) == resq.ERR_NULL
+    assert L.resq_linear(ctypes.byref(good), 16, None, None, W, fake, 0, fake, 1 << 30, None) == resq.ERR_NULL
+    assert L.resq_pack_weights(ctypes.byref(good), None, fake, fake, fake, fake, None, None) == resq.ERR_NULL
+    assert L.resq_project_quantize(fake, None, 16, 512, 64, fake, None, fake, fake, None, None, 0, None) == resq.ERR_NULL
+    wnull = resq.WeightsStruct(fake, None, fake, fake, None)
+    assert L.resq_linear(ctypes.byref(good), 16, fake, None, ctypes.byref(wnull), fake, 0, fake, 1 << 30, None) == resq.ERR_NULL
+    # alignment
+    assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake + 4, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_ALIGN
+    assert L.resq_linear(ctypes.byref(good), 16, fake, None, W, fake + 8, 0, fake, 1 << 30, None) == resq.ERR_ALIGN
+    assert L.resq_project_quantize(fake + 2, None, 16, 512, 64, fake, fake, fake, fake, None, None, 0, None) == resq.ERR_ALIGN
+    # workspace
+    need = resq.resq_workspace_bytes(good, 64, False, False)
+    assert L.resq_mixed_gemm(ctypes.byref(good), 64, fake, fake, fake, fake, W, fake, 0, None, None, fake, need - 1, None) == resq.ERR_WORKSPACE
+    assert L.resq_mixed_gemm(ctypes.byref(good), 64, fake, fake, fake, fake, W, fake, 0, None, None, None, 0, None) == resq.ERR_WORKSPACE
+    assert L.resq_linear(ctypes.byref(good), 64, fake, None, W, fake, 0, fake, 16, None) == resq.ERR_WORKSPACE
