@@ -20,6 +20,7 @@
  */
 #include <math.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 /* ---------- format helpers (bf16 / fp16 are storage formats, widened exactly) ---------- */
@@ -103,12 +104,16 @@ void oracle_unpack_nibbles(const uint8_t* packed, long n, int8_t* code) {
 void oracle_project(const uint16_t* X, const uint16_t* P, long T, int K, float* C) {
 #pragma omp parallel for schedule(static)
     for (long t = 0; t < T; ++t) {
-        for (int j = 0; j < K; ++j) {
-            double acc = 0.0;
-            for (int i = 0; i < K; ++i)
-                acc += (double)bf16_to_f32(X[t * K + i]) * (double)bf16_to_f32(P[(long)i * K + j]);
-            C[t * K + j] = (float)acc;
+        double* acc = (double*)calloc((size_t)K, sizeof(double));
+        /* acc[j] = sum over i (ascending) of X[t][i] * P[i][j]; the i loop is outermost only so that
+         * P is walked along its rows -- each coefficient's sum keeps its order. */
+        for (int i = 0; i < K; ++i) {
+            const double x = (double)bf16_to_f32(X[t * K + i]);
+            const uint16_t* prow = P + (long)i * K;
+            for (int j = 0; j < K; ++j) acc[j] += x * (double)bf16_to_f32(prow[j]);
         }
+        for (int j = 0; j < K; ++j) C[t * K + j] = (float)acc[j];
+        free(acc);
     }
 }
 

@@ -36,7 +36,7 @@ void* tensor_map_encode_fn() {
 namespace {
 
 constexpr int kDecodeMaxT = 0;  // TODO(decode): 16 once the streaming kernel lands
-constexpr int kPanelRows = 512;  // token rows of fp32 coefficients staged per projection panel
+constexpr int kPanelRows = 4096;  // token rows of fp32 coefficients staged per projection panel
 
 inline size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }

@@ -157,3 +157,90 @@ def kron_orthogonal_bf16(K: int, seed: int = SEED_P, inner: int = 128) -> np.nda
         blk = np.kron(qa[i:i + 1, :], qb)  # inner x K
         out[i * inner:(i + 1) * inner, :] = to_bf16_values(blk.astype(np.float32))
     return out
+
+
+# ----------------------------------------------------------------------------
+# The same counter-based streams on a torch device, for full-size workloads (hundreds of millions
+# of draws).  The integer stream is identical to the numpy one; log/cos may differ in the last ulp.
+# ----------------------------------------------------------------------------
+def _s64(x: int) -> int:
+    x &= (1 << 64) - 1
+    return x - (1 << 64) if x >= (1 << 63) else x
+
+
+def _t_lsr(z, k: int):
+    return (z >> k) & ((1 << (64 - k)) - 1)
+
+
+def _t_mix(z):
+    z = (z ^ _t_lsr(z, 30)) * _s64(int(_M1))
+    z = (z ^ _t_lsr(z, 27)) * _s64(int(_M2))
+    return z ^ _t_lsr(z, 31)
+
+
+def t_uniform01(seed: int, stream: int, n: int, offset: int, device):
+    import torch
+    idx = torch.arange(offset, offset + n, dtype=torch.int64, device=device)
+    bits = _t_mix(idx * _s64(int(_GOLD)) + _s64(int(_key(seed, stream))))
+    return (_t_lsr(bits, 11).to(torch.float64) + 0.5) * (1.0 / 9007199254740992.0)
+
+
+def t_normal(seed: int, stream: int, n: int, offset: int, device):
+    import torch
+    u1 = t_uniform01(seed, 2 * stream, n, offset, device)
+    u2 = t_uniform01(seed, 2 * stream + 1, n, offset, device)
+    return torch.sqrt(-2.0 * torch.log(u1)) * torch.cos(2.0 * torch.pi * u2)
+
+
+def t_student_t4(seed: int, stream: int, n: int, offset: int, device):
+    import torch
+    z = t_normal(seed, 8 * stream, n, offset, device)
+    chi = torch.zeros(n, dtype=torch.float64, device=device)
+    for j in range(1, 5):
+        g = t_normal(seed, 8 * stream + j, n, offset, device)
+        chi += g * g
+    return z / torch.sqrt(chi / 4.0)
+
+
+def t_activations(T: int, K: int, device, dist: str = "t4", seed: int = SEED_ACT, stream: int = 0,
+                  scale: float = 20.0, row_offset: int = 0, rows_per_chunk: int = 512):
+    """torch.bfloat16 [T][K] on `device`; same recipe as activations()."""
+    import torch
+    out = torch.empty((T, K), dtype=torch.bfloat16, device=device)
+    ch = torch.from_numpy(outlier_channels(K, n_outliers(K))).to(device)
+    gen = t_normal if dist == "normal" else t_student_t4
+    for t0 in range(0, T, rows_per_chunk):
+        rows = min(rows_per_chunk, T - t0)
+        x = gen(seed, stream, rows * K, (row_offset + t0) * K, device).reshape(rows, K)
+        x[:, ch] *= scale
+        out[t0:t0 + rows] = x.to(torch.float32).to(torch.bfloat16)
+    return out
+
+
+def t_projected_weights_direct(N: int, K: int, device, seed: int = SEED_W, stream: int = 0,
+                               rows_per_chunk: int = 1024):
+    """torch.float32 [N][K] on `device`; same recipe as projected_weights_direct()."""
+    import torch
+    out = torch.empty((N, K), dtype=torch.float32, device=device)
+    inv = 1.0 / float(np.sqrt(float(K)))
+    for n0 in range(0, N, rows_per_chunk):
+        rows = min(rows_per_chunk, N - n0)
+        out[n0:n0 + rows] = (t_normal(seed, stream, rows * K, n0 * K, device) * inv).reshape(rows, K).to(torch.float32)
+    return out
+
+
+def t_kron_orthogonal_bf16(K: int, device, seed: int = SEED_P, inner: int = 128):
+    """torch.bfloat16 [K][K] on `device`; same recipe as kron_orthogonal_bf16()."""
+    import torch
+    assert K % inner == 0
+    a = K // inner
+
+    def haar(n, stream):
+        q, rr = np.linalg.qr(gaussian_matrix(n, seed, stream))
+        return torch.from_numpy(q * np.sign(np.diag(rr))).to(device)
+
+    qa, qb = haar(a, 0), haar(inner, 1)
+    out = torch.empty((K, K), dtype=torch.bfloat16, device=device)
+    for i in range(a):
+        out[i * inner:(i + 1) * inner] = torch.kron(qa[i:i + 1, :], qb).to(torch.float32).to(torch.bfloat16)
+    return out

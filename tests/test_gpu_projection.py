@@ -1,0 +1,87 @@
+"""GPU parity of the online-projection path (C = X·P on the tensor cores, then split quantization).
+
+The oracle sums each coefficient in fp64 and rounds once to fp32; the kernel accumulates bf16
+products in fp32 in another order.  So: every code within +-1 of the oracle's, at most 0.1 % of the
+codes different, scales within a few ulp.  Everything downstream is exact again: feeding the
+kernel's own codes to the oracle's integer product and epilogue must reproduce resq_linear's output.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from tests.gpu_util import bf16_bits_from_dev, bf16_to_dev, dev, host
+from tests.test_gpu_parity import check_output
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def resq():
+    import paper_2412_14363_b200 as m
+    return m
+
+
+def _ulp_diff(a, b):
+    return np.abs(a.view(np.int32).astype(np.int64) - b.view(np.int32).astype(np.int64))
+
+
+@pytest.mark.parametrize("T,K,r,inner", [(16, 512, 64, 128), (200, 1024, 128, 128), (130, 1056, 128, 32),
+                                         (300, 2048, 256, 128), (70, 4096, 512, 128), (4100, 512, 64, 128), (6, 14336, 1792, 128)])
+def test_online_projection_codes(resq, T, K, r, inner):
+    X_bits = synth.f32_to_bf16_bits(synth.activations(T, K, "t4", seed=400 + T))
+    P_bits = synth.f32_to_bf16_bits(synth.kron_orthogonal_bf16(K, inner=inner))
+    C = oracle.project(X_bits, P_bits)
+    q8, q4, o8, o4 = oracle.split_quantize(C, r)
+
+    K4 = K - r
+    desc = resq.layer_desc(K, 8, r)
+    ws = resq.alloc_workspace(desc, T, True, True)
+    x8 = torch.empty((T, r), dtype=torch.int8, device="cuda")
+    x4 = torch.empty((T, K4 // 2), dtype=torch.uint8, device="cuda")
+    x4e = torch.empty((T, K4), dtype=torch.int8, device="cuda")
+    s8 = torch.empty(T, dtype=torch.float32, device="cuda")
+    s4 = torch.empty(T, dtype=torch.float32, device="cuda")
+    resq.resq_project_quantize(bf16_to_dev(X_bits), bf16_to_dev(P_bits), r, x8, x4, s8, s4, x4e, ws)
+    assert resq.resq_device_status() == resq.OK
+    g8, g4 = host(x8).astype(np.int32), host(x4e).astype(np.int32)
+    assert (host(x4) == oracle.pack_nibbles(host(x4e))).all()
+    assert np.abs(g8 - q8).max() <= 1 and np.abs(g4 - q4).max() <= 1
+    frac = ((g8 != q8).sum() + (g4 != q4).sum()) / float(T * K)
+    assert frac <= 1e-3, frac
+    # The tensor core adds each 16-term partial product into the fp32 accumulator with a truncating
+    # add: at most one ulp per instruction, K/16 instructions per coefficient, plus the final roundings.
+    tol = K // 16 + 4
+    assert _ulp_diff(host(s8), o8).max() <= tol and _ulp_diff(host(s4), o4).max() <= tol
+
+
+def test_linear_with_online_projection_is_exact_given_its_own_codes(resq):
+    T, K, N, r = 150, 1024, 520, 128
+    X_bits = synth.f32_to_bf16_bits(synth.activations(T, K, "t4", seed=77))
+    P_bits = synth.f32_to_bf16_bits(synth.kron_orthogonal_bf16(K))
+    Wp = synth.projected_weights_direct(N, K, seed=78)
+    pw = oracle.pack_weights(Wp, r)
+    desc = resq.layer_desc(K, N, r)
+    W = resq.resq_pack_weights(desc, dev(Wp))
+    ws = resq.alloc_workspace(desc, T, True, True)
+    X, P = bf16_to_dev(X_bits), bf16_to_dev(P_bits)
+    K4 = K - r
+    x8 = torch.empty((T, r), dtype=torch.int8, device="cuda")
+    x4e = torch.empty((T, K4), dtype=torch.int8, device="cuda")
+    s8 = torch.empty(T, dtype=torch.float32, device="cuda")
+    s4 = torch.empty(T, dtype=torch.float32, device="cuda")
+    resq.resq_project_quantize(X, P, r, x8, None, s8, s4, x4e, ws)
+    y32 = torch.empty((T, N), dtype=torch.float32, device="cuda")
+    resq.resq_linear(W, X, P, y32, ws)
+    ybf = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    resq.resq_linear(W, X, P, ybf, ws)
+    assert resq.resq_device_status() == resq.OK
+    acc8, acc4 = oracle.int_gemm(host(x8), pw.q8), oracle.int_gemm(host(x4e), pw.q4)
+    e32, ebf = oracle.epilogue(acc8, acc4, host(s8), host(s4), pw.s8, pw.s4)
+    res = oracle.LayerResult(None, host(x8), host(x4e), None, host(s8), host(s4), acc8, acc4, e32, ebf)
+    check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))
+    # and the layer approximates the unquantized product X·P·W_proj^T (this P is a plain rotation, not a
+    # PCA basis, so the error is that of rotation-only 4-bit quantization: a sanity bound, not parity)
+    ref = (synth.bf16_bits_to_f32(X_bits).astype(np.float64) @ synth.bf16_bits_to_f32(P_bits).astype(np.float64)) @ Wp.astype(np.float64).T
+    assert np.linalg.norm(host(y32) - ref) / np.linalg.norm(ref) < 0.35
