@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Roofline benchmark of the ResQ mixed-precision linear layer on B200.
+
+A step is one pass of the whole hot path over one batch: the seven linear layers of one
+Llama-3-8B-shaped decoder block at T = 4096 prefill tokens (q|k|v and gate|up served as one
+N-concatenated layer each; the down_proj input goes through the online bf16 projection), i.e. per
+layer: [projection GEMM] -> per-token split quantization -> mixed INT8/INT4 GEMM with the fp32 scale
+epilogue.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+`--impl reference` times the CPU oracle on a bounded row sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD = "llama3-8b-decoder-block-linears-prefill-T4096"
+T_PREFILL = 4096
+# (name, K, n_out, online projection)
+LAYERS = [("qkv", 4096, 6144, False), ("o", 4096, 4096, False), ("gate_up", 4096, 28672, False),
+          ("down", 14336, 4096, True)]
+ORACLE_SAMPLE_ROWS = 1024      # cpu_baseline leg of our arm: one pass, about 10-20 s of CPU work
+REFERENCE_STEP_ROWS = 64       # --impl reference: rows per step, so that K steps end within minutes
+NOMINAL = {"int8_tops": 4500.0, "bf16_tflops": 2250.0, "hbm_gbs": 7700.0}
+METRIC, UNIT = "prefill tokens/s through one decoder block's ResQ linear layers", "tokens/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"], "bf16_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.gpu_id, self.proc = gpu_id, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            time.sleep(0.3)  # let the first samples start
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        out, _ = self.proc.communicate(timeout=10)
+        sm, mx, pw, reasons = [], [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------- workload
+class Layer:
+    pass
+
+
+def build_layers(device, rows=T_PREFILL, with_weights=True, only=None):
+    """Seeded synthetic inputs of the workload on `device` (activations, projected weights, P)."""
+    import synth
+    layers = []
+    for li, (name, K, N, online) in enumerate(LAYERS):
+        if only and name not in only:
+            continue
+        L = Layer()
+        L.name, L.K, L.N, L.r, L.online = name, K, N, K // 8, online
+        L.X = synth.t_activations(rows, K, device, "t4", seed=synth.SEED_ACT + 10 * li)
+        L.W_proj = synth.t_projected_weights_direct(N, K, device, seed=synth.SEED_W + 10 * li) if with_weights else None
+        L.P = synth.t_kron_orthogonal_bf16(K, device) if online else None
+        layers.append(L)
+    return layers
+
+
+def oracle_sample_step(layers_host):
+    """One pass of the oracle over the sampled rows of every layer; returns the LayerResults."""
+    import oracle
+    out = []
+    for L in layers_host:
+        out.append(oracle.linear(L["X_bits"], L["P_bits"], L["pw"]))
+    return out
+
+
+def to_bits(t):
+    import torch
+    return t.contiguous().view(torch.int16).cpu().numpy().view("uint16")
+
+
+def host_sample(layers, rows):
+    """Copies the first `rows` rows of each layer's input and the full projected weights to the host
+    and quantizes the weights with the oracle (untimed set-up of the CPU baseline)."""
+    import oracle
+    hs = []
+    for L in layers:
+        hs.append({"name": L.name, "X_bits": to_bits(L.X[:rows]), "P_bits": to_bits(L.P) if L.online else None,
+                   "pw": oracle.pack_weights(L.W_proj.cpu().numpy(), L.r)})
+    return hs
+
+
+# --------------------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2412_14363_b200 as resq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    T = T_PREFILL
+
+    only = [x for x in args.layers.split(",") if x]
+    layers = build_layers(dev, only=only)
+    for L in layers:
+        L.desc = resq.layer_desc(L.K, L.N, L.r)
+        L.W = resq.resq_pack_weights(L.desc, L.W_proj, with_w4_i8=True)
+        K4 = L.K - L.r
+        L.x8 = torch.empty((T, L.r), dtype=torch.int8, device=dev)
+        L.x4e = torch.empty((T, K4), dtype=torch.int8, device=dev)
+        L.sx8 = torch.empty(T, dtype=torch.float32, device=dev)
+        L.sx4 = torch.empty(T, dtype=torch.float32, device=dev)
+        L.Y = torch.empty((T, L.N), dtype=torch.bfloat16, device=dev)
+        L.ws = resq.alloc_workspace(L.desc, T, L.online, True, device=dev)
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    # One step; with `events` an event is recorded after every C-ABI call so that each kernel's time
+    # is measured live on the launching stream.
+    # Launches per step: 4 split-quantize + 1 projection GEMM + 4 mixed GEMM = 9 kernels of this library.
+    LAUNCHES_PER_STEP = sum(3 if L.online else 2 for L in layers)
+
+    def step(events=None):
+        for L in layers:
+            e0 = ev() if events is not None else None
+            resq.resq_project_quantize(L.X, L.P, L.r, L.x8, None, L.sx8, L.sx4, L.x4e, L.ws if L.online else None)
+            e1 = ev() if events is not None else None
+            resq.resq_mixed_gemm(L.W, L.x8, None, L.sx8, L.sx4, L.Y, L.ws, x4_i8=L.x4e)
+            if events is not None:
+                events.append((L.name, e0, e1, ev()))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    st = resq.resq_device_status()
+    if st != resq.OK:
+        raise SystemExit(f"device status {st}: {resq.status_string(st)}")
+
+    gpu_id = str(getattr(torch.cuda.get_device_properties(dev), "uuid", local_rank))
+    if not gpu_id.startswith("GPU-") and "-" in gpu_id:
+        gpu_id = "GPU-" + gpu_id
+    sampler = ClockSampler(gpu_id)
+    sampler.start()
+    events = []
+    barrier()
+    t_start = ev()
+    for _ in range(args.steps):
+        step(events)
+    t_end = ev()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = t_start.elapsed_time(t_end)
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * T / (ms_per_step * 1e-3)
+
+    # ---- per-kernel times (this rank), averaged over the timed steps
+    kq = {L.name: [] for L in layers}
+    kg = {L.name: [] for L in layers}
+    for name, e0, e1, e2 in events:
+        kq[name].append(e0.elapsed_time(e1))
+        kg[name].append(e1.elapsed_time(e2))
+    per_layer = {}
+    gemm_ops = gemm_ms = 0.0
+    quant_bytes = quant_ms = 0.0
+    for L in layers:
+        q_ms, g_ms = statistics.mean(kq[L.name]), statistics.mean(kg[L.name])
+        ops = 2.0 * T * L.K * L.N
+        per_layer[L.name] = {"K": L.K, "N": L.N, "quantize_ms": round(q_ms, 4), "mixed_gemm_ms": round(g_ms, 4),
+                             "mixed_gemm_tops": round(ops / (g_ms * 1e-3) / 1e12, 1)}
+        gemm_ops += ops
+        gemm_ms += g_ms
+        if not L.online:
+            # per token: read 2K bytes of bf16, write r + (K - r) codes + 8 bytes of scales
+            quant_bytes += T * (2.0 * L.K + L.K + 8)
+            quant_ms += q_ms
+    online = [L for L in layers if L.online]
+    proj_ms = sum(per_layer[L.name]["quantize_ms"] for L in online)  # projection GEMM + its split-quantize pass
+    proj_flops = sum(2.0 * T * L.K * L.K for L in online)
+    timed_seconds = ms_total * 1e-3
+    bf16_peak = peaks["bf16_sustained"] if timed_seconds > 1.0 else peaks["bf16_burst"]
+    peak_kind = ("sustained" if timed_seconds > 1.0 else "burst") + " of " + peaks["source"]
+    int8_peak = 2.0 * bf16_peak  # no measured INT8 figure: measured bf16 peak x nominal INT8/bf16 ratio (4500/2250)
+    kernels = {
+        "mixed_gemm": {"bound": "tensor", "dtype": "int8", "achieved": round(gemm_ops / (gemm_ms * 1e-3) / 1e12, 1),
+                       "peak": round(int8_peak, 1), "unit": "TOP/s", "ms_per_step": round(gemm_ms, 4),
+                       "frac_of_nominal_4500": round(gemm_ops / (gemm_ms * 1e-3) / 1e12 / NOMINAL["int8_tops"], 4)},
+    }
+    if online:
+        kernels["project_gemm+quantize"] = {"bound": "tensor", "dtype": "bf16",
+                                            "achieved": round(proj_flops / (proj_ms * 1e-3) / 1e12, 1),
+                                            "peak": round(bf16_peak, 1), "unit": "TFLOP/s", "ms_per_step": round(proj_ms, 4)}
+    if quant_ms > 0:
+        kernels["split_quantize"] = {"bound": "hbm", "dtype": "f32",
+                                     "achieved": round(quant_bytes / (quant_ms * 1e-3) / 1e9, 1),
+                                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "ms_per_step": round(quant_ms, 4)}
+    for k in kernels.values():
+        k["frac"] = round(k["achieved"] / k["peak"], 4)
+    dom_name = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    dom = kernels[dom_name]
+    roofline = {"kernel": dom_name, "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
+                "unit": dom["unit"], "frac": dom["frac"], "traffic": None, "peak_kind": peak_kind,
+                "kernels": kernels}
+
+    # ---- end to end through the public whole-layer call with host buffers
+    e2e = None
+    if not args.no_e2e:
+        hx = [torch.empty(L.X.shape, dtype=torch.bfloat16).pin_memory() for L in layers]
+        hy = [torch.empty(L.Y.shape, dtype=torch.bfloat16).pin_memory() for L in layers]
+        for h, L in zip(hx, layers):
+            h.copy_(L.X)
+        dx = [torch.empty_like(L.X) for L in layers]
+        h2d = sum(h.numel() * 2 for h in hx)
+        d2h = sum(h.numel() * 2 for h in hy)
+
+        def e2e_step():
+            for i, L in enumerate(layers):
+                dx[i].copy_(hx[i], non_blocking=True)
+                resq.resq_linear(L.W, dx[i], L.P, L.Y, L.ws)
+                hy[i].copy_(L.Y, non_blocking=True)
+
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        e_steps = max(3, min(args.steps, 10))
+        s0 = ev()
+        for _ in range(e_steps):
+            e2e_step()
+        s1 = ev()
+        barrier()
+        e_ms = s0.elapsed_time(s1)
+        if world > 1:
+            t = torch.tensor([e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": round(world * T / (e_ms / e_steps * 1e-3), 1), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": round(e_ms / e_steps, 4), "steps": e_steps}
+    st = resq.resq_device_status()
+    if st != resq.OK:
+        raise SystemExit(f"device status {st}: {resq.status_string(st)}")
+
+    # ---- CPU baseline: the oracle on a row sample, rank 0 at N = 1 only; also a parity spot check
+    cpu_baseline, parity = None, None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        S = min(ORACLE_SAMPLE_ROWS, T)
+        hs = host_sample(layers, S)
+        t0 = time.perf_counter()
+        res = oracle_sample_step(hs)
+        dt = time.perf_counter() - t0
+        cpu_baseline = {"value": round(S / dt, 2), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                        "sample": f"first {S} of {T} token rows through all four fused layers "
+                                  f"(incl. the fp64 online projection), {dt:.1f} s"}
+        # GPU outputs of the last step against the oracle on the sampled rows (folded layers: exact path)
+        worst = 0.0
+        for L, h, r_ in zip(layers, hs, res):
+            if L.online:
+                continue
+            y = L.Y[:S].float().cpu().numpy()
+            mag = (np.abs(r_.acc8.astype(np.float64) * r_.s_x8[:, None] * h["pw"].s8[None, :])
+                   + np.abs(r_.acc4.astype(np.float64) * r_.s_x4[:, None] * h["pw"].s4[None, :]))
+            # bf16 output: half an ulp of bf16 (2^-9 relative) on top of the fp32 tolerance
+            worst = max(worst, float((np.abs(y - r_.y32) / (np.abs(r_.y32) * 2.0 ** -8 + 1e-5 * mag + 1e-30)).max()))
+        parity = {"sampled_rows": S, "folded_layers_within_tolerance": bool(worst <= 1.0)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "tokens_per_step_per_gpu": T,
+                       "layers": {n: [k, o] for n, k, o, _ in LAYERS}, "r": "K/8",
+                       "l2": "working set per step (weights 0.2 GB + P 0.41 GB + activations) exceeds the 126 MB L2",
+                       "parallelism": f"replicas x{world}, no collective"},
+            "mixed_gemm_tops": kernels["mixed_gemm"]["achieved"],
+            "mixed_gemm_frac_of_int8_peak": {"vs_measured_bf16_x2": kernels["mixed_gemm"]["frac"],
+                                             "vs_nominal_4500": kernels["mixed_gemm"]["frac_of_nominal_4500"]},
+            "per_layer": per_layer,
+            "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline, "parity_spot_check": parity,
+            "gpu_launches": LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import torch
+
+    import oracle
+    dev = torch.device("cuda", 0) if torch.cuda.is_available() else torch.device("cpu")
+    S = REFERENCE_STEP_ROWS
+    layers = build_layers(dev, rows=S)
+    hs = host_sample(layers, S)
+    del layers
+    W = max(args.warmup, 1)
+    for _ in range(W):
+        oracle_sample_step(hs)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_step(hs)
+    dt = (time.perf_counter() - t0) / args.steps
+    v = round(S / dt, 2)
+    sample = f"first {S} of {T_PREFILL} token rows through all four fused layers per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": W, "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--layers", default="", help="comma-separated subset of qkv,o,gate_up,down (profiling runs)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

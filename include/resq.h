@@ -118,10 +118,15 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
  *     y = (float)acc8 * (s_x8[t] * s_w8[n]) + (float)acc4 * (s_x4[t] * s_w4[n])
  * rounded to bf16 (nearest even) when y_dtype == RESQ_Y_BF16.  Y is [T][n_out].
  * T <= 16 runs the weight-streaming split-K kernel, larger T the tensor-core tile kernel.
+ * The INT4 activation codes come packed (x4, uint8 [T][(K-r)/2]) and/or one per byte (x4_i8, int8
+ * [T][K-r], as resq_project_quantize can emit them).  The streaming kernel reads x4, so x4 is
+ * required when T <= 16; the tile kernel reads x4_i8 and, if only x4 is given, first expands it
+ * into the workspace.  At least one of the two must be non-NULL.
  * dbg_acc8 / dbg_acc4: optional int32 [T][n_out] dumps of the two accumulators (NULL = off).
  */
 int resq_mixed_gemm(const resq_layer_desc_t* desc, int T, const int8_t* x8, const uint8_t* x4,
-                    const float* s_x8, const float* s_x4, const resq_weights_t* W, void* Y, int y_dtype,
+                    const int8_t* x4_i8, const float* s_x8, const float* s_x4, const resq_weights_t* W,
+                    void* Y, int y_dtype,
                     int32_t* dbg_acc8, int32_t* dbg_acc4, void* workspace, size_t workspace_bytes,
                     void* stream);
 

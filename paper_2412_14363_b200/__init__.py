@@ -56,7 +56,7 @@ lib.resq_workspace_bytes.restype = _sz
 lib.resq_workspace_bytes.argtypes = [_dp, _i, _i, _i]
 lib.resq_pack_weights.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_project_quantize.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
-lib.resq_mixed_gemm.argtypes = [_dp, _i, _vp, _vp, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _i, _vp, _vp,
+lib.resq_mixed_gemm.argtypes = [_dp, _i, _vp, _vp, _vp, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _i, _vp, _vp,
                                 _vp, _sz, _vp]
 lib.resq_linear.argtypes = [_dp, _i, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _i, _vp, _sz, _vp]
 lib.resq_unpack_int4.argtypes = [_vp, _vp, _sz, _sz, _vp]
@@ -133,12 +133,12 @@ def resq_project_quantize(X, P, r: int, x8, x4, s_x8, s_x4, x4_i8=None, workspac
                                      _stream()), "resq_project_quantize")
 
 
-def resq_mixed_gemm(W: Weights, x8, x4, s_x8, s_x4, Y, workspace, dbg_acc8=None, dbg_acc4=None):
+def resq_mixed_gemm(W: Weights, x8, x4, s_x8, s_x4, Y, workspace, dbg_acc8=None, dbg_acc4=None, x4_i8=None):
     import torch
     T = x8.shape[0]
     y_dtype = Y_BF16 if Y.dtype == torch.bfloat16 else Y_FP32
     ws = W.struct()
-    _check(lib.resq_mixed_gemm(ctypes.byref(W.desc), T, _ptr(x8), _ptr(x4), _ptr(s_x8), _ptr(s_x4),
+    _check(lib.resq_mixed_gemm(ctypes.byref(W.desc), T, _ptr(x8), _ptr(x4), _ptr(x4_i8), _ptr(s_x8), _ptr(s_x4),
                                ctypes.byref(ws), _ptr(Y), y_dtype, _ptr(dbg_acc8), _ptr(dbg_acc4), _ptr(workspace),
                                0 if workspace is None else workspace.numel() * workspace.element_size(),
                                _stream()), "resq_mixed_gemm")

@@ -35,7 +35,7 @@ void* tensor_map_encode_fn() {
 
 namespace {
 
-constexpr int kDecodeMaxT = 0;  // TODO(decode): 16 once the streaming kernel lands
+constexpr int kDecodeMaxT = 16;  // up to here the weight-streaming kernel runs, above it the tile kernel
 constexpr int kPanelRows = 4096;  // token rows of fp32 coefficients staged per projection panel
 
 inline size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
@@ -187,21 +187,22 @@ static int check_weights(const resq_weights_t* W) {
     return RESQ_OK;
 }
 
-int resq_mixed_gemm(const resq_layer_desc_t* d, int T, const int8_t* x8, const uint8_t* x4, const float* s_x8,
-                    const float* s_x4, const resq_weights_t* W, void* Y, int y_dtype, int32_t* dbg_acc8,
-                    int32_t* dbg_acc4, void* workspace, size_t workspace_bytes, void* stream) {
+int resq_mixed_gemm(const resq_layer_desc_t* d, int T, const int8_t* x8, const uint8_t* x4, const int8_t* x4_i8,
+                    const float* s_x8, const float* s_x4, const resq_weights_t* W, void* Y, int y_dtype,
+                    int32_t* dbg_acc8, int32_t* dbg_acc4, void* workspace, size_t workspace_bytes, void* stream) {
     if (int e = check_desc(d)) return e;
     if (T < 1 || (y_dtype != RESQ_Y_BF16 && y_dtype != RESQ_Y_FP32)) return RESQ_ERR_SHAPE;
-    if (!x8 || !x4 || !s_x8 || !s_x4 || !Y) return RESQ_ERR_NULL;
+    if (!x8 || !s_x8 || !s_x4 || !Y) return RESQ_ERR_NULL;
+    if (!x4 && (!x4_i8 || T <= kDecodeMaxT)) return RESQ_ERR_NULL;
     if ((dbg_acc8 == nullptr) != (dbg_acc4 == nullptr)) return RESQ_ERR_NULL;
     if (int e = check_weights(W)) return e;
-    if (!aligned16(x8) || !aligned16(x4) || !aligned16(s_x8) || !aligned16(s_x4) || !aligned16(Y) ||
-        !aligned16(dbg_acc8) || !aligned16(dbg_acc4) || !aligned16(workspace))
+    if (!aligned16(x8) || !aligned16(x4) || !aligned16(x4_i8) || !aligned16(s_x8) || !aligned16(s_x4) ||
+        !aligned16(Y) || !aligned16(dbg_acc8) || !aligned16(dbg_acc4) || !aligned16(workspace))
         return RESQ_ERR_ALIGN;
     const Workspace map = carve(d->K, d->n_out, d->r, T, false, W->w4_i8 != nullptr);
     if (!workspace || workspace_bytes < map.total) return RESQ_ERR_WORKSPACE;
     if (int e = check_arch()) return e;
-    return mixed_gemm_impl(d, T, x8, x4, nullptr, s_x8, s_x4, W, Y, y_dtype, dbg_acc8, dbg_acc4,
+    return mixed_gemm_impl(d, T, x8, x4, x4_i8, s_x8, s_x4, W, Y, y_dtype, dbg_acc8, dbg_acc4,
                            static_cast<char*>(workspace), map, static_cast<cudaStream_t>(stream));
 }
 

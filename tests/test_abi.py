@@ -66,26 +66,26 @@ def test_host_validation_happens_before_any_launch(resq):
     # shape rules
     for K, N, r in ((512, 512, 0), (512, 512, 512), (512, 512, 48), (500, 512, 64), (512, 508, 64), (0, 8, 0)):
         bad = resq.layer_desc(K, N, r)
-        assert L.resq_mixed_gemm(ctypes.byref(bad), 16, fake, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
+        assert L.resq_mixed_gemm(ctypes.byref(bad), 16, fake, fake, None, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
         assert L.resq_pack_weights(ctypes.byref(bad), fake, fake, fake, fake, fake, None, None) == resq.ERR_SHAPE
-    assert L.resq_mixed_gemm(ctypes.byref(good), 0, fake, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
-    assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake, fake, fake, fake, W, fake, 7, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
+    assert L.resq_mixed_gemm(ctypes.byref(good), 0, fake, fake, None, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
+    assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake, fake, None, fake, fake, W, fake, 7, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
     assert L.resq_project_quantize(fake, None, 16, 512, 60, fake, fake, fake, fake, None, None, 0, None) == resq.ERR_SHAPE
     # null pointers
-    assert L.resq_mixed_gemm(None, 16, fake, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_NULL
-    assert L.resq_mixed_gemm(ctypes.byref(good), 16, None, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_NULL
-    assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake, fake, fake, fake, W, fake, 0, fake, None, fake, 1 << 30, None) == resq.ERR_NULL
+    assert L.resq_mixed_gemm(None, 16, fake, fake, None, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_NULL
+    assert L.resq_mixed_gemm(ctypes.byref(good), 16, None, fake, None, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_NULL
+    assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake, fake, None, fake, fake, W, fake, 0, fake, None, fake, 1 << 30, None) == resq.ERR_NULL
     assert L.resq_linear(ctypes.byref(good), 16, None, None, W, fake, 0, fake, 1 << 30, None) == resq.ERR_NULL
     assert L.resq_pack_weights(ctypes.byref(good), None, fake, fake, fake, fake, None, None) == resq.ERR_NULL
     assert L.resq_project_quantize(fake, None, 16, 512, 64, fake, None, fake, fake, None, None, 0, None) == resq.ERR_NULL
     wnull = resq.WeightsStruct(fake, None, fake, fake, None)
     assert L.resq_linear(ctypes.byref(good), 16, fake, None, ctypes.byref(wnull), fake, 0, fake, 1 << 30, None) == resq.ERR_NULL
     # alignment
-    assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake + 4, fake, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_ALIGN
+    assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake + 4, fake, None, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_ALIGN
     assert L.resq_linear(ctypes.byref(good), 16, fake, None, W, fake + 8, 0, fake, 1 << 30, None) == resq.ERR_ALIGN
     assert L.resq_project_quantize(fake + 2, None, 16, 512, 64, fake, fake, fake, fake, None, None, 0, None) == resq.ERR_ALIGN
     # workspace
     need = resq.resq_workspace_bytes(good, 64, False, False)
-    assert L.resq_mixed_gemm(ctypes.byref(good), 64, fake, fake, fake, fake, W, fake, 0, None, None, fake, need - 1, None) == resq.ERR_WORKSPACE
-    assert L.resq_mixed_gemm(ctypes.byref(good), 64, fake, fake, fake, fake, W, fake, 0, None, None, None, 0, None) == resq.ERR_WORKSPACE
+    assert L.resq_mixed_gemm(ctypes.byref(good), 64, fake, fake, None, fake, fake, W, fake, 0, None, None, fake, need - 1, None) == resq.ERR_WORKSPACE
+    assert L.resq_mixed_gemm(ctypes.byref(good), 64, fake, fake, None, fake, fake, W, fake, 0, None, None, None, 0, None) == resq.ERR_WORKSPACE
     assert L.resq_linear(ctypes.byref(good), 64, fake, None, W, fake, 0, fake, 16, None) == resq.ERR_WORKSPACE

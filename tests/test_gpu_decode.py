@@ -1,0 +1,72 @@
+"""GPU parity of the few-token (T <= 16) weight-streaming kernel: int32 accumulators bit-exact for every
+K split, fp32 epilogue within tolerance, packed canonical weights with fp16 scales (the decode config)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from tests.gpu_util import bf16_bits_from_dev, bf16_to_dev, dev, host
+from tests.test_gpu_parity import check_output, oracle_case, run_mixed_gemm
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def resq():
+    import paper_2412_14363_b200 as m
+    return m
+
+
+@pytest.mark.parametrize("T,K,N,r,fp16", [
+    (1, 4096, 4096, 512, True),     # o_proj shape, one token (K split over a cluster of 8)
+    (4, 4096, 1024, 512, True),
+    (16, 4096, 4096, 512, True),
+    (9, 2048, 264, 256, False),     # ragged channel block, second token tile partly filled
+    (8, 512, 512, 64, False),       # r < one 64-byte step
+    (16, 14336, 128, 1792, True),   # down_proj reduction length, few channels
+    (3, 1056, 72, 96, False),       # segment lengths that are not multiples of a step
+    (16, 4096, 28672, 512, True),   # gate|up: enough channel blocks that K is not split
+])
+def test_decode_bit_exact(resq, T, K, N, r, fp16):
+    _, _, pw, res = oracle_case(T, K, N, r, fp16, seed_shift=50 + T)
+    a8, a4, y32, ybf = run_mixed_gemm(resq, pw, res, fp16, with_w4_i8=False)
+    assert (a8 == res.acc8).all()
+    assert (a4 == res.acc4).all()
+    check_output(res, pw, y32, ybf)
+
+
+def test_decode_extreme_codes(resq):
+    T, K, N, r = 16, 2048, 192, 256
+    K4 = K - r
+    x8 = np.full((T, r), -128, np.int8)
+    x4 = np.full((T, K4), -8, np.int8)
+    x4[:, 1::2] = 7
+    q4 = np.full((N, K4), -8, np.int8)
+    q4[::2, ::3] = 7
+    pw = oracle.PackedWeights(K, N, r, np.full((N, r), -128, np.int8), q4, oracle.pack_nibbles(q4),
+                              np.full(N, 0.01, np.float32), np.full(N, 0.1, np.float32))
+    acc8, acc4 = oracle.int_gemm(x8, pw.q8), oracle.int_gemm(x4, pw.q4)
+    sx8, sx4 = np.full(T, 0.5, np.float32), np.full(T, 2.0, np.float32)
+    y32, ybf = oracle.epilogue(acc8, acc4, sx8, sx4, pw.s8, pw.s4)
+    res = oracle.LayerResult(None, x8, x4, oracle.pack_nibbles(x4), sx8, sx4, acc8, acc4, y32, ybf)
+    a8, a4, y, yb = run_mixed_gemm(resq, pw, res, with_w4_i8=False)
+    assert (a8 == acc8).all() and (a4 == acc4).all()
+    check_output(res, pw, y, yb)
+
+
+@pytest.mark.parametrize("T", [1, 16])
+def test_decode_linear_end_to_end(resq, T):
+    """resq_linear for few tokens: quantize kernel + streaming kernel, packed weights only."""
+    K, N, r = 4096, 1024, 512
+    C_bits, Wp, _, _ = oracle_case(T, K, N, r, True, seed_shift=70 + T)
+    pw = oracle.pack_weights(Wp, r, scale_fp16=True)
+    res = oracle.linear(C_bits, None, pw)
+    desc = resq.layer_desc(K, N, r, resq.SCALE_FP16)
+    W = resq.resq_pack_weights(desc, dev(Wp), with_w4_i8=False)
+    ws = resq.alloc_workspace(desc, T, False, False)
+    y32 = torch.empty((T, N), dtype=torch.float32, device="cuda")
+    resq.resq_linear(W, bf16_to_dev(C_bits), None, y32, ws)
+    ybf = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    resq.resq_linear(W, bf16_to_dev(C_bits), None, ybf, ws)
+    assert resq.resq_device_status() == resq.OK
+    check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))

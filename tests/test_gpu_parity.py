@@ -127,7 +127,7 @@ def run_mixed_gemm(resq, pw, res, fp16=False, with_w4_i8=True, W=None):
     y32 = torch.full((T, pw.N), float("nan"), dtype=torch.float32, device="cuda")
     a8 = torch.full((T, pw.N), -1, dtype=torch.int32, device="cuda")
     a4 = torch.full((T, pw.N), -1, dtype=torch.int32, device="cuda")
-    resq.resq_mixed_gemm(W, x8, x4, s8, s4, y32, ws, a8, a4)
+    resq.resq_mixed_gemm(W, x8, x4, s8, s4, y32, ws, a8, a4)  # packed activations in
     ybf = torch.zeros((T, pw.N), dtype=torch.bfloat16, device="cuda")
     resq.resq_mixed_gemm(W, x8, x4, s8, s4, ybf, ws)
     _check_status(resq)
