@@ -138,6 +138,29 @@ int resq_linear(const resq_layer_desc_t* desc, int T, const void* X, const void*
                 const resq_weights_t* W, void* Y, int y_dtype, void* workspace, size_t workspace_bytes,
                 void* stream);
 
+/*
+ * (No counterpart in the paper: a deployment aid.)  Same result as resq_project_quantize with
+ * P != NULL, for callers that cannot allocate device memory at all -- a server whose start-up code
+ * gave the whole GPU to its own pool, a plug-in living inside another program's memory plan, a
+ * real-time loop that cannot afford cudaMalloc's device-wide synchronisation.  The fp32 staging panel
+ * that the regular call takes from the caller's workspace is instead a fixed array of
+ * RESQ_STATIC_SCRATCH_BYTES built into the library (each GPU that loads the library holds it until
+ * the process exits).  The call allocates nothing, frees nothing and takes no workspace argument;
+ * inputs and outputs are still the caller's buffers, with the meanings and layouts of
+ * resq_project_quantize.
+ *  - Limit: T * K * 4 bytes must not exceed RESQ_STATIC_SCRATCH_BYTES (K = 4096: T <= 512; K = 14336:
+ *    T <= 146; K = 28672: T <= 73); beyond it the call returns RESQ_ERR_WORKSPACE and launches nothing.
+ *    P must be non-NULL (without a projection no scratch is needed: use resq_project_quantize).
+ *  - The first call on each device looks up the array's device address (and sets a kernel
+ *    attribute); make that first call outside any stream capture, with that device current.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call wrote.  Nothing
+ *    in it needs clearing (each call overwrites every element it later reads), but two calls that
+ *    overlap on the GPU -- different streams, no ordering between them -- race on it: order them.
+ */
+#define RESQ_STATIC_SCRATCH_BYTES (8u << 20)
+int resq_project_quantize_static(const void* X, const void* P, int T, int K, int r, int8_t* x8, uint8_t* x4,
+                                 float* s_x8, float* s_x4, int8_t* x4_i8, void* stream);
+
 /* Inverse of the INT4 packing, for inspection: packed [rows][cols/2] -> int8 [rows][cols]. */
 int resq_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, void* stream);
 

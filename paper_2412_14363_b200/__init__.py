@@ -21,7 +21,8 @@ Y_BF16, Y_FP32 = 0, 1
 
 EXPORTS = [
     "resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_bytes", "resq_workspace_bytes",
-    "resq_pack_weights", "resq_project_quantize", "resq_mixed_gemm", "resq_linear", "resq_unpack_int4",
+    "resq_pack_weights", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
+    "resq_unpack_int4",
     "resq_device_status", "resq_status_string",
 ]
 
@@ -43,7 +44,7 @@ class WeightsStruct(ctypes.Structure):
 
 
 if not os.path.exists(LIB_PATH):
-    raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2412_14363_b200.build` "
+    raise ImportError(f"{LIB_PATH} not found: build it with `python __graft_entry__.py` "
                       "(there is no CPU or PyTorch fallback)")
 lib = ctypes.CDLL(LIB_PATH)
 
@@ -56,6 +57,7 @@ lib.resq_workspace_bytes.restype = _sz
 lib.resq_workspace_bytes.argtypes = [_dp, _i, _i, _i]
 lib.resq_pack_weights.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_project_quantize.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.resq_project_quantize_static.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_mixed_gemm.argtypes = [_dp, _i, _vp, _vp, _vp, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _i, _vp, _vp,
                                 _vp, _sz, _vp]
 lib.resq_linear.argtypes = [_dp, _i, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _i, _vp, _sz, _vp]
@@ -131,6 +133,19 @@ def resq_project_quantize(X, P, r: int, x8, x4, s_x8, s_x4, x4_i8=None, workspac
                                      _ptr(x4_i8), _ptr(workspace),
                                      0 if workspace is None else workspace.numel() * workspace.element_size(),
                                      _stream()), "resq_project_quantize")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def resq_project_quantize_static(X, P, r: int, x8, x4, s_x8, s_x4, x4_i8=None):
+    """resq_project_quantize with P given, for callers that cannot allocate a workspace (a process whose
+    memory is all owned by another pool, or a loop that must not hit cudaMalloc's device-wide sync):
+    the fp32 staging panel is an 8 MiB array inside the library, so T * K * 4 must fit in it.  Calls
+    share that array: do not let two of them overlap on the GPU."""
+    T, K = X.shape
+    _check(lib.resq_project_quantize_static(_ptr(X), _ptr(P), T, K, r, _ptr(x8), _ptr(x4), _ptr(s_x8), _ptr(s_x4),
+                                            _ptr(x4_i8), _stream()), "resq_project_quantize_static")
 
 
 def resq_mixed_gemm(W: Weights, x8, x4, s_x8, s_x4, Y, workspace, dbg_acc8=None, dbg_acc4=None, x4_i8=None):

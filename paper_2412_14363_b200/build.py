@@ -1,4 +1,4 @@
-"""Builds libresq.so (sm_100a) in-tree with nvcc.  `python -m paper_2412_14363_b200.build [--force]`."""
+"""Builds libresq.so (sm_100a) in-tree with nvcc.  `python paper_2412_14363_b200/build.py [--force] [-v]` (or `python __graft_entry__.py`)."""
 from __future__ import annotations
 
 import os
@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libresq.so")
-SOURCES = ["api.cu", "quantize.cu", "mixed_gemm.cu", "decode.cu", "project.cu"]
+SOURCES = ["api.cu", "quantize.cu", "mixed_gemm.cu", "decode.cu", "project.cu", "static_scratch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
