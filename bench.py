@@ -130,6 +130,83 @@ def host_sample(layers, rows):
     return hs
 
 
+# --------------------------------------------------------------------------------------- decode leg
+DECODE_T = (1, 4, 16)
+DECODE_COPIES = 3  # distinct copies of the packed weights, cycled per step: one block's 123 MB would sit in the 126 MB L2
+
+
+def decode_leg(resq, torch, dev, peaks, layers, steps):
+    """Few-token variant of the same block: packed INT8 + nibble-packed INT4 weights with fp16 scales,
+    streamed once per step.  Reports the weight-stream rate of the mixed GEMV kernels against the HBM
+    peak, the P stream of the online projection separately, and the latency of the block's linears."""
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    sets, weight_bytes = [], 0
+    for L in layers:
+        desc = resq.layer_desc(L.K, L.N, L.r, resq.SCALE_FP16)
+        base = resq.resq_pack_weights(desc, L.W_proj, with_w4_i8=False)
+        copies = [base] + [resq.Weights(desc, base.w8.clone(), base.w4.clone(), base.s_w8.clone(), base.s_w4.clone())
+                           for _ in range(DECODE_COPIES - 1)]
+        sets.append((L, desc, copies))
+        weight_bytes += L.N * (L.r + (L.K - L.r) // 2) + 2 * 2 * L.N
+    p_bytes = sum(2 * L.K * L.K for L in layers if L.online)
+    out = {"workload": "llama3-8b-decoder-block-linears-decode", "weight_bytes_per_step": weight_bytes,
+           "p_bytes_per_step": p_bytes, "weight_copies_cycled": DECODE_COPIES, "steps": steps}
+    for T in DECODE_T:
+        bufs = []
+        for L, desc, _ in sets:
+            K4 = L.K - L.r
+            bufs.append(dict(X=L.X[:T].contiguous(), x8=torch.empty((T, L.r), dtype=torch.int8, device=dev),
+                             x4=torch.empty((T, K4 // 2), dtype=torch.uint8, device=dev),
+                             sx8=torch.empty(T, dtype=torch.float32, device=dev),
+                             sx4=torch.empty(T, dtype=torch.float32, device=dev),
+                             Y=torch.empty((T, L.N), dtype=torch.bfloat16, device=dev),
+                             ws=resq.alloc_workspace(desc, T, L.online, False, device=dev)))
+
+        def step(i, events=None):
+            for (L, desc, copies), b in zip(sets, bufs):
+                e0 = ev() if events is not None else None
+                resq.resq_project_quantize(b["X"], L.P, L.r, b["x8"], b["x4"], b["sx8"], b["sx4"], None,
+                                           b["ws"] if L.online else None)
+                e1 = ev() if events is not None else None
+                resq.resq_mixed_gemm(copies[i % DECODE_COPIES], b["x8"], b["x4"], b["sx8"], b["sx4"], b["Y"], b["ws"])
+                if events is not None:
+                    events.append((L, e0, e1, ev()))
+
+        for i in range(3):
+            step(i)
+        torch.cuda.synchronize()
+        events = []
+        torch.cuda._sleep(3_000_000)  # the host queues the whole batch while the device idles on this
+        t0 = ev()
+        for i in range(steps):
+            step(i, events)
+        t1 = ev()
+        torch.cuda.synchronize()
+        gemv = sum(e1.elapsed_time(e2) for _, _, e1, e2 in events) / steps
+        quant = sum(e0.elapsed_time(e1) for L, e0, e1, _ in events if not L.online) / steps
+        proj = sum(e0.elapsed_time(e1) for L, e0, e1, _ in events if L.online) / steps
+        total = t0.elapsed_time(t1) / steps
+        gbs = weight_bytes / (gemv * 1e-3) / 1e9
+        out[f"T{T}"] = {"mixed_gemv_us": round(gemv * 1e3, 2), "weight_stream_gbs": round(gbs, 1),
+                        "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
+                        "frac_of_nominal_8000": round(gbs / 8000.0, 4),
+                        "folded_quantize_us": round(quant * 1e3, 2),
+                        "online_projection_us": round(proj * 1e3, 2),
+                        "online_projection_p_stream_gbs": round(p_bytes / (proj * 1e-3) / 1e9, 1) if proj > 0 else None,
+                        "block_linears_us": round(total * 1e3, 2),
+                        "tokens_per_s": round(T / (total * 1e-3), 1)}
+    st = resq.resq_device_status()
+    if st != resq.OK:
+        raise SystemExit(f"device status {st}: {resq.status_string(st)}")
+    return out
+
+
 # --------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import numpy as np
@@ -187,6 +264,10 @@ def run_ours(args):
         if world > 1:
             dist.barrier()
             torch.cuda.synchronize()
+
+    if args.decode_only:  # profiling runs: the few-token leg alone
+        print(json.dumps({"decode": decode_leg(resq, torch, dev, peaks, layers, max(5, min(args.steps, 20)))}))
+        return
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -300,6 +381,16 @@ def run_ours(args):
     if st != resq.OK:
         raise SystemExit(f"device status {st}: {resq.status_string(st)}")
 
+    # ---- decode variant of the same block (this rank only; reported by rank 0)
+    decode = None
+    if not args.no_decode and not only:
+        decode = decode_leg(resq, torch, dev, peaks, layers, max(5, min(args.steps, 20)))
+        k = decode["T1"]
+        kernels["mixed_gemm_decode_T1"] = {"bound": "hbm", "dtype": "int8", "achieved": k["weight_stream_gbs"],
+                                           "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                           "ms_per_step": round(k["mixed_gemv_us"] * 1e-3, 5),
+                                           "frac": k["frac_of_hbm_peak"]}
+
     # ---- CPU baseline: the oracle on a row sample, rank 0 at N = 1 only; also a parity spot check
     cpu_baseline, parity = None, None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -337,7 +428,7 @@ def run_ours(args):
             "mixed_gemm_frac_of_int8_peak": {"vs_measured_bf16_x2": kernels["mixed_gemm"]["frac"],
                                              "vs_nominal_4500": kernels["mixed_gemm"]["frac_of_nominal_4500"]},
             "per_layer": per_layer,
-            "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline, "parity_spot_check": parity,
+            "roofline": roofline, "decode": decode, "e2e": e2e, "cpu_baseline": cpu_baseline, "parity_spot_check": parity,
             "gpu_launches": LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
         }
         print(json.dumps(line))
@@ -385,6 +476,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--no-decode", action="store_true", help="skip the few-token leg (profiling runs)")
+    ap.add_argument("--decode-only", action="store_true", help="run only the few-token leg (profiling runs)")
     ap.add_argument("--layers", default="", help="comma-separated subset of qkv,o,gate_up,down (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":

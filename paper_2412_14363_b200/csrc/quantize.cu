@@ -8,6 +8,7 @@
 #include <cuda_fp16.h>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace resq {
 namespace {
@@ -155,6 +156,176 @@ split_quantize_kernel(const void* __restrict__ in, size_t in_row_bytes, size_t r
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Fast path (fp32 scales).  Same codes as the kernel above, bit for bit, at a fraction of its
+// instructions and with the row staged in shared memory instead of registers.
+//
+// Staging.  A CTA takes a group of 1, 2, 4 or 8 consecutive rows (about 32 KB); one thread issues a
+// bulk copy (cp.async.bulk, completion counted on an mbarrier) per row, so the whole group is in
+// flight at once and several CTAs per SM keep HBM busy while others compute.  Each row is then read
+// twice from shared memory: once for the two absmax values, once for the codes.
+//
+// Rounding.  The definition is code = round-half-even(fl(x / s)) with an IEEE division.  Here
+// t = fma(x, inv, M) with inv = RN(1 / s) and M = 1.5 * 2^23 rounds the exact product x * inv to the
+// nearest integer (ties to even) in one instruction, and the low byte of t's bit pattern is the
+// two's-complement code.  x * inv and fl(x / s) both lie within 2^-16 of x / s for |x / s| <= 128, so
+// the two roundings can only disagree when x * inv is within 2^-16 of a half-integer; whenever the
+// residual of a chunk comes within 2^-15 of one half, the chunk is redone with the true division.
+constexpr int kFastGroupBytes = 32 * 1024;
+constexpr int kFastMaxRowBytes = 200 * 1024;
+constexpr float kMagic = 12582912.f;                    // 1.5 * 2^23
+constexpr float kTieGuard = 0.5f - 0.000030517578125f;  // 1/2 - 2^-15
+
+template <bool F32>
+__device__ __forceinline__ Chunk<F32> lds_chunk(const uint8_t* row, int c) {
+    Chunk<F32> o;
+    if constexpr (F32) {
+        const uint4* p = reinterpret_cast<const uint4*>(row) + 2 * c;
+        const uint4 a = p[0], b = p[1];
+        o.w[0] = a.x; o.w[1] = a.y; o.w[2] = a.z; o.w[3] = a.w;
+        o.w[4] = b.x; o.w[5] = b.y; o.w[6] = b.z; o.w[7] = b.w;
+    } else {
+        const uint4 u = reinterpret_cast<const uint4*>(row)[c];
+        o.w[0] = u.x; o.w[1] = u.y; o.w[2] = u.z; o.w[3] = u.w;
+    }
+    return o;
+}
+
+template <bool F32>
+__device__ __forceinline__ void fast_codes(const Chunk<F32>& ch, float s, float inv, bool exact_only, uint32_t (&t)[8]) {
+    float dmax = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float x = ch.get(i);
+        const float tf = fmaf(x, inv, kMagic);
+        const float d = fmaf(x, inv, -(tf - kMagic));
+        dmax = fmaxf(dmax, fabsf(d));
+        t[i] = __float_as_uint(tf);
+    }
+    if (exact_only || !(dmax < kTieGuard)) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t[i] = __float_as_uint(rintf(__fdiv_rn(ch.get(i), s)) + kMagic);
+    }
+}
+
+// Low bytes of four words -> one word.
+__device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+}
+
+template <bool F32>
+__global__ void __launch_bounds__(kThreads)
+split_quantize_fast_kernel(const void* __restrict__ in, size_t in_row_bytes, size_t rows, int K, int r,
+                           int rows_per_cta, int8_t* __restrict__ q8, uint8_t* __restrict__ q4,
+                           float* __restrict__ s8_out, float* __restrict__ s4_out, int8_t* __restrict__ q4e,
+                           int* __restrict__ status) {
+    extern __shared__ __align__(128) uint8_t stage[];
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    __shared__ float red[2][kThreads / 32];
+    const uint32_t row_bytes = static_cast<uint32_t>(K) * (F32 ? 4u : 2u);
+    const size_t row0 = static_cast<size_t>(blockIdx.x) * rows_per_cta;
+    const int nrows = static_cast<int>(rows - row0 < static_cast<size_t>(rows_per_cta) ? rows - row0 : rows_per_cta);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&bar, 1);
+        fence_mbar_init();
+        mbar_arrive_expect_tx(&bar, row_bytes * static_cast<uint32_t>(nrows));
+        for (int i = 0; i < nrows; ++i)
+            bulk_load(stage + static_cast<size_t>(i) * row_bytes,
+                      reinterpret_cast<const char*>(in) + (row0 + i) * in_row_bytes, row_bytes, &bar);
+    }
+    __syncthreads();
+    const bool landed = mbar_wait(&bar, 0, &abort_flag);
+    if (__syncthreads_or(!landed)) {
+        // The copy did not land in time: report it and leave the outputs of this group unwritten.
+        if (threadIdx.x == 0) atomicOr(status, RESQ_ERR_TIMEOUT);
+        return;
+    }
+
+    const int tpr = kThreads / rows_per_cta;  // threads per row, a multiple of 32
+    const int grp = threadIdx.x / tpr, j = threadIdx.x - grp * tpr;
+    const int nchunks = K >> 3, rchunks = r >> 3;
+    const int K4 = K - r;
+    const bool live = grp < nrows;
+    const uint8_t* srow = stage + static_cast<size_t>(live ? grp : 0) * row_bytes;
+
+    float a8 = 0.f, a4 = 0.f;
+    if (live) {
+        for (int c = j; c < rchunks; c += tpr) a8 = fmaxf(a8, chunk_absmax(lds_chunk<F32>(srow, c)));
+        float m0 = 0.f, m1 = 0.f;  // two chains: the INT4 segment is 7/8 of the row
+        int c = rchunks + j;
+        for (; c + tpr < nchunks; c += 2 * tpr) {
+            m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
+            m1 = fmaxf(m1, chunk_absmax(lds_chunk<F32>(srow, c + tpr)));
+        }
+        if (c < nchunks) m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
+        a4 = fmaxf(m0, m1);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a8 = fmaxf(a8, __shfl_xor_sync(0xffffffffu, a8, o));
+        a4 = fmaxf(a4, __shfl_xor_sync(0xffffffffu, a4, o));
+    }
+    if (tpr > 32) {
+        const int warp = threadIdx.x >> 5, wpr = tpr >> 5;
+        if ((threadIdx.x & 31) == 0) {
+            red[0][warp] = a8;
+            red[1][warp] = a4;
+        }
+        __syncthreads();
+        for (int w = 0; w < wpr; ++w) {
+            a8 = fmaxf(a8, red[0][grp * wpr + w]);
+            a4 = fmaxf(a4, red[1][grp * wpr + w]);
+        }
+    }
+    if (!live) return;
+
+    const size_t row = row0 + grp;
+    const float s8 = __fdiv_rn(a8, 127.f), s4 = __fdiv_rn(a4, 7.f);
+    const float inv8 = s8 > 0.f ? __frcp_rn(s8) : 0.f, inv4 = s4 > 0.f ? __frcp_rn(s4) : 0.f;
+    // The product form needs a finite, normal reciprocal; otherwise every chunk takes the division.
+    const bool exact8 = s8 > 0.f && !(inv8 >= 1.1754944e-38f && inv8 <= 3.0e38f);
+    const bool exact4 = s4 > 0.f && !(inv4 >= 1.1754944e-38f && inv4 <= 3.0e38f);
+    if (j == 0) {
+        s8_out[row] = s8;
+        s4_out[row] = s4;
+    }
+    int8_t* q8row = q8 + row * static_cast<size_t>(r);
+    uint8_t* q4row = q4 ? q4 + row * static_cast<size_t>(K4 >> 1) : nullptr;
+    int8_t* q4e_row = q4e ? q4e + row * static_cast<size_t>(K4) : nullptr;
+
+    for (int c = j; c < rchunks; c += tpr) {
+        uint32_t t[8];
+        if (s8 > 0.f) fast_codes(lds_chunk<F32>(srow, c), s8, inv8, exact8, t);
+        else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) t[k] = 0;
+        }
+        *reinterpret_cast<uint2*>(q8row + c * 8) =
+            make_uint2(pack_low_bytes(t[0], t[1], t[2], t[3]), pack_low_bytes(t[4], t[5], t[6], t[7]));
+    }
+#pragma unroll 2
+    for (int c = rchunks + j; c < nchunks; c += tpr) {
+        uint32_t t[8];
+        if (s4 > 0.f) fast_codes(lds_chunk<F32>(srow, c), s4, inv4, exact4, t);
+        else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) t[k] = 0;
+        }
+        const int jj = (c - rchunks) * 8;
+        if (q4e_row)
+            *reinterpret_cast<uint2*>(q4e_row + jj) =
+                make_uint2(pack_low_bytes(t[0], t[1], t[2], t[3]), pack_low_bytes(t[4], t[5], t[6], t[7]));
+        if (q4row) {
+            uint32_t packed = 0;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) packed |= (t[k] & 0xFu) << (4 * k);
+            *reinterpret_cast<uint32_t*>(q4row + (jj >> 1)) = packed;
+        }
+    }
+}
+
 __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* __restrict__ out, size_t nwords) {
     // one 32-bit packed word (8 codes) per thread -> 8 bytes
     for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < nwords;
@@ -177,6 +348,29 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
                                   uint8_t* q4, void* s8, void* s4, bool scale_fp16, int8_t* q4_i8,
                                   size_t in_row_stride_bytes, cudaStream_t st) {
     if (rows == 0) return cudaSuccess;
+    const size_t row_bytes = static_cast<size_t>(K) * (in_is_f32 ? 4 : 2);
+    if (!scale_fp16 && row_bytes <= static_cast<size_t>(kFastMaxRowBytes) && in_row_stride_bytes % 16 == 0) {
+        int rpc = 1;  // rows per CTA: 1, 2, 4 or 8, about kFastGroupBytes of staging
+        while (rpc < 8 && row_bytes * rpc * 2 <= static_cast<size_t>(kFastGroupBytes)) rpc *= 2;
+        const size_t smem = row_bytes * rpc;
+        auto kern = in_is_f32 ? split_quantize_fast_kernel<true> : split_quantize_fast_kernel<false>;
+        static bool attr_set[2][64] = {};
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 64 && !attr_set[in_is_f32][dev]) {
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kFastMaxRowBytes);
+            if (e != cudaSuccess) return e;
+            attr_set[in_is_f32][dev] = true;
+        }
+        const size_t groups = (rows + rpc - 1) / rpc;
+        if (groups <= 0x7fffffffu) {
+            kern<<<static_cast<unsigned>(groups), kThreads, smem, st>>>(in, in_row_stride_bytes, rows, K, r, rpc, q8, q4,
+                                                                    static_cast<float*>(s8), static_cast<float*>(s4),
+                                                                    q4_i8, device_status_ptr());
+            return cudaGetLastError();
+        }
+    }
     const unsigned grid = static_cast<unsigned>(rows < 148u * 64u ? rows : 148u * 64u);
     if (in_is_f32)
         split_quantize_kernel<true><<<grid, kThreads, 0, st>>>(in, in_row_stride_bytes, rows, K, r, q8, q4, s8, s4,

@@ -77,6 +77,55 @@ def test_split_quantize_tie_rows(resq):
     assert_quantize_matches(resq, synth.f32_to_bf16_bits(C), r)
 
 
+def test_split_quantize_power_of_two_scales(resq):
+    """Rows whose absmax is 127 * 2^m / 7 * 2^m: the scales are powers of two, so bf16 inputs hit exact
+    .5 ties by the thousand; a subnormal row and a huge row exercise the range ends of the reciprocal."""
+    T, K, r = 40, 4096, 512
+    rng = np.random.default_rng(5)
+    C = synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(rng.uniform(-1, 1, (T, K)).astype(np.float32)))
+    for t in range(T):
+        m = float(2.0 ** (t % 9 - 4))
+        half8 = (rng.integers(-126, 126, r) + 0.5) * m          # exact ties of the INT8 segment
+        half4 = (rng.integers(-7, 7, K - r) + 0.5) * m
+        C[t, :r] = np.where(rng.random(r) < 0.5, half8, C[t, :r] * 127 * m)
+        C[t, r:] = np.where(rng.random(K - r) < 0.5, half4, C[t, r:] * 7 * m)
+        C[t, 0], C[t, r] = 127 * m, -7 * m
+    C[37] *= np.float32(2.0 ** -140)       # subnormal scales: 1/s overflows
+    C[38] *= np.float32(2.0 ** 118)        # huge values
+    C[39, r:] = 0.0
+    bits = synth.f32_to_bf16_bits(C.astype(np.float32))
+    assert_quantize_matches(resq, bits, r)
+
+
+def test_pack_weights_near_ties(resq):
+    """fp32 rows built so that x / s lands on, just below and just above k + 1/2 (a few ulp): the
+    product-with-reciprocal shortcut must fall back to the division exactly where the two disagree."""
+    N, K, r = 96, 2048, 256
+    rng = np.random.default_rng(11)
+    Wp = rng.standard_normal((N, K)).astype(np.float32)
+    for n in range(N):
+        for lo, hi, qmax in ((0, r, 127), (r, K, 7)):
+            seg = Wp[n, lo:hi]
+            a = np.float32(np.abs(seg).max() * (1.5 if n % 2 else 1.0))
+            s = np.float32(a / np.float32(qmax))
+            k = rng.integers(-qmax, qmax, seg.size).astype(np.float32) + np.float32(0.5)
+            x = (k * s).astype(np.float32)
+            ulps = rng.integers(-3, 4, seg.size).astype(np.int32)
+            x = (x.view(np.int32) + ulps).view(np.float32)
+            take = rng.random(seg.size) < 0.7
+            seg[take] = x[take]
+            seg[0] = a
+    pw = oracle.pack_weights(Wp, r)
+    desc = resq.layer_desc(K, N, r)
+    W = resq.resq_pack_weights(desc, dev(Wp))
+    _check_status(resq)
+    assert (host(W.s_w8).view(np.uint32) == pw.s8.view(np.uint32)).all()
+    assert (host(W.s_w4).view(np.uint32) == pw.s4.view(np.uint32)).all()
+    assert (host(W.w8) == pw.q8).all()
+    assert (host(W.w4_i8) == pw.q4).all()
+    assert (host(W.w4) == pw.w4_packed).all()
+
+
 @pytest.mark.parametrize("N,K,r,fp16", [(512, 512, 64, False), (512, 512, 64, True), (1024, 4096, 512, True),
                                         (264, 2048, 256, False), (64, 14336, 1792, True)])
 def test_pack_weights_bit_exact(resq, N, K, r, fp16):

@@ -1,0 +1,52 @@
+"""Host-side check of the claim the fast quantizer kernel rests on.
+
+The kernel replaces code = rint(fl(x / s)) (the definition, Eq. 1 with round-half-even and an IEEE
+fp32 division) by rint(x * inv) with inv = RN(1 / s), evaluated exactly by a fused multiply-add, and
+falls back to the division whenever x * inv comes within 2^-15 of a half-integer.  Claim: outside that
+guard band both roundings agree for every |x / s| <= 128.  Checked here with exact rationals on random
+and on adversarial near-tie inputs; the defined value comes from the oracle's quantizer.
+"""
+from fractions import Fraction
+
+import numpy as np
+
+import oracle
+
+GUARD = Fraction(1, 2) - Fraction(1, 2 ** 15)
+
+
+def _rint_half_even(q: Fraction) -> int:
+    f = q.numerator // q.denominator
+    rem = q - f
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and f % 2):
+        return f + 1
+    return f
+
+
+def test_product_rounding_agrees_outside_guard_band():
+    rng = np.random.default_rng(3)
+    checked = fallbacks = 0
+    for qmax in (127, 7):
+        for _ in range(40):
+            a = np.float32(np.exp(rng.uniform(-20, 20)))
+            s = np.float32(a / np.float32(qmax))
+            inv = np.float32(np.float32(1.0) / s)  # numpy's fp32 division is correctly rounded
+            k = rng.integers(-qmax, qmax, 200).astype(np.float32) + np.float32(0.5)
+            near = ((k * s).astype(np.float32).view(np.int32) + rng.integers(-4, 5, 200).astype(np.int32)).view(np.float32)
+            rand = (rng.uniform(-1, 1, 200) * a).astype(np.float32)
+            x = np.concatenate([near, rand, [a, -a]]).astype(np.float32)
+            x = x[np.abs(x) <= a]
+            # the definition, through the oracle: one row whose absmax is a
+            row = np.concatenate([[a], x]).astype(np.float32)
+            s_o, codes = oracle.quantize_vector(row, 8 if qmax == 127 else 4)
+            assert s_o == s
+            codes = codes[1:]
+            for xv, code in zip(x, codes):
+                p = Fraction(float(xv)) * Fraction(float(inv))
+                n = _rint_half_even(p)
+                if abs(p - n) < GUARD:
+                    assert n == int(code), (float(xv), float(s), n, int(code))
+                    checked += 1
+                else:
+                    fallbacks += 1
+    assert checked > 10000 and fallbacks > 1000  # both branches were exercised
