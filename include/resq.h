@@ -117,7 +117,8 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
  * Integer products accumulate exactly in int32; the epilogue is fp32:
  *     y = (float)acc8 * (s_x8[t] * s_w8[n]) + (float)acc4 * (s_x4[t] * s_w4[n])
  * rounded to bf16 (nearest even) when y_dtype == RESQ_Y_BF16.  Y is [T][n_out].
- * T <= 16 runs the weight-streaming split-K kernel, larger T the tensor-core tile kernel.
+ * T <= 16 runs a weight-streaming kernel (exact integer sums whatever its work split), larger T the
+ * tensor-core tile kernel.
  * The INT4 activation codes come packed (x4, uint8 [T][(K-r)/2]) and/or one per byte (x4_i8, int8
  * [T][K-r], as resq_project_quantize can emit them).  The streaming kernel reads x4, so x4 is
  * required when T <= 16; the tile kernel reads x4_i8 and, if only x4 is given, first expands it
@@ -160,6 +161,20 @@ int resq_linear(const resq_layer_desc_t* desc, int T, const void* X, const void*
 #define RESQ_STATIC_SCRATCH_BYTES (8u << 20)
 int resq_project_quantize_static(const void* X, const void* P, int T, int K, int r, int8_t* x8, uint8_t* x4,
                                  float* s_x8, float* s_x4, int8_t* x4_i8, void* stream);
+
+/*
+ * Process-wide options (host state of the library; not thread-safe against concurrent calls).
+ *  RESQ_OPT_DECODE_EARLY_WEIGHTS (default 0): when 1, the few-token kernel (T <= 16) is launched so
+ *    that it may begin while the preceding kernel of the stream is still running; it then streams its
+ *    packed weights into shared memory at once and only waits for that kernel before it reads the
+ *    activation codes and scales.  Generation is memory-bound (paper, Introduction), and this hides
+ *    the ramp of each short kernel behind the tail of the previous one.  The caller promises that the
+ *    packed weights and their scales were complete before the preceding kernel was enqueued (true
+ *    for weights packed at load time; false if resq_pack_weights is the preceding kernel).
+ * Returns RESQ_ERR_SHAPE for an unknown option.
+ */
+enum { RESQ_OPT_DECODE_EARLY_WEIGHTS = 1 };
+int resq_set_option(int option, int value);
 
 /* Inverse of the INT4 packing, for inspection: packed [rows][cols/2] -> int8 [rows][cols]. */
 int resq_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, void* stream);

@@ -17,12 +17,13 @@ LIB_PATH = os.path.join(_HERE, "libresq.so")
 
 OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(8)
 SCALE_FP32, SCALE_FP16 = 0, 1
+OPT_DECODE_EARLY_WEIGHTS = 1
 Y_BF16, Y_FP32 = 0, 1
 
 EXPORTS = [
     "resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_bytes", "resq_workspace_bytes",
     "resq_pack_weights", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
-    "resq_unpack_int4",
+    "resq_unpack_int4", "resq_set_option",
     "resq_device_status", "resq_status_string",
 ]
 
@@ -62,6 +63,7 @@ lib.resq_mixed_gemm.argtypes = [_dp, _i, _vp, _vp, _vp, _vp, _vp, ctypes.POINTER
                                 _vp, _sz, _vp]
 lib.resq_linear.argtypes = [_dp, _i, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _i, _vp, _sz, _vp]
 lib.resq_unpack_int4.argtypes = [_vp, _vp, _sz, _sz, _vp]
+lib.resq_set_option.argtypes = [_i, _i]
 lib.resq_device_status.argtypes = [_vp]
 lib.resq_status_string.restype = ctypes.c_char_p
 lib.resq_status_string.argtypes = [_i]
@@ -173,6 +175,10 @@ def resq_linear(W: Weights, X, P, Y, workspace):
 def resq_unpack_int4(packed, out):
     rows, half = packed.shape
     _check(lib.resq_unpack_int4(_ptr(packed), _ptr(out), rows, half * 2, _stream()), "resq_unpack_int4")
+
+
+def resq_set_option(option: int, value: int):
+    _check(lib.resq_set_option(int(option), int(value)), "resq_set_option")
 
 
 def resq_device_status() -> int:

@@ -159,6 +159,11 @@ static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, 
                            cudaStream_t st) {
     const bool fp16 = d->w_scale_dtype == RESQ_SCALE_FP16;
     const size_t K4 = static_cast<size_t>(d->K - d->r);
+    if (T <= kDecodeMaxT) {
+        const cudaError_t e = launch_mixed_gemm_stream(T, d->n_out, d->K, d->r, x8, x4, s_x8, s_x4, W->w8, W->w4,
+                                                       W->s_w8, W->s_w4, fp16, Y, y_dtype, dbg8, dbg4, st);
+        if (e != cudaErrorNotSupported) return cuda_status(e);
+    }
     if (T <= kDecodeMaxT)
         return cuda_status(launch_mixed_gemm_decode(T, d->n_out, d->K, d->r, x8, x4, s_x8, s_x4, W->w8, W->w4,
                                                     W->s_w8, W->s_w4, fp16, Y, y_dtype, dbg8, dbg4,
@@ -236,6 +241,14 @@ int resq_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t col
     if (cols % 8 != 0) return RESQ_ERR_SHAPE;
     if (!aligned16(packed) || !aligned16(out)) return RESQ_ERR_ALIGN;
     return cuda_status(launch_unpack_int4(packed, out, rows, cols, static_cast<cudaStream_t>(stream)));
+}
+
+int resq_set_option(int option, int value) {
+    if (option == RESQ_OPT_DECODE_EARLY_WEIGHTS) {
+        set_decode_early_weights(value);
+        return RESQ_OK;
+    }
+    return RESQ_ERR_SHAPE;
 }
 
 int resq_device_status(void* stream) {

@@ -36,6 +36,15 @@ cudaError_t launch_mixed_gemm_decode(int T, int N, int K, int r, const int8_t* x
                                      const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
                                      int32_t* dbg8, int32_t* dbg4, void* scratch, cudaStream_t st);
 
+// Few-token streaming kernel (persistent grid, bulk-copy ring).  Returns cudaErrorNotSupported, with
+// nothing launched, when the staged activations leave no room for the ring; the caller then uses
+// launch_mixed_gemm_decode.
+cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x8, const uint8_t* x4,
+                                     const float* s_x8, const float* s_x4, const int8_t* w8, const uint8_t* w4,
+                                     const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
+                                     int32_t* dbg8, int32_t* dbg4, cudaStream_t st);
+void set_decode_early_weights(int on);
+
 // Online projection C = X·P (bf16 x bf16 -> fp32) on tcgen05 kind::f16; writes fp32 C [T][K].
 cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, float* C, cudaStream_t st);
 

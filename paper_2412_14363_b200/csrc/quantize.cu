@@ -223,6 +223,9 @@ split_quantize_fast_kernel(const void* __restrict__ in, size_t in_row_bytes, siz
     __shared__ uint64_t bar;
     __shared__ int abort_flag;
     __shared__ float red[2][kThreads / 32];
+    // A kernel enqueued behind this one with programmatic stream serialization may start its own
+    // input-independent prologue now; it still waits for this grid to finish before reading the codes.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const uint32_t row_bytes = static_cast<uint32_t>(K) * (F32 ? 4u : 2u);
     const size_t row0 = static_cast<size_t>(blockIdx.x) * rows_per_cta;
     const int nrows = static_cast<int>(rows - row0 < static_cast<size_t>(rows_per_cta) ? rows - row0 : rows_per_cta);

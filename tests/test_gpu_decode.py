@@ -25,7 +25,11 @@ def resq():
     (8, 512, 512, 64, False),       # r < one 64-byte step
     (16, 14336, 128, 1792, True),   # down_proj reduction length, few channels
     (3, 1056, 72, 96, False),       # segment lengths that are not multiples of a step
-    (16, 4096, 28672, 512, True),   # gate|up: enough channel blocks that K is not split
+    (16, 4096, 28672, 512, True),   # gate|up: many units per CTA
+    (16, 14336, 4096, 1792, True),  # down_proj: INT4 rows of 6272 bytes span four ring stages
+    (16, 28672, 64, 3584, False),   # activations too large to stage whole: the cluster split-K kernel runs
+    (5, 28672, 64, 3584, False),    # ... while 8 token rows of the same shape still fit
+    (2, 4096, 8, 512, False),       # a single unit
 ])
 def test_decode_bit_exact(resq, T, K, N, r, fp16):
     _, _, pw, res = oracle_case(T, K, N, r, fp16, seed_shift=50 + T)
@@ -70,3 +74,32 @@ def test_decode_linear_end_to_end(resq, T):
     resq.resq_linear(W, bf16_to_dev(C_bits), None, ybf, ws)
     assert resq.resq_device_status() == resq.OK
     check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))
+
+
+def test_decode_early_weights_back_to_back(resq):
+    """With the early-weights option each launch may start while the previous one still runs and
+    prefetches its weights before waiting for it; a chain of launches over different layers must give
+    exactly what the same launches give one by one."""
+    cases = [oracle_case(T, 4096, N, 512, True, seed_shift=90 + i) for i, (T, N) in enumerate([(16, 1024), (3, 2048), (16, 512)])]
+    packs = []
+    for _, _, pw, res in cases:
+        desc = resq.layer_desc(pw.K, pw.N, pw.r, resq.SCALE_FP16)
+        W = resq.Weights(desc, dev(pw.q8), dev(pw.w4_packed), dev(pw.s8).half(), dev(pw.s4).half(), None)
+        T = res.x8.shape[0]
+        packs.append((W, dev(res.x8), dev(res.x4_packed), dev(res.s_x8), dev(res.s_x4),
+                      torch.zeros((T, pw.N), dtype=torch.float32, device="cuda"),
+                      torch.full((T, pw.N), -1, dtype=torch.int32, device="cuda"),
+                      torch.full((T, pw.N), -1, dtype=torch.int32, device="cuda"),
+                      resq.alloc_workspace(desc, T, False, False)))
+    torch.cuda.synchronize()
+    resq.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 1)
+    try:
+        for _ in range(3):
+            for W, x8, x4, s8, s4, y, a8, a4, ws in packs:
+                resq.resq_mixed_gemm(W, x8, x4, s8, s4, y, ws, a8, a4)
+    finally:
+        resq.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 0)
+    assert resq.resq_device_status() == resq.OK
+    for (_, _, pw, res), (W, x8, x4, s8, s4, y, a8, a4, ws) in zip(cases, packs):
+        assert (host(a8) == res.acc8).all() and (host(a4) == res.acc4).all()
+        check_output(res, pw, host(y))
