@@ -135,19 +135,16 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
     uint8_t* ring = rings + static_cast<size_t>(warp) * p.nstages * kStageBytes;
     uint64_t* full = ctl->full[warp];
 
-    for (int i = threadIdx.x; i < kWarps * kSlotInts; i += kThreads) slots[i] = 0;
-    if (threadIdx.x < kWarps) ctl->arrived[threadIdx.x] = 0;
-    if (threadIdx.x == 0) {
-        ctl->abort_flag = 0;
-        tma_prefetch_desc(&tmW8);
-        tma_prefetch_desc(&tmW4);
-    }
-    if (lane == 0)
+    // Each warp owns its barriers, so its lane 0 can start the first copies without a CTA-wide barrier.
+    if (lane == 0) {
         for (int s = 0; s < p.nstages; ++s) mbar_init(&full[s], 1);
-    fence_mbar_init();
-    __syncthreads();
+        fence_mbar_init();
+    }
     griddep_launch_dependents();
 
+    // Every weight byte is read once: mark the lines evict-first so that the activations, the scales
+    // and whatever the neighbouring kernels keep in L2 stay there.
+    const uint64_t stream_policy = l2_policy_evict_first();
     // Issue cursor of this warp (only lane 0 uses it): next (item, chunk) to copy.
     int is_idx = cb, is_item = cb / nchunks, is_chunk = cb - (cb / nchunks) * nchunks;
     auto issue = [&](int stage) {
@@ -155,59 +152,96 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         const bool seg8 = is_chunk < p.c8;
         const int x = (seg8 ? is_chunk : is_chunk - p.c8) * (kChunkBytes / 4);  // in 32-bit elements: a multiple of 16
         mbar_arrive_expect_tx(&full[stage], kStageBytes);
-        tma_load_2d(ring + static_cast<size_t>(stage) * kStageBytes, seg8 ? &tmW8 : &tmW4, &full[stage], x, ub * kUnitRows);
+        tma_load_2d_hint(ring + static_cast<size_t>(stage) * kStageBytes, seg8 ? &tmW8 : &tmW4, &full[stage], x, ub * kUnitRows,
+                         stream_policy);
         ++is_idx;
         if (++is_chunk == nchunks) { is_chunk = 0; ++is_item; }
     };
 
     if (!p.early_weights) griddep_wait();
     int issued = 0;
-    if (lane == 0) {
-        const int total = ce - cb;
-        issued = total < p.nstages ? total : p.nstages;
-        for (int s = 0; s < issued; ++s) issue(s);
+    // One stage per warp goes out now; the rest follow once the (small, latency-critical) activation
+    // loads below have been issued, so that those do not queue behind a full ring of weight traffic.
+    const int first_burst = ce - cb < p.nstages ? ce - cb : p.nstages;
+    if (lane == 0 && first_burst > 0) {
+        issue(0);
+        issued = 1;
     }
+    for (int i = threadIdx.x; i < kWarps * kSlotInts; i += kThreads) slots[i] = 0;
+    if (threadIdx.x < kWarps) ctl->arrived[threadIdx.x] = 0;
+    if (threadIdx.x == 0) ctl->abort_flag = 0;
     if (p.early_weights) griddep_wait();
 
-    // Stage the activation codes: zero padded to the pitch, zero rows for tokens >= T.
-    {
-        const int v8 = p.pitch8 >> 4, v4 = p.pitch4 >> 4;  // 16-byte vectors per token
-        for (int i = threadIdx.x; i < TP * v8; i += kThreads) {
-            const int t = i / v8, o = (i - t * v8) << 4;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (t < p.T && o < p.r) v = *reinterpret_cast<const uint4*>(p.x8 + static_cast<size_t>(t) * p.r + o);
-            *reinterpret_cast<uint4*>(act8 + static_cast<size_t>(t) * p.pitch8 + o) = v;
-        }
-        // INT4: warp w stages tokens w (and w + 8) and sums their even codes on the way.
-#pragma unroll
-        for (int tt = 0; tt < TT; ++tt) {
-            const int t = warp + 8 * tt;
-            int se = 0;
-            for (int i = lane; i < v4; i += 32) {
-                const int o = i << 4;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (t < p.T && o < p.row4) v = *reinterpret_cast<const uint4*>(p.x4 + static_cast<size_t>(t) * p.row4 + o);
-                const uint4 ev = make_uint4((v.x << 4) & kHi, (v.y << 4) & kHi, (v.z << 4) & kHi, (v.w << 4) & kHi);
-                se = __dp4a(static_cast<int>(ev.x), 0x01010101, se);
-                se = __dp4a(static_cast<int>(ev.y), 0x01010101, se);
-                se = __dp4a(static_cast<int>(ev.z), 0x01010101, se);
-                se = __dp4a(static_cast<int>(ev.w), 0x01010101, se);
-                if (kSplit) {
-                    *reinterpret_cast<uint4*>(act4 + static_cast<size_t>(t) * p.pitch4 + o) = ev;
-                    *reinterpret_cast<uint4*>(act4 + static_cast<size_t>(TP + t) * p.pitch4 + o) =
-                        make_uint4(v.x & kHi, v.y & kHi, v.z & kHi, v.w & kHi);
-                } else {
-                    *reinterpret_cast<uint4*>(act4 + static_cast<size_t>(t) * p.pitch4 + o) = v;
-                }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
-            if (lane == 0) ctl->s_even[t] = se >> 4;  // the lanes held 16 x the codes
-        }
-    }
     // Token scales of the two accumulator rows this thread holds.
     const float sx8a = g < p.T ? p.s_x8[g] : 0.f, sx4a = g < p.T ? p.s_x4[g] : 0.f;
     const float sx8b = g + 8 < p.T ? p.s_x8[g + 8] : 0.f, sx4b = g + 8 < p.T ? p.s_x4[g + 8] : 0.f;
+    // Stage the activation codes: zero padded to the pitch, zero rows for tokens >= T.  The loads of a
+    // batch all go out before the first of them is used.
+    {
+        const int v8 = p.pitch8 >> 4, v4 = p.pitch4 >> 4;  // 16-byte vectors per token
+        const int r8 = p.r >> 4, r4 = p.row4 >> 4;         // ... that hold data
+#pragma unroll 4
+        for (int i = threadIdx.x; i < TP * v8; i += kThreads) {
+            const int t = i / v8, o = i - t * v8;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (t < p.T && o < r8) v = __ldg(reinterpret_cast<const uint4*>(p.x8 + static_cast<size_t>(t) * p.r) + o);
+            *reinterpret_cast<uint4*>(act8 + static_cast<size_t>(t) * p.pitch8 + (o << 4)) = v;
+        }
+        constexpr int kBatch = 4;
+        const int total4 = TP * v4;
+        for (int base = 0; base < total4; base += kBatch * kThreads) {
+            uint4 v[kBatch];
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                const int i = base + b * kThreads + threadIdx.x;
+                const int t = i / v4, o = i - t * v4;
+                v[b] = make_uint4(0, 0, 0, 0);
+                if (i < total4 && t < p.T && o < r4)
+                    v[b] = __ldg(reinterpret_cast<const uint4*>(p.x4 + static_cast<size_t>(t) * p.row4) + o);
+            }
+            if (base + kBatch * kThreads >= total4 && lane == 0) {
+                // The last activation loads are on their way: the rest of the ring may go out now.
+                for (int s = issued; s < first_burst; ++s) issue(s);
+                issued = first_burst;
+            }
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                const int i = base + b * kThreads + threadIdx.x;
+                if (i >= total4) continue;
+                const int t = i / v4, o = i - t * v4;
+                uint8_t* dst = act4 + static_cast<size_t>(t) * p.pitch4 + (o << 4);
+                if (kSplit) {
+                    *reinterpret_cast<uint4*>(dst) =
+                        make_uint4((v[b].x << 4) & kHi, (v[b].y << 4) & kHi, (v[b].z << 4) & kHi, (v[b].w << 4) & kHi);
+                    *reinterpret_cast<uint4*>(dst + static_cast<size_t>(TP) * p.pitch4) =
+                        make_uint4(v[b].x & kHi, v[b].y & kHi, v[b].z & kHi, v[b].w & kHi);
+                } else {
+                    *reinterpret_cast<uint4*>(dst) = v[b];
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // Sum of the even-position INT4 codes per token (warp w: tokens w and w + 8), from the staged rows.
+#pragma unroll
+    for (int tt = 0; tt < TT; ++tt) {
+        const int t = warp + 8 * tt;
+        int se = 0;
+        if (t < p.T) {
+            const uint8_t* row = act4 + static_cast<size_t>(t) * p.pitch4;
+            for (int i = lane; i < (p.pitch4 >> 4); i += 32) {
+                uint4 v = *reinterpret_cast<const uint4*>(row + (i << 4));
+                if (!kSplit) v = make_uint4((v.x << 4) & kHi, (v.y << 4) & kHi, (v.z << 4) & kHi, (v.w << 4) & kHi);
+                se = __dp4a(static_cast<int>(v.x), 0x01010101, se);
+                se = __dp4a(static_cast<int>(v.y), 0x01010101, se);
+                se = __dp4a(static_cast<int>(v.z), 0x01010101, se);
+                se = __dp4a(static_cast<int>(v.w), 0x01010101, se);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+        if (lane == 0) ctl->s_even[t] = se >> 4;  // the lanes held 16 x the codes
+    }
     __syncthreads();
     const int sev_a = ctl->s_even[g], sev_b = TT == 2 ? ctl->s_even[g + 8] : 0;
 
