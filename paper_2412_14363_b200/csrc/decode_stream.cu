@@ -103,11 +103,12 @@ __device__ __forceinline__ float2 load_scale2(const void* p, int n, int fp16) {
     return *reinterpret_cast<const float2*>(reinterpret_cast<const float*>(p) + n);
 }
 
-// TT = 1: T <= 8.  Token rows 8..15 of the 16-row operand are zero and are not staged, and the INT4
-//         activations are staged already split into their even / odd codes times 16.
-// TT = 2: T <= 16.  The INT4 activations stay packed in shared memory and are split when used.
+// TT:     1 for T <= 8 (token rows 8..15 of the 16-row operand are zero and are not staged), 2 for T <= 16.
 // CS:     64-byte steps per chunk (3 or 5).
-template <int TT, int CS>
+// kSplit: the INT4 activations are staged already split into their even / odd codes times 16 (twice
+//         the shared memory, a third of the logic operations); otherwise they stay packed and are
+//         split when used.
+template <int TT, int CS, bool kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_constant__ CUtensorMap tmW4,
                          const Params p) {
@@ -115,7 +116,6 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
     constexpr int TP = TT * 8;
     constexpr int kChunkBytes = CS * 64;
     constexpr int kStageBytes = kItemRows * kChunkBytes;
-    constexpr bool kSplit = TT == 1;
     Control* ctl = reinterpret_cast<Control*>(smem);
     int* slots = reinterpret_cast<int*>(smem + kControlBytes);                        // [kWarps][kSlotInts]
     uint8_t* act8 = smem + kControlBytes + kSlotBytes;                                // [TP][pitch8]
@@ -175,39 +175,46 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
     // Token scales of the two accumulator rows this thread holds.
     const float sx8a = g < p.T ? p.s_x8[g] : 0.f, sx4a = g < p.T ? p.s_x4[g] : 0.f;
     const float sx8b = g + 8 < p.T ? p.s_x8[g + 8] : 0.f, sx4b = g + 8 < p.T ? p.s_x4[g + 8] : 0.f;
-    // Stage the activation codes: zero padded to the pitch, zero rows for tokens >= T.  The loads of a
-    // batch all go out before the first of them is used.
+    // Stage the activation codes: zero padded to the pitch, zero rows for tokens >= T.  The first
+    // batch of INT8 and of INT4 vectors is loaded before anything is stored (one round trip to L2 for
+    // the usual sizes); the rest of the ring goes out right behind those loads.
     {
         const int v8 = p.pitch8 >> 4, v4 = p.pitch4 >> 4;  // 16-byte vectors per token
         const int r8 = p.r >> 4, r4 = p.row4 >> 4;         // ... that hold data
-#pragma unroll 4
-        for (int i = threadIdx.x; i < TP * v8; i += kThreads) {
-            const int t = i / v8, o = i - t * v8;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (t < p.T && o < r8) v = __ldg(reinterpret_cast<const uint4*>(p.x8 + static_cast<size_t>(t) * p.r) + o);
-            *reinterpret_cast<uint4*>(act8 + static_cast<size_t>(t) * p.pitch8 + (o << 4)) = v;
-        }
+        const int n8 = TP * v8, n4 = TP * v4;
         constexpr int kBatch = 4;
-        const int total4 = TP * v4;
-        for (int base = 0; base < total4; base += kBatch * kThreads) {
-            uint4 v[kBatch];
+        auto load8 = [&](int base, uint4 (&v)[kBatch]) {
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                const int i = base + b * kThreads + threadIdx.x;
+                const int t = i / v8, o = i - t * v8;
+                v[b] = make_uint4(0, 0, 0, 0);
+                if (i < n8 && t < p.T && o < r8) v[b] = __ldg(reinterpret_cast<const uint4*>(p.x8 + static_cast<size_t>(t) * p.r) + o);
+            }
+        };
+        auto store8 = [&](int base, const uint4 (&v)[kBatch]) {
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b) {
+                const int i = base + b * kThreads + threadIdx.x;
+                if (i >= n8) continue;
+                const int t = i / v8, o = i - t * v8;
+                *reinterpret_cast<uint4*>(act8 + static_cast<size_t>(t) * p.pitch8 + (o << 4)) = v[b];
+            }
+        };
+        auto load4 = [&](int base, uint4 (&v)[kBatch]) {
 #pragma unroll
             for (int b = 0; b < kBatch; ++b) {
                 const int i = base + b * kThreads + threadIdx.x;
                 const int t = i / v4, o = i - t * v4;
                 v[b] = make_uint4(0, 0, 0, 0);
-                if (i < total4 && t < p.T && o < r4)
-                    v[b] = __ldg(reinterpret_cast<const uint4*>(p.x4 + static_cast<size_t>(t) * p.row4) + o);
+                if (i < n4 && t < p.T && o < r4) v[b] = __ldg(reinterpret_cast<const uint4*>(p.x4 + static_cast<size_t>(t) * p.row4) + o);
             }
-            if (base + kBatch * kThreads >= total4 && lane == 0) {
-                // The last activation loads are on their way: the rest of the ring may go out now.
-                for (int s = issued; s < first_burst; ++s) issue(s);
-                issued = first_burst;
-            }
+        };
+        auto store4 = [&](int base, const uint4 (&v)[kBatch]) {
 #pragma unroll
             for (int b = 0; b < kBatch; ++b) {
                 const int i = base + b * kThreads + threadIdx.x;
-                if (i >= total4) continue;
+                if (i >= n4) continue;
                 const int t = i / v4, o = i - t * v4;
                 uint8_t* dst = act4 + static_cast<size_t>(t) * p.pitch4 + (o << 4);
                 if (kSplit) {
@@ -219,6 +226,23 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                     *reinterpret_cast<uint4*>(dst) = v[b];
                 }
             }
+        };
+        uint4 va[kBatch], vb[kBatch];
+        load8(0, va);
+        load4(0, vb);
+        if (lane == 0) {
+            for (int s = issued; s < first_burst; ++s) issue(s);
+            issued = first_burst;
+        }
+        store8(0, va);
+        store4(0, vb);
+        for (int base = kBatch * kThreads; base < n8; base += kBatch * kThreads) {
+            load8(base, va);
+            store8(base, va);
+        }
+        for (int base = kBatch * kThreads; base < n4; base += kBatch * kThreads) {
+            load4(base, vb);
+            store4(base, vb);
         }
     }
     __syncthreads();
@@ -298,15 +322,22 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                 for (int s = 0; s < CS; ++s) {
                     uint32_t xe[4], xo[4], ye[4], yo[4];
                     if (kSplit) {
+                        const uint8_t* xod = xa + static_cast<size_t>(TP) * p.pitch4;
                         const uint4 e = *reinterpret_cast<const uint4*>(xa + 64 * s);
-                        const uint4 o = *reinterpret_cast<const uint4*>(xa + static_cast<size_t>(TP) * p.pitch4 + 64 * s);
+                        const uint4 o = *reinterpret_cast<const uint4*>(xod + 64 * s);
                         xe[0] = e.x; xe[1] = e.y; xe[2] = e.z; xe[3] = e.w;
                         xo[0] = o.x; xo[1] = o.y; xo[2] = o.z; xo[3] = o.w;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) ye[j] = yo[j] = 0;
+                        uint4 e2 = make_uint4(0, 0, 0, 0), o2 = e2;
+                        if (TT == 2) {
+                            e2 = *reinterpret_cast<const uint4*>(xa + 8 * p.pitch4 + 64 * s);
+                            o2 = *reinterpret_cast<const uint4*>(xod + 8 * p.pitch4 + 64 * s);
+                        }
+                        ye[0] = e2.x; ye[1] = e2.y; ye[2] = e2.z; ye[3] = e2.w;
+                        yo[0] = o2.x; yo[1] = o2.y; yo[2] = o2.z; yo[3] = o2.w;
                     } else {
                         const uint4 x = *reinterpret_cast<const uint4*>(xa + 64 * s);
-                        const uint4 y = *reinterpret_cast<const uint4*>(xa + 8 * p.pitch4 + 64 * s);
+                        uint4 y = make_uint4(0, 0, 0, 0);
+                        if (TT == 2) y = *reinterpret_cast<const uint4*>(xa + 8 * p.pitch4 + 64 * s);
                         const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -446,10 +477,10 @@ bool make_map_rows(CUtensorMap* m, const void* base, uint64_t rows, uint64_t row
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int TT, int CS>
+template <int TT, int CS, bool SPLIT>
 cudaError_t launch_variant(const CUtensorMap& t8, const CUtensorMap& t4, const Params& p, int grid, size_t smem,
                            cudaStream_t st) {
-    auto kern = mixed_gemm_stream_kernel<TT, CS>;
+    auto kern = mixed_gemm_stream_kernel<TT, CS, SPLIT>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -486,27 +517,36 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
     p.T = T; p.N = N; p.r = r; p.row4 = (K - r) / 2;
     p.units = N / kUnitRows;
     const int TT = T <= 8 ? 1 : 2, TP = 8 * TT;
-    // The larger chunk (5 steps) if every warp still gets four stages, else the smaller one (3 steps).
-    int cs = 0, nstages = 0;
+    // Configurations in order of preference: split staging of the INT4 activations before packed
+    // for T <= 8 and the reverse above, the
+    // larger chunk (5 steps) before the smaller (3 steps); the first that leaves every warp four
+    // stages wins, else the last one tried that leaves two.
+    int cs = 0, nstages = 0, split = 0;
     size_t fixed = 0;
-    for (int lim : {kSmemLimit}) {
-        for (int c : {5, 3}) {
-            const int chunk = 64 * c;
-            p.c8 = (r + chunk - 1) / chunk;
-            p.c4 = (p.row4 + chunk - 1) / chunk;
-            p.pitch8 = round_up(p.c8 * chunk, 128) + 64;
-            p.pitch4 = round_up(p.c4 * chunk, 128) + 64;
-            fixed = kControlBytes + kSlotBytes + static_cast<size_t>(TP) * p.pitch8 +
-                    static_cast<size_t>(TT == 1 ? 2 : 1) * TP * p.pitch4;
-            cs = c;
-            nstages = fixed < static_cast<size_t>(lim)
-                          ? static_cast<int>((lim - fixed) / kWarps / (static_cast<size_t>(kItemRows) * chunk))
-                          : 0;
-            if (nstages >= 4) break;
+    bool found = false;
+    for (int pass = 0; pass < 2 && !found; ++pass) {
+        const int need = pass == 0 ? 4 : kMinStages;
+        for (int k = 0; k < 2; ++k) {
+            const int sp = TT == 1 ? 1 - k : k;  // measured: split staging pays for T <= 8 only
+            for (int c : {5, 3}) {
+                const int chunk = 64 * c;
+                p.c8 = (r + chunk - 1) / chunk;
+                p.c4 = (p.row4 + chunk - 1) / chunk;
+                p.pitch8 = round_up(p.c8 * chunk, 128) + 64;
+                p.pitch4 = round_up(p.c4 * chunk, 128) + 64;
+                fixed = kControlBytes + kSlotBytes + static_cast<size_t>(TP) * p.pitch8 +
+                        static_cast<size_t>(sp ? 2 : 1) * TP * p.pitch4;
+                cs = c;
+                split = sp;
+                nstages = fixed < static_cast<size_t>(kSmemLimit)
+                              ? static_cast<int>((kSmemLimit - fixed) / kWarps / (static_cast<size_t>(kItemRows) * chunk))
+                              : 0;
+                if (nstages >= need) { found = true; break; }
+            }
+            if (found) break;
         }
-        if (nstages >= kMinStages) break;
     }
-    if (nstages < kMinStages) return cudaErrorNotSupported;
+    if (!found) return cudaErrorNotSupported;
     if (nstages > kMaxStages) nstages = kMaxStages;
     p.nstages = nstages;
     p.early_weights = g_early_weights;
@@ -523,8 +563,17 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
     if (e != cudaSuccess) return e;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int grid = p.units < sms ? p.units : sms;
-    if (TT == 1) return cs == 5 ? launch_variant<1, 5>(t8, t4, p, grid, smem, st) : launch_variant<1, 3>(t8, t4, p, grid, smem, st);
-    return cs == 5 ? launch_variant<2, 5>(t8, t4, p, grid, smem, st) : launch_variant<2, 3>(t8, t4, p, grid, smem, st);
+    const int variant = (TT == 2 ? 4 : 0) + (cs == 5 ? 2 : 0) + split;
+    switch (variant) {
+        case 0: return launch_variant<1, 3, false>(t8, t4, p, grid, smem, st);
+        case 1: return launch_variant<1, 3, true>(t8, t4, p, grid, smem, st);
+        case 2: return launch_variant<1, 5, false>(t8, t4, p, grid, smem, st);
+        case 3: return launch_variant<1, 5, true>(t8, t4, p, grid, smem, st);
+        case 4: return launch_variant<2, 3, false>(t8, t4, p, grid, smem, st);
+        case 5: return launch_variant<2, 3, true>(t8, t4, p, grid, smem, st);
+        case 6: return launch_variant<2, 5, false>(t8, t4, p, grid, smem, st);
+        default: return launch_variant<2, 5, true>(t8, t4, p, grid, smem, st);
+    }
 }
 
 }  // namespace resq
