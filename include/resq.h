@@ -183,6 +183,10 @@ int resq_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t col
  * RESQ_OK, RESQ_ERR_TIMEOUT, or RESQ_ERR_CUDA if the stream reported an error. */
 int resq_device_status(void* stream);
 
+/* The CUDA runtime's description of the error behind the latest RESQ_ERR_CUDA that any entry point of
+ * this process returned ("no error" if there was none).  Host state, for diagnostics. */
+const char* resq_last_cuda_error(void);
+
 /* Static, human-readable name of a status code. */
 const char* resq_status_string(int status);
 

@@ -24,14 +24,15 @@ EXPORTS = [
     "resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_bytes", "resq_workspace_bytes",
     "resq_pack_weights", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
     "resq_unpack_int4", "resq_set_option",
-    "resq_device_status", "resq_status_string",
+    "resq_device_status", "resq_status_string", "resq_last_cuda_error",
 ]
 
 
 class ResqError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: status {status} ({status_string(status)})")
+        detail = f": {lib.resq_last_cuda_error().decode()}" if status == ERR_CUDA else ""
+        super().__init__(f"{where}: status {status} ({status_string(status)}{detail})")
 
 
 class LayerDesc(ctypes.Structure):
@@ -66,6 +67,8 @@ lib.resq_unpack_int4.argtypes = [_vp, _vp, _sz, _sz, _vp]
 lib.resq_set_option.argtypes = [_i, _i]
 lib.resq_device_status.argtypes = [_vp]
 lib.resq_status_string.restype = ctypes.c_char_p
+lib.resq_last_cuda_error.restype = ctypes.c_char_p
+lib.resq_last_cuda_error.argtypes = []
 lib.resq_status_string.argtypes = [_i]
 
 

@@ -79,7 +79,12 @@ Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     return w;
 }
 
-int cuda_status(cudaError_t e) { return e == cudaSuccess ? RESQ_OK : RESQ_ERR_CUDA; }
+cudaError_t g_last_cuda_error = cudaSuccess;  // what the latest RESQ_ERR_CUDA stood for
+int cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return RESQ_OK;
+    g_last_cuda_error = e;
+    return RESQ_ERR_CUDA;
+}
 
 }  // namespace
 }  // namespace resq
@@ -141,14 +146,14 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
     for (int t0 = 0; t0 < T; t0 += kPanelRows) {
         const int rows = T - t0 < kPanelRows ? T - t0 : kPanelRows;
         const char* Xp = static_cast<const char*>(X) + static_cast<size_t>(t0) * K * 2;
-        if (cudaError_t e = launch_project_gemm(Xp, P, rows, K, panel, st); e != cudaSuccess) return RESQ_ERR_CUDA;
+        if (cudaError_t e = launch_project_gemm(Xp, P, rows, K, panel, st); e != cudaSuccess) return cuda_status(e);
         if (cudaError_t e = launch_split_quantize(panel, true, rows, K, r, x8 + static_cast<size_t>(t0) * r,
                                                   x4 ? x4 + static_cast<size_t>(t0) * K4 / 2 : nullptr, s_x8 + t0,
                                                   s_x4 + t0, false,
                                                   x4_i8 ? x4_i8 + static_cast<size_t>(t0) * K4 : nullptr,
                                                   static_cast<size_t>(K) * 4, st);
             e != cudaSuccess)
-            return RESQ_ERR_CUDA;
+            return cuda_status(e);
     }
     return RESQ_OK;
 }
@@ -171,13 +176,13 @@ static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, 
     const int8_t* x4e = x4e_ready;
     if (!x4e) {
         int8_t* buf = reinterpret_cast<int8_t*>(ws + map.x4e);
-        if (cudaError_t e = launch_unpack_int4(x4, buf, T, K4, st); e != cudaSuccess) return RESQ_ERR_CUDA;
+        if (cudaError_t e = launch_unpack_int4(x4, buf, T, K4, st); e != cudaSuccess) return cuda_status(e);
         x4e = buf;
     }
     const int8_t* w4e = W->w4_i8;
     if (!w4e) {
         int8_t* buf = reinterpret_cast<int8_t*>(ws + map.w4e);
-        if (cudaError_t e = launch_unpack_int4(W->w4, buf, d->n_out, K4, st); e != cudaSuccess) return RESQ_ERR_CUDA;
+        if (cudaError_t e = launch_unpack_int4(W->w4, buf, d->n_out, K4, st); e != cudaSuccess) return cuda_status(e);
         w4e = buf;
     }
     return cuda_status(launch_mixed_gemm_tiles(T, d->n_out, d->K, d->r, x8, x4e, s_x8, s_x4, W->w8, w4e, W->s_w8,
@@ -264,6 +269,8 @@ int resq_device_status(void* stream) {
     }
     return RESQ_OK;
 }
+
+const char* resq_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 const char* resq_status_string(int s) {
     switch (s) {

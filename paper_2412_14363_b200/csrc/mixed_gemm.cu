@@ -2,13 +2,18 @@
 //
 // Persistent, warp-specialised kernel, one CTA per SM, 128 x 256 output tiles:
 //   warp 0     TMA producer: streams 128-byte-wide K blocks of the activation and weight codes
-//              into a 4-stage shared-memory ring (128-byte swizzle), first the INT8 segment, then
-//              the INT4 segment (codes one per byte, so both run on the i8 tensor path exactly);
+//              into a 4-stage shared-memory ring (128-byte swizzle), first the INT4 segment (codes
+//              one per byte, so both segments run on the i8 tensor path exactly), then the INT8 one;
 //   warp 1     owns TMEM (512 columns) and issues tcgen05.mma: the INT8 segment accumulates into
 //              columns [0,256), the INT4 segment into [256,512) -- two int32 accumulators per output
 //              because the two segments carry different (token, channel) scales;
-//   warps 2-5  epilogue: tcgen05.ld both accumulators, y = acc8*(sx8*sw8) + acc4*(sx4*sw4) in fp32,
-//              convert and store.
+//   warps 2-9  epilogue, two threads per tile row (128 columns each).
+// Two full-width accumulators fill TMEM, so there is no second buffer; the epilogue instead frees
+// the tensor pipe early.  It first copies its INT4 accumulator values into registers (raw int32,
+// 128 per thread) and releases those columns: the next tile's INT4 segment -- 7/8 of its work --
+// starts at once, while the epilogue goes on to read the INT8 accumulator, form
+// y = acc8*(sx8*sw8) + acc4*(sx4*sw4) in fp32, convert and store; the INT8 columns are released
+// long before the next tile's short INT8 segment needs them.
 // Out-of-range rows/columns/K are zero-filled by TMA and masked at the store.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -23,8 +28,8 @@ namespace {
 constexpr int BM = 128, BN = 256, BK = 128;  // BK in bytes == int8 elements
 constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK;
-constexpr int kThreads = 192;
-constexpr int kEpiThreads = 128;
+constexpr int kThreads = 320;
+constexpr int kEpiThreads = 256;
 constexpr uint32_t kTmemCols = 512;
 
 struct Params {
@@ -46,7 +51,8 @@ struct __align__(8) Shared {
     uint64_t full[STAGES];
     uint64_t empty[STAGES];
     uint64_t acc_full;
-    uint64_t acc_empty;
+    uint64_t acc4_empty;
+    uint64_t acc8_empty;
     uint64_t drain;
     uint32_t tmem_base;
     int abort_flag;
@@ -84,7 +90,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             mbar_init(&sh->empty[s], 1);
         }
         mbar_init(&sh->acc_full, 1);
-        mbar_init(&sh->acc_empty, kEpiThreads);
+        mbar_init(&sh->acc4_empty, kEpiThreads);
+        mbar_init(&sh->acc8_empty, kEpiThreads);
         mbar_init(&sh->drain, 1);
         sh->abort_flag = 0;
         fence_mbar_init();
@@ -114,12 +121,12 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                 for (int kb = 0; kb < kb_total; ++kb) {
                     if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
                     mbar_arrive_expect_tx(&sh->full[stage], A_BYTES + B_BYTES);
-                    if (kb < p.kb8) {
-                        tma_load_2d(sA + stage * A_BYTES, &tmA8, &sh->full[stage], kb * BK, m0);
-                        tma_load_2d(sB + stage * B_BYTES, &tmB8, &sh->full[stage], kb * BK, n0);
+                    if (kb < p.kb4) {
+                        tma_load_2d(sA + stage * A_BYTES, &tmA4, &sh->full[stage], kb * BK, m0);
+                        tma_load_2d(sB + stage * B_BYTES, &tmB4, &sh->full[stage], kb * BK, n0);
                     } else {
-                        tma_load_2d(sA + stage * A_BYTES, &tmA4, &sh->full[stage], (kb - p.kb8) * BK, m0);
-                        tma_load_2d(sB + stage * B_BYTES, &tmB4, &sh->full[stage], (kb - p.kb8) * BK, n0);
+                        tma_load_2d(sA + stage * A_BYTES, &tmA8, &sh->full[stage], (kb - p.kb4) * BK, m0);
+                        tma_load_2d(sB + stage * B_BYTES, &tmB8, &sh->full[stage], (kb - p.kb4) * BK, n0);
                     }
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -144,16 +151,22 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                if (!mbar_wait(&sh->acc_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+                // INT4 columns are free once the previous tile's epilogue has copied them out.
+                if (!mbar_wait(&sh->acc4_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 for (int kb = 0; kb < kb_total; ++kb) {
+                    const bool seg4 = kb < p.kb4;
+                    if (kb == p.kb4) {
+                        // ... the INT8 columns once it has finished with the tile.
+                        if (!mbar_wait(&sh->acc8_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                    }
                     if (!mbar_wait(&sh->full[stage], phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t a_desc = make_smem_desc_k128(smem_u32(sA + stage * A_BYTES));
                     const uint64_t b_desc = make_smem_desc_k128(smem_u32(sB + stage * B_BYTES));
-                    const bool seg8 = kb < p.kb8;
-                    const uint32_t d = tmem_base + (seg8 ? 0u : static_cast<uint32_t>(BN));
-                    const bool first = seg8 ? (kb == 0) : (kb == p.kb8);
+                    const uint32_t d = tmem_base + (seg4 ? static_cast<uint32_t>(BN) : 0u);
+                    const bool first = kb == 0 || kb == p.kb4;
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)
                         mma_i8_ss(d, a_desc + 2 * k, b_desc + 2 * k, idesc, (first && k == 0) ? 0u : 1u);
@@ -172,19 +185,20 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        const int quad = warp & 3;  // TMEM lane quadrant this warp may access
+        const int quad = warp & 3;            // TMEM lane quadrant this warp may access
+        const int ch = (warp - 2) >> 2;       // column half of the tile this warp handles
         const int et = threadIdx.x - 64;
         uint32_t acc_phase = 0;
-        // The 128 epilogue threads meet at named barriers, so they must leave the loop together:
+        // The epilogue threads meet at named barriers, so they must leave the loop together:
         // one thread samples the abort flag and the others take its reading.
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
             const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * BN;
             epi_barrier();  // previous tile's readers of sw8/sw4/epi_stop are done
             if (et == 0) sh->epi_stop = *abort_flag;
-            for (int j = et; j < BN; j += kEpiThreads) {
-                const int n = n0 + j;
-                sh->sw8[j] = n < p.N ? load_scale(p.s_w8, n, p.w_fp16) : 0.f;
-                sh->sw4[j] = n < p.N ? load_scale(p.s_w4, n, p.w_fp16) : 0.f;
+            {
+                const int n = n0 + et;
+                sh->sw8[et] = n < p.N ? load_scale(p.s_w8, n, p.w_fp16) : 0.f;
+                sh->sw4[et] = n < p.N ? load_scale(p.s_w4, n, p.w_fp16) : 0.f;
             }
             epi_barrier();
             if (sh->epi_stop) break;
@@ -195,37 +209,46 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             if (!mbar_wait(&sh->acc_full, acc_phase, abort_flag)) continue;  // flag is set; leave at the next sample
             acc_phase ^= 1;
             tc_fence_after();
-            const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t a8[32], a4[32];
-                tmem_ld32(lane_addr + c * 32, a8);
-                tmem_ld32(lane_addr + BN + c * 32, a4);
+            const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + ch * (BN / 2);
+            // Phase 1: the INT4 accumulator values of this thread's 128 columns, raw, into registers.
+            uint32_t a4[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(lane_addr + BN + c * 32, a4[c]);
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(&sh->acc4_empty);
+            // Phase 2: the INT8 accumulator, the scales, the store -- 16 columns at a time.
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                uint32_t a8[16];
+                tmem_ld16(lane_addr + c * 16, a8);
                 tmem_ld_wait();
-                const int nb = n0 + c * 32;
+                const int cb = ch * (BN / 2) + c * 16;  // first column of the chunk inside the tile
+                const int nb = n0 + cb;
+                const uint32_t* a4c = &a4[c >> 1][(c & 1) * 16];
                 if (row_ok) {
                     const size_t off = static_cast<size_t>(row) * p.N + nb;
                     if (p.dbg8) {
 #pragma unroll
-                        for (int g = 0; g < 8; ++g)
+                        for (int g = 0; g < 4; ++g)
                             if (nb + g * 4 < p.N) {
                                 reinterpret_cast<uint4*>(p.dbg8 + off)[g] =
                                     make_uint4(a8[4 * g], a8[4 * g + 1], a8[4 * g + 2], a8[4 * g + 3]);
                                 reinterpret_cast<uint4*>(p.dbg4 + off)[g] =
-                                    make_uint4(a4[4 * g], a4[4 * g + 1], a4[4 * g + 2], a4[4 * g + 3]);
+                                    make_uint4(a4c[4 * g], a4c[4 * g + 1], a4c[4 * g + 2], a4c[4 * g + 3]);
                             }
                     }
-                    float y[32];
+                    float y[16];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float t8 = static_cast<float>(static_cast<int>(a8[j])) * (sx8 * sh->sw8[c * 32 + j]);
-                        const float t4 = static_cast<float>(static_cast<int>(a4[j])) * (sx4 * sh->sw4[c * 32 + j]);
+                    for (int j = 0; j < 16; ++j) {
+                        const float t8 = static_cast<float>(static_cast<int>(a8[j])) * (sx8 * sh->sw8[cb + j]);
+                        const float t4 = static_cast<float>(static_cast<int>(a4c[j])) * (sx4 * sh->sw4[cb + j]);
                         y[j] = t8 + t4;
                     }
                     if (p.y_dtype == RESQ_Y_BF16) {
                         __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.Y) + off;
 #pragma unroll
-                        for (int g = 0; g < 4; ++g)
+                        for (int g = 0; g < 2; ++g)
                             if (nb + g * 8 < p.N) {
                                 uint32_t w[4];
 #pragma unroll
@@ -238,7 +261,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                     } else {
                         float* yp = reinterpret_cast<float*>(p.Y) + off;
 #pragma unroll
-                        for (int g = 0; g < 8; ++g)
+                        for (int g = 0; g < 4; ++g)
                             if (nb + g * 4 < p.N)
                                 reinterpret_cast<float4*>(yp)[g] =
                                     make_float4(y[4 * g], y[4 * g + 1], y[4 * g + 2], y[4 * g + 3]);
@@ -246,7 +269,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                 }
             }
             tc_fence_before();
-            mbar_arrive(&sh->acc_empty);
+            mbar_arrive(&sh->acc8_empty);
         }
     }
 
