@@ -48,6 +48,9 @@ void set_decode_early_weights(int on);
 // Online projection C = X·P (bf16 x bf16 -> fp32) on tcgen05 kind::f16; writes fp32 C [T][K].
 cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, float* C, cudaStream_t st);
 
+// Output-tile width of the two tile GEMMs (see the definition for what was measured).
+int pick_tile_width(int m_tiles, int N, int sms);
+
 // Driver entry point for tensor-map encoding (resolved once, without linking libcuda).
 void* tensor_map_encode_fn();
 

@@ -28,6 +28,8 @@ constexpr uint32_t kTmemCols = 512;
 struct Params {
     int T, K;
     int m_tiles, n_tiles, kb_total;
+    int bn;          // output columns per tile: a multiple of 16, <= BN (B loads and TMEM offsets stay BN wide)
+    int panel_tiles; // m tiles per row panel of the tile order
     float* C;
     int* status;
 };
@@ -59,6 +61,17 @@ __device__ __forceinline__ uint64_t make_smem_desc_mn128(uint32_t smem_addr, uin
 }
 
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+
+// Tile order: row panels of `panel_tiles` m tiles; inside a panel the m index runs fastest.  The CTAs
+// of one round then share a panel of X small enough to stay in L2 while the columns of P stream by.
+__device__ __forceinline__ void tile_coords(const Params& p, int tile, int& m0, int& n0) {
+    const int per_panel = p.panel_tiles * p.n_tiles;
+    const int panel = tile / per_panel, rem = tile - panel * per_panel;
+    const int mp = min(p.panel_tiles, p.m_tiles - panel * p.panel_tiles);  // m tiles in this panel
+    const int n = rem / mp, m = rem - n * mp;
+    m0 = (panel * p.panel_tiles + m) * BM;
+    n0 = n * p.bn;
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 project_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmP,
@@ -103,7 +116,8 @@ project_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * BN;
+                int m0, n0;
+                tile_coords(p, tile, m0, n0);
                 for (int kb = 0; kb < p.kb_total; ++kb) {
                     if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
                     mbar_arrive_expect_tx(&sh->full[stage], A_BYTES + B_BYTES);
@@ -128,7 +142,7 @@ project_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(BM, BN) | (1u << 16);  // B is N-major
+            const uint32_t idesc = make_idesc_bf16(BM, p.bn) | (1u << 16);  // B is N-major
             int stage = 0;
             uint32_t phase = 0;
             uint32_t acc_phase[2] = {0, 0};
@@ -166,7 +180,9 @@ project_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         uint32_t acc_phase[2] = {0, 0};
         int buf = 0;
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-            const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * BN;
+            int m0, n0;
+            tile_coords(p, tile, m0, n0);
+            const int n_end = min(p.K, n0 + p.bn);  // first column past this tile
             epi_barrier();
             if (et == 0) sh->epi_stop = *abort_flag;
             epi_barrier();
@@ -186,7 +202,7 @@ project_gemm_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                     float* cp = p.C + static_cast<size_t>(row) * p.K + nb;
 #pragma unroll
                     for (int g = 0; g < 8; ++g)
-                        if (nb + g * 4 < p.K)
+                        if (nb + g * 4 < n_end)
                             reinterpret_cast<uint4*>(cp)[g] = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
                 }
             }
@@ -239,13 +255,20 @@ cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, floa
     if (!make_map_bf16(&tX, X, T, K, BM) || !make_map_bf16(&tP, P, K, K, BK)) return cudaErrorInvalidValue;
     Params p;
     p.T = T; p.K = K;
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     p.m_tiles = (T + BM - 1) / BM;
-    p.n_tiles = (K + BN - 1) / BN;
+    p.bn = pick_tile_width(p.m_tiles, K, sms);
+    p.n_tiles = (K + p.bn - 1) / p.bn;
+    // Row panel: as many m tiles as keep the panel of X (rows x K bf16) within about 64 MB of L2.
+    {
+        const size_t tile_bytes = static_cast<size_t>(BM) * K * 2;
+        size_t pt = (64u << 20) / tile_bytes;
+        p.panel_tiles = pt < 1 ? 1 : (pt > static_cast<size_t>(p.m_tiles) ? p.m_tiles : static_cast<int>(pt));
+    }
     p.kb_total = (K + BK - 1) / BK;
     p.C = C;
     p.status = device_status_ptr();
-    int sms = 148;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int tiles = p.m_tiles * p.n_tiles;
     project_gemm_kernel<<<tiles < sms ? tiles : sms, kThreads, kSmemBytes, st>>>(tX, tP, p);
     return cudaGetLastError();
