@@ -375,11 +375,33 @@ def run_ours(args):
         h2d = sum(h.numel() * 2 for h in hx)
         d2h = sum(h.numel() * 2 for h in hy)
 
+        # Copies run on their own streams (PCIe is full duplex) so that the upload of the next layer's
+        # input and the download of the previous layer's output overlap the kernels of this one; every
+        # step still uploads all of its inputs and downloads all of its outputs inside the timed region.
+        up, down = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        in_ready = [torch.cuda.Event() for _ in layers]    # upload of layer i's input done
+        in_free = [torch.cuda.Event() for _ in layers]     # kernels that read dx[i] done
+        out_ready = [torch.cuda.Event() for _ in layers]   # kernels that wrote Y[i] done
+        out_free = [torch.cuda.Event() for _ in layers]    # download of Y[i] done
+        for e in in_free + out_free:
+            e.record(stream)
+
         def e2e_step():
             for i, L in enumerate(layers):
-                dx[i].copy_(hx[i], non_blocking=True)
+                with torch.cuda.stream(up):
+                    up.wait_event(in_free[i])
+                    dx[i].copy_(hx[i], non_blocking=True)
+                    in_ready[i].record(up)
+                stream.wait_event(in_ready[i])
+                stream.wait_event(out_free[i])
                 resq.resq_linear(L.W, dx[i], L.P, L.Y, L.ws)
-                hy[i].copy_(L.Y, non_blocking=True)
+                in_free[i].record(stream)
+                out_ready[i].record(stream)
+                with torch.cuda.stream(down):
+                    down.wait_event(out_ready[i])
+                    hy[i].copy_(L.Y, non_blocking=True)
+                    out_free[i].record(down)
+            stream.wait_stream(down)  # the step ends when its last result is on the host
 
         for _ in range(3):
             e2e_step()

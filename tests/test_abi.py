@@ -89,3 +89,12 @@ def test_host_validation_happens_before_any_launch(resq):
     assert L.resq_mixed_gemm(ctypes.byref(good), 64, fake, fake, None, fake, fake, W, fake, 0, None, None, fake, need - 1, None) == resq.ERR_WORKSPACE
     assert L.resq_mixed_gemm(ctypes.byref(good), 64, fake, fake, None, fake, fake, W, fake, 0, None, None, None, 0, None) == resq.ERR_WORKSPACE
     assert L.resq_linear(ctypes.byref(good), 64, fake, None, W, fake, 0, fake, 16, None) == resq.ERR_WORKSPACE
+
+
+def test_options_and_error_text(resq):
+    """Host-only entry points: an unknown option is refused, the known one toggles, and the CUDA error
+    text is a string even when no CUDA error has occurred."""
+    assert resq.lib.resq_set_option(12345, 1) == resq.ERR_SHAPE
+    assert resq.lib.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 1) == resq.OK
+    assert resq.lib.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 0) == resq.OK
+    assert isinstance(resq.lib.resq_last_cuda_error(), bytes)
