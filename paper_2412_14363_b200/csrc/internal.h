@@ -51,6 +51,9 @@ cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, floa
 // Output-tile width of the two tile GEMMs (see the definition for what was measured).
 int pick_tile_width(int m_tiles, int N, int sms);
 
+// Same product on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles).
+cudaError_t launch_project_gemm_pair(const void* X, const void* P, int T, int K, float* C, cudaStream_t st);
+
 // Driver entry point for tensor-map encoding (resolved once, without linking libcuda).
 void* tensor_map_encode_fn();
 
