@@ -1,20 +1,28 @@
-// Many-token mixed-precision GEMM (Eq. 4 + dequantizing epilogue) on tcgen05 kind::i8.
+// Many-token mixed-precision GEMM (Eq. 4 + dequantizing epilogue) on tcgen05 kind::i8, CTA pairs.
 //
-// Persistent, warp-specialised kernel, one CTA per SM, 128 x 256 output tiles:
-//   warp 0     TMA producer: streams 128-byte-wide K blocks of the activation and weight codes
-//              into a 4-stage shared-memory ring (128-byte swizzle), first the INT4 segment (codes
-//              one per byte, so both segments run on the i8 tensor path exactly), then the INT8 one;
-//   warp 1     owns TMEM (512 columns) and issues tcgen05.mma: the INT8 segment accumulates into
-//              columns [0,256), the INT4 segment into [256,512) -- two int32 accumulators per output
-//              because the two segments carry different (token, channel) scales;
-//   warps 2-9  epilogue, two threads per tile row (128 columns each).
+// Persistent, warp-specialised kernel.  Two CTAs on neighbouring SMs (a cluster of 2) share one
+// 256 x 256 output tile (tcgen05 cta_group::2): each stages its own 128 token rows and only its own
+// 128 of the tile's 256 weight rows, 32 KB per K block, so six stages fit and the shared-memory read
+// rate per MMA is a third lower than with one CTA per 128 x 256 tile.
+//   warp 0     TMA producer (both CTAs): streams 128-byte-wide K blocks of the activation and weight
+//              codes into the ring (128-byte swizzle), first the INT4 segment (codes one per byte, so
+//              both segments run on the i8 tensor path exactly), then the INT8 one.  Completion bytes
+//              of both CTAs are counted on the even CTA's barrier.
+//   warp 1     TMEM allocation (both CTAs; 512 columns); MMA issue (even CTA only): the INT8 segment
+//              accumulates into columns [0,256), the INT4 segment into [256,512) -- two int32
+//              accumulators per output because the two segments carry different (token, channel)
+//              scales.  Each CTA's TMEM receives the rows of its own 128 tokens.
+//   warps 2-9  epilogue (both CTAs), two threads per tile row (128 columns each).
 // Two full-width accumulators fill TMEM, so there is no second buffer; the epilogue instead frees
 // the tensor pipe early.  It first copies its INT4 accumulator values into registers (raw int32,
 // 128 per thread) and releases those columns: the next tile's INT4 segment -- 7/8 of its work --
 // starts at once, while the epilogue goes on to read the INT8 accumulator, form
 // y = acc8*(sx8*sw8) + acc4*(sx4*sw4) in fp32, convert and store; the INT8 columns are released
 // long before the next tile's short INT8 segment needs them.
-// Out-of-range rows/columns/K are zero-filled by TMA and masked at the store.
+// Barriers signalled across the pair: `full` (odd CTA's copies -> even CTA), `empty` and `acc_full`
+// (tcgen05.commit, multicast to both), `acc4_empty` / `acc8_empty` (epilogue threads of both CTAs ->
+// even CTA).  No TMA multicast.  Out-of-range rows/columns/K are zero-filled by TMA and masked at
+// the store.  All waits are bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -26,8 +34,9 @@ namespace resq {
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 128;  // BK in bytes == int8 elements
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK;
+constexpr int STAGES = 6;
+constexpr int BN_HALF = BN / 2;  // weight rows staged by each CTA of the pair
+constexpr int A_BYTES = BM * BK, B_BYTES = BN_HALF * BK;
 constexpr int kThreads = 320;
 constexpr int kEpiThreads = 256;
 constexpr uint32_t kTmemCols = 512;
@@ -54,7 +63,6 @@ struct __align__(8) Shared {
     uint64_t acc_full;
     uint64_t acc4_empty;
     uint64_t acc8_empty;
-    uint64_t drain;
     uint32_t tmem_base;
     int abort_flag;
     int epi_stop;
@@ -70,7 +78,7 @@ __device__ __forceinline__ float load_scale(const void* p, int i, int fp16) {
 
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constant__ CUtensorMap tmA4,
                   const __grid_constant__ CUtensorMap tmB8, const __grid_constant__ CUtensorMap tmB4,
                   const Params p) {
@@ -82,7 +90,9 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
     volatile int* abort_flag = &sh->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_tiles = p.m_tiles * p.n_tiles;
+    const int rank = static_cast<int>(cluster_ctarank());  // 0: even CTA (issues the MMAs), 1: its peer
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int num_tiles = p.m_tiles * p.n_tiles;  // m_tiles counts 256-row pair tiles
     const int kb_total = p.kb8 + p.kb4;
 
     if (threadIdx.x == 0) {
@@ -91,9 +101,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             mbar_init(&sh->empty[s], 1);
         }
         mbar_init(&sh->acc_full, 1);
-        mbar_init(&sh->acc4_empty, kEpiThreads);
-        mbar_init(&sh->acc8_empty, kEpiThreads);
-        mbar_init(&sh->drain, 1);
+        mbar_init(&sh->acc4_empty, 2 * kEpiThreads);  // used in the even CTA: epilogue threads of both CTAs
+        mbar_init(&sh->acc8_empty, 2 * kEpiThreads);
         sh->abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tmA8);
@@ -102,11 +111,12 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
         tma_prefetch_desc(&tmB4);
     }
     if (warp == 1) {
-        tmem_alloc(&sh->tmem_base, kTmemCols);
-        tmem_relinquish();
+        tmem_alloc_pair(&sh->tmem_base, kTmemCols);
+        tmem_relinquish_pair();
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();  // the peer's barriers exist before anything is signalled across
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
 
@@ -115,43 +125,40 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            int issued = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * p.bn;
+            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+                const int m0 = (tile % p.m_tiles) * 2 * BM + rank * BM;        // this CTA's token rows
+                const int n0 = (tile / p.m_tiles) * p.bn + rank * BN_HALF;     // this CTA's weight rows
                 for (int kb = 0; kb < kb_total; ++kb) {
                     if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
-                    mbar_arrive_expect_tx(&sh->full[stage], A_BYTES + B_BYTES);
+                    // The even CTA arms its barrier for the bytes of both CTAs; the peer only sends its
+                    // bytes there (if they land first, the pending arrival keeps the phase open).
+                    const uint32_t full_addr = cluster_map(&sh->full[stage], 0);
+                    if (rank == 0) mbar_arrive_expect_tx(&sh->full[stage], 2 * (A_BYTES + B_BYTES));
                     if (kb < p.kb4) {
-                        tma_load_2d(sA + stage * A_BYTES, &tmA4, &sh->full[stage], kb * BK, m0);
-                        tma_load_2d(sB + stage * B_BYTES, &tmB4, &sh->full[stage], kb * BK, n0);
+                        tma_load_2d_pair(sA + stage * A_BYTES, &tmA4, full_addr, kb * BK, m0);
+                        tma_load_2d_pair(sB + stage * B_BYTES, &tmB4, full_addr, kb * BK, n0);
                     } else {
-                        tma_load_2d(sA + stage * A_BYTES, &tmA8, &sh->full[stage], (kb - p.kb4) * BK, m0);
-                        tma_load_2d(sB + stage * B_BYTES, &tmB8, &sh->full[stage], (kb - p.kb4) * BK, n0);
+                        tma_load_2d_pair(sA + stage * A_BYTES, &tmA8, full_addr, (kb - p.kb4) * BK, m0);
+                        tma_load_2d_pair(sB + stage * B_BYTES, &tmB8, full_addr, (kb - p.kb4) * BK, n0);
                     }
-                    ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
             if (!ok) {
-                // Let the copies already in flight land before the CTA gives up its shared memory.
-                int n = issued < STAGES ? issued : STAGES;
-                for (int i = 0; i < n; ++i) {
-                    if (stage == 0) { stage = STAGES; phase ^= 1; }
-                    --stage;
-                    const uint64_t t0 = global_timer_ns();
-                    while (!mbar_try_wait(&sh->full[stage], phase) && global_timer_ns() - t0 < 100000000ull) {}
-                }
+                // Give the copies already in flight time to land before the CTA gives up its shared memory.
+                const uint64_t t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 1000000ull) {}
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_i8(BM, p.bn);
+        // ------------------------------------------------------------ MMA issuer (even CTA only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_i8(2 * BM, p.bn);
             int stage = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
                 // INT4 columns are free once the previous tile's epilogue has copied them out.
                 if (!mbar_wait(&sh->acc4_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -170,18 +177,13 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                     const bool first = kb == 0 || kb == p.kb4;
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)
-                        mma_i8_ss(d, a_desc + 2 * k, b_desc + 2 * k, idesc, (first && k == 0) ? 0u : 1u);
-                    tc_commit(&sh->empty[stage]);  // frees the ring slot once these MMAs have read it
+                        mma_i8_ss_pair(d, a_desc + 2 * k, b_desc + 2 * k, idesc, (first && k == 0) ? 0u : 1u);
+                    tc_commit_pair(&sh->empty[stage], 3);  // frees the ring slot in both CTAs once these MMAs have read it
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
-                tc_commit(&sh->acc_full);
+                tc_commit_pair(&sh->acc_full, 3);
                 acc_phase ^= 1;
-            }
-            if (!ok) {
-                tc_commit(&sh->drain);
-                const uint64_t t0 = global_timer_ns();
-                while (!mbar_try_wait(&sh->drain, 0) && global_timer_ns() - t0 < 100000000ull) {}
             }
         }
     } else {
@@ -192,8 +194,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
         uint32_t acc_phase = 0;
         // The epilogue threads meet at named barriers, so they must leave the loop together:
         // one thread samples the abort flag and the others take its reading.
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-            const int m0 = (tile % p.m_tiles) * BM, n0 = (tile / p.m_tiles) * p.bn;
+        for (int tile = pair; tile < num_tiles; tile += npairs) {
+            const int m0 = (tile % p.m_tiles) * 2 * BM + rank * BM, n0 = (tile / p.m_tiles) * p.bn;
             epi_barrier();  // previous tile's readers of sw8/sw4/epi_stop are done
             if (et == 0) sh->epi_stop = *abort_flag;
             const int n_end = min(p.N, n0 + p.bn);  // first column past this tile
@@ -218,7 +220,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             for (int c = 0; c < 4; ++c) tmem_ld32(lane_addr + BN + c * 32, a4[c]);
             tmem_ld_wait();
             tc_fence_before();
-            mbar_arrive(&sh->acc4_empty);
+            mbar_arrive_cluster(cluster_map(&sh->acc4_empty, 0));
             // Phase 2: the INT8 accumulator, the scales, the store -- 16 columns at a time.
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
@@ -271,17 +273,18 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                 }
             }
             tc_fence_before();
-            mbar_arrive(&sh->acc8_empty);
+            mbar_arrive_cluster(cluster_map(&sh->acc8_empty, 0));
         }
     }
 
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();  // neither CTA leaves while the other may still read its shared memory or signal it
     if (threadIdx.x == 0 && sh->abort_flag) atomicOr(p.status, RESQ_ERR_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
+        tmem_dealloc_pair(tmem_base, kTmemCols);
     }
 }
 
@@ -327,13 +330,13 @@ cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8
     const int K4 = K - r;
     CUtensorMap tA8, tA4, tB8, tB4;
     if (!make_map_u8(&tA8, x8, T, r, BM) || !make_map_u8(&tA4, x4e, T, K4, BM) ||
-        !make_map_u8(&tB8, w8, N, r, BN) || !make_map_u8(&tB4, w4e, N, K4, BN))
+        !make_map_u8(&tB8, w8, N, r, BN_HALF) || !make_map_u8(&tB4, w4e, N, K4, BN_HALF))
         return cudaErrorInvalidValue;
     Params p;
     p.T = T; p.N = N; p.r = r; p.K4 = K4;
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    p.m_tiles = (T + BM - 1) / BM;
+    p.m_tiles = (T + 2 * BM - 1) / (2 * BM);
     p.bn = pick_tile_width(p.m_tiles, N, sms);
     p.n_tiles = (N + p.bn - 1) / p.bn;
     p.kb8 = (r + BK - 1) / BK;
@@ -343,8 +346,8 @@ cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8
     p.Y = Y; p.y_dtype = y_dtype; p.dbg8 = dbg8; p.dbg4 = dbg8 ? dbg4 : nullptr;
     p.status = device_status_ptr();
     const int tiles = p.m_tiles * p.n_tiles;
-    const int grid = tiles < sms ? tiles : sms;
-    mixed_gemm_kernel<<<grid, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
+    const int pairs = tiles < sms / 2 ? tiles : sms / 2;
+    mixed_gemm_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
     return cudaGetLastError();
 }
 
