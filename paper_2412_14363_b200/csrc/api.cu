@@ -79,7 +79,6 @@ Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     return w;
 }
 
-int g_projection_pair = 1;  // TEMP: A/B switch
 cudaError_t g_last_cuda_error = cudaSuccess;  // what the latest RESQ_ERR_CUDA stood for
 int cuda_status(cudaError_t e) {
     if (e == cudaSuccess) return RESQ_OK;
@@ -147,9 +146,7 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
     for (int t0 = 0; t0 < T; t0 += kPanelRows) {
         const int rows = T - t0 < kPanelRows ? T - t0 : kPanelRows;
         const char* Xp = static_cast<const char*>(X) + static_cast<size_t>(t0) * K * 2;
-        if (cudaError_t e = (g_projection_pair ? launch_project_gemm_pair : launch_project_gemm)(Xp, P, rows, K, panel, st);
-            e != cudaSuccess)
-            return cuda_status(e);
+        if (cudaError_t e = launch_project_gemm(Xp, P, rows, K, panel, st); e != cudaSuccess) return cuda_status(e);
         if (cudaError_t e = launch_split_quantize(panel, true, rows, K, r, x8 + static_cast<size_t>(t0) * r,
                                                   x4 ? x4 + static_cast<size_t>(t0) * K4 / 2 : nullptr, s_x8 + t0,
                                                   s_x4 + t0, false,
@@ -256,7 +253,6 @@ int resq_set_option(int option, int value) {
         set_decode_early_weights(value);
         return RESQ_OK;
     }
-    if (option == 2) { g_projection_pair = value; return RESQ_OK; }  // TEMP
     return RESQ_ERR_SHAPE;
 }
 

@@ -45,14 +45,11 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
                                      int32_t* dbg8, int32_t* dbg4, cudaStream_t st);
 void set_decode_early_weights(int on);
 
-// Online projection C = X·P (bf16 x bf16 -> fp32) on tcgen05 kind::f16; writes fp32 C [T][K].
+// Online projection C = X·P (bf16 x bf16 -> fp32) on tcgen05 kind::f16, CTA pairs; writes fp32 C [T][K].
 cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, float* C, cudaStream_t st);
 
 // Output-tile width of the two tile GEMMs (see the definition for what was measured).
 int pick_tile_width(int m_tiles, int N, int sms);
-
-// Same product on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles).
-cudaError_t launch_project_gemm_pair(const void* X, const void* P, int T, int K, float* C, cudaStream_t st);
 
 // Driver entry point for tensor-map encoding (resolved once, without linking libcuda).
 void* tensor_map_encode_fn();
