@@ -113,6 +113,14 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
                           size_t workspace_bytes, void* stream);
 
 /*
+ * The online projection alone (Section 4.3, U_D): C = X·P with X bf16 [T][K], P bf16 [K][K] (row i =
+ * input feature, column j = coefficient), C fp32 [T][K], bf16 products accumulated in fp32 on the
+ * tensor cores.  This is the first half of resq_project_quantize with P != NULL, exposed so that the
+ * coefficients can be inspected and the GEMM timed on its own.  K % 8 == 0.
+ */
+int resq_project(const void* X, const void* P, int T, int K, float* C, void* stream);
+
+/*
  * Eq. 4 with the dequantizing epilogue: Y = diag(s_x8)(x8·w8^T)diag(s_w8) + diag(s_x4)(x4·w4^T)diag(s_w4).
  * Integer products accumulate exactly in int32; the epilogue is fp32:
  *     y = (float)acc8 * (s_x8[t] * s_w8[n]) + (float)acc4 * (s_x4[t] * s_w4[n])

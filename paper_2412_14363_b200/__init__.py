@@ -22,7 +22,7 @@ Y_BF16, Y_FP32 = 0, 1
 
 EXPORTS = [
     "resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_bytes", "resq_workspace_bytes",
-    "resq_pack_weights", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
+    "resq_pack_weights", "resq_project", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
     "resq_unpack_int4", "resq_set_option",
     "resq_device_status", "resq_status_string", "resq_last_cuda_error",
 ]
@@ -58,6 +58,7 @@ for _n in ("resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_byt
 lib.resq_workspace_bytes.restype = _sz
 lib.resq_workspace_bytes.argtypes = [_dp, _i, _i, _i]
 lib.resq_pack_weights.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.resq_project.argtypes = [_vp, _vp, _i, _i, _vp, _vp]
 lib.resq_project_quantize.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 lib.resq_project_quantize_static.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_mixed_gemm.argtypes = [_dp, _i, _vp, _vp, _vp, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _i, _vp, _vp,
@@ -138,6 +139,12 @@ def resq_project_quantize(X, P, r: int, x8, x4, s_x8, s_x4, x4_i8=None, workspac
                                      _ptr(x4_i8), _ptr(workspace),
                                      0 if workspace is None else workspace.numel() * workspace.element_size(),
                                      _stream()), "resq_project_quantize")
+
+
+def resq_project(X, P, C):
+    """C (fp32 [T][K]) = X (bf16 [T][K]) · P (bf16 [K][K]): the online projection alone."""
+    T, K = X.shape
+    _check(lib.resq_project(_ptr(X), _ptr(P), T, K, _ptr(C), _stream()), "resq_project")
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

@@ -158,6 +158,14 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
     return RESQ_OK;
 }
 
+int resq_project(const void* X, const void* P, int T, int K, float* C, void* stream) {
+    if (T < 1 || K <= 0 || K % 8 != 0) return RESQ_ERR_SHAPE;
+    if (!X || !P || !C) return RESQ_ERR_NULL;
+    if (!aligned16(X) || !aligned16(P) || !aligned16(C)) return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_project_gemm(X, P, T, K, C, static_cast<cudaStream_t>(stream)));
+}
+
 static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, const uint8_t* x4,
                            const int8_t* x4e_ready, const float* s_x8, const float* s_x4, const resq_weights_t* W,
                            void* Y, int y_dtype, int32_t* dbg8, int32_t* dbg4, char* ws, const Workspace& map,

@@ -85,3 +85,19 @@ def test_linear_with_online_projection_is_exact_given_its_own_codes(resq):
     # PCA basis, so the error is that of rotation-only 4-bit quantization: a sanity bound, not parity)
     ref = (synth.bf16_bits_to_f32(X_bits).astype(np.float64) @ synth.bf16_bits_to_f32(P_bits).astype(np.float64)) @ Wp.astype(np.float64).T
     assert np.linalg.norm(host(y32) - ref) / np.linalg.norm(ref) < 0.35
+
+
+@pytest.mark.parametrize("T,K", [(1, 512), (130, 1056), (300, 2048), (520, 4096)])
+def test_projection_alone_against_fp64_sums(resq, T, K):
+    """resq_project: every fp32 coefficient within the accumulation error of the fp64-summed oracle value
+    (one truncating fp32 add per 16-term block: K/16 + 4 ulp of the sum of the term magnitudes)."""
+    X_bits = synth.f32_to_bf16_bits(synth.activations(T, K, "t4", seed=700 + T))
+    P_bits = synth.f32_to_bf16_bits(synth.kron_orthogonal_bf16(K, inner=32 if K % 128 else 128))
+    C_ref = oracle.project(X_bits, P_bits)
+    C = torch.full((T, K), float("nan"), dtype=torch.float32, device="cuda")
+    resq.resq_project(bf16_to_dev(X_bits), bf16_to_dev(P_bits), C)
+    assert resq.resq_device_status() == resq.OK
+    Xf = np.abs(synth.bf16_bits_to_f32(X_bits).astype(np.float64))
+    Pf = np.abs(synth.bf16_bits_to_f32(P_bits).astype(np.float64))
+    bound = (K // 16 + 4) * 2.0 ** -24 * (Xf @ Pf) + 1e-30
+    assert (np.abs(host(C).astype(np.float64) - C_ref.astype(np.float64)) <= bound).all()
