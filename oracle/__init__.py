@@ -37,6 +37,7 @@ def _c():
         _lib = ctypes.CDLL(build())
         _lib.oracle_quantize_vector.restype = ctypes.c_float
         _lib.oracle_int_gemm.restype = ctypes.c_long
+        _lib.oracle_int_gemm_u8.restype = ctypes.c_long
         _lib.oracle_num_threads.restype = ctypes.c_int
     return _lib
 
@@ -199,3 +200,91 @@ def linear(X_bits, P_bits, pw: PackedWeights) -> LayerResult:
     the previous layer's weights, Section 4.3); otherwise C = X·P is formed online first."""
     C = bf16_bits_to_f32(X_bits) if P_bits is None else project(X_bits, P_bits)
     return linear_from_coeff(C, pw)
+
+
+# --------------------------------------------------------------------------- asymmetric activations (Section 5.1)
+def split_quantize_asym(C, r: int):
+    """Rows of C [rows][K] fp32 -> (u8 [rows][r], u4 [rows][K-r] one code per byte, s8, s4, z8, z4):
+    Eq. 1 in its asymmetric form per row and segment (z = min, s = (max - min) / (2^N - 1))."""
+    C = _chk(C, np.float32)
+    rows, K = C.shape
+    u8 = np.empty((rows, r), np.uint8)
+    u4 = np.empty((rows, K - r), np.uint8)
+    s8, s4, z8, z4 = (np.empty(rows, np.float32) for _ in range(4))
+    _c().oracle_split_quantize_asym(_p(C), ctypes.c_long(rows), int(K), int(r), _p(u8), _p(u4),
+                                    _p(s8), _p(s4), _p(z8), _p(z4))
+    return u8, u4, s8, s4, z8, z4
+
+
+def int_gemm_u8(u, w):
+    """acc[t][n] = sum_j u[t][j]·w[n][j], unsigned activation codes, int64 checked to fit int32."""
+    u = _chk(u, np.uint8)
+    w = _chk(w, np.int8)
+    T, Ks = u.shape
+    N, Ks2 = w.shape
+    assert Ks == Ks2
+    acc = np.empty((T, N), np.int32)
+    bad = _c().oracle_int_gemm_u8(_p(u), _p(w), ctypes.c_long(T), ctypes.c_long(N), int(Ks), _p(acc))
+    if bad:
+        raise OverflowError(f"{bad} accumulators exceed int32")
+    return acc
+
+
+def weight_row_sums(w):
+    w = _chk(w, np.int8)
+    N, Ks = w.shape
+    out = np.empty(N, np.int32)
+    _c().oracle_weight_row_sums(_p(w), ctypes.c_long(N), int(Ks), _p(out))
+    return out
+
+
+def pack_nibbles_u(code):
+    """Unsigned 4-bit codes (0..15), one per byte -> two per byte, code 2i in the low nibble."""
+    code = _chk(code, np.uint8)
+    return pack_nibbles(code.view(np.int8))
+
+
+def epilogue_asym(acc8, acc4, s_x8, s_x4, z_x8, z_x4, s_w8, s_w4, wsum8, wsum4):
+    acc8, acc4 = _chk(acc8, np.int32), _chk(acc4, np.int32)
+    T, N = acc8.shape
+    f = lambda a: _chk(a, np.float32)
+    s_x8, s_x4, z_x8, z_x4, s_w8, s_w4 = f(s_x8), f(s_x4), f(z_x8), f(z_x4), f(s_w8), f(s_w4)
+    wsum8, wsum4 = _chk(wsum8, np.int32), _chk(wsum4, np.int32)
+    y32 = np.empty((T, N), np.float32)
+    ybf = np.empty((T, N), np.uint16)
+    _c().oracle_epilogue_asym(_p(acc8), _p(acc4), _p(s_x8), _p(s_x4), _p(z_x8), _p(z_x4), _p(s_w8), _p(s_w4),
+                              _p(wsum8), _p(wsum4), ctypes.c_long(T), ctypes.c_long(N), _p(y32), _p(ybf))
+    return y32, ybf
+
+
+@dataclass
+class AsymLayerResult:
+    coeff: np.ndarray
+    u8: np.ndarray          # uint8 codes [T][r]
+    u4: np.ndarray          # uint8 codes 0..15, one per byte [T][K-r]
+    u4_packed: np.ndarray
+    s_x8: np.ndarray
+    s_x4: np.ndarray
+    z_x8: np.ndarray
+    z_x4: np.ndarray
+    acc8: np.ndarray
+    acc4: np.ndarray
+    wsum8: np.ndarray
+    wsum4: np.ndarray
+    y32: np.ndarray
+    ybf: np.ndarray
+
+
+def linear_asym_from_coeff(C, pw: PackedWeights) -> AsymLayerResult:
+    u8, u4, s8, s4, z8, z4 = split_quantize_asym(C, pw.r)
+    acc8, acc4 = int_gemm_u8(u8, pw.q8), int_gemm_u8(u4, pw.q4)
+    ws8, ws4 = weight_row_sums(pw.q8), weight_row_sums(pw.q4)
+    y32, ybf = epilogue_asym(acc8, acc4, s8, s4, z8, z4, pw.s8, pw.s4, ws8, ws4)
+    return AsymLayerResult(np.asarray(C, np.float32), u8, u4, pack_nibbles_u(u4), s8, s4, z8, z4, acc8, acc4,
+                           ws8, ws4, y32, ybf)
+
+
+def linear_asym(X_bits, P_bits, pw: PackedWeights) -> AsymLayerResult:
+    """Whole layer with asymmetric per-token activations and symmetric per-channel weights."""
+    C = bf16_bits_to_f32(X_bits) if P_bits is None else project(X_bits, P_bits)
+    return linear_asym_from_coeff(C, pw)

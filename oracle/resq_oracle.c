@@ -9,6 +9,7 @@
  *   Eq. 2 (Section 4.1) activation coefficients X·U: r of them at H = 8 bits, the other d - r at L = 4 bits
  *   Eq. 3 (Section 4.1) projected weights U^T·W quantized the same way, one scale per output channel and segment
  *   Eq. 4 (Section 4.1) layer output = low-precision product + high-precision product (no cross terms)
+ * and, further down, the asymmetric form of Eq. 1 for the activations (Section 5.1) with its epilogue.
  *
  * Readings where the paper is silent: rounding is to nearest, ties to even, in fp32 (rintf under the
  * default rounding mode); s and x/s are IEEE fp32 divisions; a zero segment gets s = 0 and codes 0;
@@ -143,6 +144,96 @@ void oracle_epilogue(const int32_t* acc8, const int32_t* acc4, const float* s_x8
         for (long n = 0; n < N; ++n) {
             double y = (double)acc8[t * N + n] * (double)s_x8[t] * (double)s_w8[n] +
                        (double)acc4[t * N + n] * (double)s_x4[t] * (double)s_w4[n];
+            float yf = (float)y;
+            y32[t * N + n] = yf;
+            if (ybf) ybf[t * N + n] = f32_to_bf16(yf);
+        }
+    }
+}
+
+/* ====================================================================================================
+ * Asymmetric per-token activations (Eq. 1, second form; the setting of the paper's experiments, Section 5.1):
+ *     z = min(x),  s = (max(x) - min(x)) / (2^N - 1),  code = round((x - z) / s) clipped to [0, 2^N - 1],
+ *     dequantized value = code * s + z.
+ * Readings where the paper is silent: max - min, x - z and the two divisions are IEEE fp32 operations in this
+ * order; rounding is to nearest, ties to even; a constant segment gets s = 0 and codes 0 (its dequantized value
+ * is z exactly); the zero-point stays an fp32 number (it is not snapped to the integer grid).
+ * With symmetric weights (Eq. 3) the layer output (Eq. 4) becomes, per segment,
+ *     sum_j (code_j * s_x + z_x) * (w_j * s_w) = s_x * s_w * sum_j code_j * w_j  +  z_x * s_w * sum_j w_j,
+ * i.e. the integer product plus a rank-one term with the integer row sums of the weight codes.
+ * ==================================================================================================== */
+void oracle_quantize_vector_asym(const float* x, long n, int bits, uint8_t* code, float* s_out, float* z_out) {
+    const float qmax = (float)((1 << bits) - 1);
+    float lo = x[0], hi = x[0];
+    for (long j = 1; j < n; ++j) {
+        if (x[j] < lo) lo = x[j];
+        if (x[j] > hi) hi = x[j];
+    }
+    const float range = hi - lo;
+    const float s = range / qmax;
+    *z_out = lo;
+    if (!(s > 0.0f)) {
+        for (long j = 0; j < n; ++j) code[j] = 0;
+        *s_out = 0.0f;
+        return;
+    }
+    *s_out = s;
+    for (long j = 0; j < n; ++j) {
+        const float d = x[j] - lo;
+        float q = rintf(d / s);
+        if (q < 0.0f) q = 0.0f;
+        if (q > qmax) q = qmax;
+        code[j] = (uint8_t)q;
+    }
+}
+
+/* u8 [rows][r], u4 [rows][K-r] (one code per byte), s8/s4/z8/z4 [rows]. */
+void oracle_split_quantize_asym(const float* C, long rows, int K, int r, uint8_t* u8, uint8_t* u4,
+                                float* s8, float* s4, float* z8, float* z4) {
+    const int K4 = K - r;
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < rows; ++t) {
+        oracle_quantize_vector_asym(C + t * K, r, 8, u8 + t * r, s8 + t, z8 + t);
+        oracle_quantize_vector_asym(C + t * K + r, K4, 4, u4 + t * K4, s4 + t, z4 + t);
+    }
+}
+
+/* acc[t][n] = sum_j u[t][j] * w[n][j] with unsigned activation codes; int64, overflow count returned. */
+long oracle_int_gemm_u8(const uint8_t* u, const int8_t* w, long T, long N, int Kseg, int32_t* acc) {
+    long overflow = 0;
+#pragma omp parallel for schedule(static) reduction(+ : overflow)
+    for (long t = 0; t < T; ++t) {
+        for (long n = 0; n < N; ++n) {
+            int64_t a = 0;
+            for (int j = 0; j < Kseg; ++j) a += (int64_t)u[t * Kseg + j] * (int64_t)w[n * Kseg + j];
+            if (a > INT32_MAX || a < INT32_MIN) overflow += 1;
+            acc[t * N + n] = (int32_t)a;
+        }
+    }
+    return overflow;
+}
+
+/* Row sums of the weight codes: wsum[n] = sum_j w[n][j]. */
+void oracle_weight_row_sums(const int8_t* w, long N, int Kseg, int32_t* wsum) {
+    for (long n = 0; n < N; ++n) {
+        int64_t a = 0;
+        for (int j = 0; j < Kseg; ++j) a += w[n * Kseg + j];
+        wsum[n] = (int32_t)a;
+    }
+}
+
+/* y = acc8*s_x8*s_w8 + z_x8*s_w8*wsum8 + acc4*s_x4*s_w4 + z_x4*s_w4*wsum4 in fp64 from the stored fp32
+ * values, rounded once to fp32 and from there to bf16. */
+void oracle_epilogue_asym(const int32_t* acc8, const int32_t* acc4, const float* s_x8, const float* s_x4,
+                          const float* z_x8, const float* z_x4, const float* s_w8, const float* s_w4,
+                          const int32_t* wsum8, const int32_t* wsum4, long T, long N, float* y32, uint16_t* ybf) {
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < T; ++t) {
+        for (long n = 0; n < N; ++n) {
+            double y = (double)acc8[t * N + n] * (double)s_x8[t] * (double)s_w8[n] +
+                       (double)z_x8[t] * (double)s_w8[n] * (double)wsum8[n] +
+                       (double)acc4[t * N + n] * (double)s_x4[t] * (double)s_w4[n] +
+                       (double)z_x4[t] * (double)s_w4[n] * (double)wsum4[n];
             float yf = (float)y;
             y32[t * N + n] = yf;
             if (ybf) ybf[t * N + n] = f32_to_bf16(yf);
