@@ -148,6 +148,41 @@ int resq_linear(const resq_layer_desc_t* desc, int T, const void* X, const void*
                 void* stream);
 
 /*
+ * ---- Asymmetric per-token activations (Eq. 1, second form; the activation setting of the paper's
+ * experiments, Section 5.1), symmetric per-channel weights as before. ----
+ * Per token and segment: z = min, s = (max - min) / (2^N - 1), code = round-half-even((x - z) / s) in
+ * [0, 2^N - 1] (fp32 subtraction and divisions in this order; a constant segment gives s = 0, codes 0),
+ * dequantized value code * s + z.  Expanding Eq. 4 with these activations gives, per segment, the integer
+ * product of the unsigned codes with the weight codes plus a rank-one term:
+ *     Y[t][n] = s_x8[t]*s_w8[n]*sum_j u8[t][j]*w8[n][j] + z_x8[t]*s_w8[n]*wsum8[n]
+ *             + s_x4[t]*s_w4[n]*sum_j u4[t][j]*w4[n][j] + z_x4[t]*s_w4[n]*wsum4[n],
+ * wsum8[n] = sum_j w8[n][j] and wsum4[n] = sum_j w4[n][j] being the integer row sums of the weight codes
+ * (computed once per layer by resq_weight_row_sums).  The products run as u8 x s8 on the same tensor-core
+ * tile kernel for every T >= 1.  Unsigned INT4 codes pack like the signed ones (code 2i in the low nibble).
+ * The epilogue is fp32: (float)acc*(s_x*s_w) per segment plus z_x*((float)wsum*s_w) per segment.
+ * K * 4 bytes (a staged fp32 row) must not exceed 200 KB, else RESQ_ERR_SHAPE.
+ */
+int resq_weight_row_sums(const resq_layer_desc_t* desc, const resq_weights_t* W, int32_t* wsum8, int32_t* wsum4,
+                         void* stream);
+/* As resq_project_quantize; u8 uint8 [T][r], u4 packed uint8 [T][(K-r)/2] and/or u4_u8 uint8 [T][K-r] (one code
+ * per byte), scales s_x8/s_x4 and zero-points z_x8/z_x4 fp32 [T]. */
+int resq_project_quantize_asym(const void* X, const void* P, int T, int K, int r, uint8_t* u8, uint8_t* u4,
+                               float* s_x8, float* s_x4, float* z_x8, float* z_x4, uint8_t* u4_u8, void* workspace,
+                               size_t workspace_bytes, void* stream);
+/* As resq_mixed_gemm, with unsigned activation codes, zero-points and the weight row sums. */
+int resq_mixed_gemm_asym(const resq_layer_desc_t* desc, int T, const uint8_t* u8, const uint8_t* u4,
+                         const uint8_t* u4_u8, const float* s_x8, const float* s_x4, const float* z_x8,
+                         const float* z_x4, const resq_weights_t* W, const int32_t* wsum8, const int32_t* wsum4,
+                         void* Y, int y_dtype, int32_t* dbg_acc8, int32_t* dbg_acc4, void* workspace,
+                         size_t workspace_bytes, void* stream);
+/* As resq_linear. */
+int resq_linear_asym(const resq_layer_desc_t* desc, int T, const void* X, const void* P, const resq_weights_t* W,
+                     const int32_t* wsum8, const int32_t* wsum4, void* Y, int y_dtype, void* workspace,
+                     size_t workspace_bytes, void* stream);
+/* Scratch bytes the three calls above need (0 on an invalid descriptor). */
+size_t resq_workspace_bytes_asym(const resq_layer_desc_t* desc, int T, int has_P, int has_w4_i8);
+
+/*
  * (No counterpart in the paper: a deployment aid.)  Same result as resq_project_quantize with
  * P != NULL, for callers that cannot allocate device memory at all -- a server whose start-up code
  * gave the whole GPU to its own pool, a plug-in living inside another program's memory plan, a

@@ -24,6 +24,8 @@ EXPORTS = [
     "resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_bytes", "resq_workspace_bytes",
     "resq_pack_weights", "resq_project", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
     "resq_unpack_int4", "resq_set_option",
+    "resq_weight_row_sums", "resq_project_quantize_asym", "resq_mixed_gemm_asym", "resq_linear_asym",
+    "resq_workspace_bytes_asym",
     "resq_device_status", "resq_status_string", "resq_last_cuda_error",
 ]
 
@@ -65,6 +67,13 @@ lib.resq_mixed_gemm.argtypes = [_dp, _i, _vp, _vp, _vp, _vp, _vp, ctypes.POINTER
                                 _vp, _sz, _vp]
 lib.resq_linear.argtypes = [_dp, _i, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _i, _vp, _sz, _vp]
 lib.resq_unpack_int4.argtypes = [_vp, _vp, _sz, _sz, _vp]
+lib.resq_weight_row_sums.argtypes = [_dp, ctypes.POINTER(WeightsStruct), _vp, _vp, _vp]
+lib.resq_project_quantize_asym.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.resq_mixed_gemm_asym.argtypes = [_dp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _vp,
+                                     _vp, _i, _vp, _vp, _vp, _sz, _vp]
+lib.resq_linear_asym.argtypes = [_dp, _i, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _vp, _vp, _i, _vp, _sz, _vp]
+lib.resq_workspace_bytes_asym.restype = _sz
+lib.resq_workspace_bytes_asym.argtypes = [_dp, _i, _i, _i]
 lib.resq_set_option.argtypes = [_i, _i]
 lib.resq_device_status.argtypes = [_vp]
 lib.resq_status_string.restype = ctypes.c_char_p
@@ -198,4 +207,55 @@ def resq_device_status() -> int:
 def alloc_workspace(desc: LayerDesc, T: int, has_P: bool, has_w4_i8: bool, device="cuda"):
     import torch
     n = resq_workspace_bytes(desc, T, has_P, has_w4_i8)
+    return torch.empty(max(n, 256), dtype=torch.uint8, device=device)
+
+
+# --------------------------------------------------------------------------- asymmetric activations
+def _nbytes(t) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def resq_weight_row_sums(W: Weights):
+    """int32 row sums of the INT8 and INT4 weight codes of a packed layer: (wsum8 [n_out], wsum4 [n_out])."""
+    import torch
+    dev = W.w8.device
+    s8 = torch.empty(W.desc.n_out, dtype=torch.int32, device=dev)
+    s4 = torch.empty(W.desc.n_out, dtype=torch.int32, device=dev)
+    ws = W.struct()
+    _check(lib.resq_weight_row_sums(ctypes.byref(W.desc), ctypes.byref(ws), _ptr(s8), _ptr(s4), _stream()),
+           "resq_weight_row_sums")
+    return s8, s4
+
+
+def resq_project_quantize_asym(X, P, r: int, u8, u4, s_x8, s_x4, z_x8, z_x4, u4_u8=None, workspace=None):
+    T, K = X.shape
+    _check(lib.resq_project_quantize_asym(_ptr(X), _ptr(P), T, K, r, _ptr(u8), _ptr(u4), _ptr(s_x8), _ptr(s_x4),
+                                          _ptr(z_x8), _ptr(z_x4), _ptr(u4_u8), _ptr(workspace), _nbytes(workspace),
+                                          _stream()), "resq_project_quantize_asym")
+
+
+def resq_mixed_gemm_asym(W: Weights, wsum8, wsum4, u8, u4, s_x8, s_x4, z_x8, z_x4, Y, workspace, dbg_acc8=None,
+                         dbg_acc4=None, u4_u8=None):
+    import torch
+    T = u8.shape[0]
+    y_dtype = Y_BF16 if Y.dtype == torch.bfloat16 else Y_FP32
+    ws = W.struct()
+    _check(lib.resq_mixed_gemm_asym(ctypes.byref(W.desc), T, _ptr(u8), _ptr(u4), _ptr(u4_u8), _ptr(s_x8), _ptr(s_x4),
+                                    _ptr(z_x8), _ptr(z_x4), ctypes.byref(ws), _ptr(wsum8), _ptr(wsum4), _ptr(Y), y_dtype,
+                                    _ptr(dbg_acc8), _ptr(dbg_acc4), _ptr(workspace), _nbytes(workspace), _stream()),
+           "resq_mixed_gemm_asym")
+
+
+def resq_linear_asym(W: Weights, wsum8, wsum4, X, P, Y, workspace):
+    import torch
+    T = X.shape[0]
+    y_dtype = Y_BF16 if Y.dtype == torch.bfloat16 else Y_FP32
+    ws = W.struct()
+    _check(lib.resq_linear_asym(ctypes.byref(W.desc), T, _ptr(X), _ptr(P), ctypes.byref(ws), _ptr(wsum8), _ptr(wsum4),
+                                _ptr(Y), y_dtype, _ptr(workspace), _nbytes(workspace), _stream()), "resq_linear_asym")
+
+
+def alloc_workspace_asym(desc: LayerDesc, T: int, has_P: bool, has_w4_i8: bool, device="cuda"):
+    import torch
+    n = int(lib.resq_workspace_bytes_asym(ctypes.byref(desc), T, int(has_P), int(has_w4_i8)))
     return torch.empty(max(n, 256), dtype=torch.uint8, device=device)

@@ -60,7 +60,7 @@ int check_arch() {
 
 // Carving of the caller's workspace.  Every entry point uses the same map (and its own subset).
 struct Workspace {
-    size_t x8, x4, sx8, sx4, x4e, w4e, panel, decode, total;
+    size_t x8, x4, sx8, sx4, zx8, zx4, x4e, w4e, panel, decode, total;
 };
 Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     Workspace w{};
@@ -70,6 +70,8 @@ Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     w.x4 = o;  o += align_up(Tz * K4 / 2);
     w.sx8 = o; o += align_up(Tz * 4);
     w.sx4 = o; o += align_up(Tz * 4);
+    w.zx8 = o; o += align_up(Tz * 4);  // zero-points (asymmetric activations only)
+    w.zx4 = o; o += align_up(Tz * 4);
     const bool tiles = T > kDecodeMaxT;
     w.x4e = o;    o += tiles ? align_up(Tz * K4) : 0;
     w.w4e = o;    o += (tiles && !has_w4_i8) ? align_up(N * K4) : 0;
@@ -247,6 +249,134 @@ int resq_linear(const resq_layer_desc_t* d, int T, const void* X, const void* P,
         return e;
     return mixed_gemm_impl(d, T, x8, x4, x4e, s_x8, s_x4, W, Y, y_dtype, nullptr, nullptr, ws, map,
                            static_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------- asymmetric activations (Section 5.1)
+int resq_weight_row_sums(const resq_layer_desc_t* d, const resq_weights_t* W, int32_t* wsum8, int32_t* wsum4,
+                         void* stream) {
+    if (int e = check_desc(d)) return e;
+    if (int e = check_weights(W)) return e;
+    if (!wsum8 || !wsum4) return RESQ_ERR_NULL;
+    if (!aligned16(wsum8) || !aligned16(wsum4)) return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_weight_row_sums(W->w8, W->w4, d->n_out, d->K, d->r, wsum8, wsum4,
+                                              static_cast<cudaStream_t>(stream)));
+}
+
+int resq_project_quantize_asym(const void* X, const void* P, int T, int K, int r, uint8_t* u8, uint8_t* u4,
+                               float* s_x8, float* s_x4, float* z_x8, float* z_x4, uint8_t* u4_u8, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+    if (T < 1) return RESQ_ERR_SHAPE;
+    if (int e = check_shape(K, 8, r)) return e;
+    if (!X || !u8 || !s_x8 || !s_x4 || !z_x8 || !z_x4 || (!u4 && !u4_u8)) return RESQ_ERR_NULL;
+    if (!aligned16(X) || !aligned16(P) || !aligned16(u8) || !aligned16(u4) || !aligned16(s_x8) || !aligned16(s_x4) ||
+        !aligned16(z_x8) || !aligned16(z_x4) || !aligned16(u4_u8) || !aligned16(workspace))
+        return RESQ_ERR_ALIGN;
+    if (static_cast<size_t>(K) * 4 > 200u * 1024u) return RESQ_ERR_SHAPE;  // row staging limit of this quantizer
+    if (int e = check_arch()) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!P)
+        return cuda_status(launch_split_quantize_asym(X, false, T, K, r, u8, u4, s_x8, s_x4, z_x8, z_x4, u4_u8,
+                                                      static_cast<size_t>(K) * 2, st));
+    const int rows_max = T < kPanelRows ? T : kPanelRows;
+    const size_t need = align_up(static_cast<size_t>(rows_max) * K * 4);
+    if (!workspace || workspace_bytes < need) return RESQ_ERR_WORKSPACE;
+    float* panel = static_cast<float*>(workspace);
+    const size_t K4 = static_cast<size_t>(K - r);
+    for (int t0 = 0; t0 < T; t0 += kPanelRows) {
+        const int rows = T - t0 < kPanelRows ? T - t0 : kPanelRows;
+        const char* Xp = static_cast<const char*>(X) + static_cast<size_t>(t0) * K * 2;
+        if (cudaError_t e = launch_project_gemm(Xp, P, rows, K, panel, st); e != cudaSuccess) return cuda_status(e);
+        if (cudaError_t e = launch_split_quantize_asym(panel, true, rows, K, r, u8 + static_cast<size_t>(t0) * r,
+                                                       u4 ? u4 + static_cast<size_t>(t0) * K4 / 2 : nullptr, s_x8 + t0,
+                                                       s_x4 + t0, z_x8 + t0, z_x4 + t0,
+                                                       u4_u8 ? u4_u8 + static_cast<size_t>(t0) * K4 : nullptr,
+                                                       static_cast<size_t>(K) * 4, st);
+            e != cudaSuccess)
+            return cuda_status(e);
+    }
+    return RESQ_OK;
+}
+
+static int mixed_gemm_asym_impl(const resq_layer_desc_t* d, int T, const uint8_t* u8, const uint8_t* u4,
+                                const uint8_t* u4e_ready, const float* s_x8, const float* s_x4, const float* z_x8,
+                                const float* z_x4, const resq_weights_t* W, const int32_t* wsum8, const int32_t* wsum4,
+                                void* Y, int y_dtype, int32_t* dbg8, int32_t* dbg4, char* ws, const Workspace& map,
+                                cudaStream_t st) {
+    const size_t K4 = static_cast<size_t>(d->K - d->r);
+    const int8_t* x4e = reinterpret_cast<const int8_t*>(u4e_ready);
+    if (!x4e) {
+        int8_t* buf = reinterpret_cast<int8_t*>(ws + map.x4e);
+        if (cudaError_t e = launch_unpack_int4(u4, buf, T, K4, st, true); e != cudaSuccess) return cuda_status(e);
+        x4e = buf;
+    }
+    const int8_t* w4e = W->w4_i8;
+    if (!w4e) {
+        int8_t* buf = reinterpret_cast<int8_t*>(ws + map.w4e);
+        if (cudaError_t e = launch_unpack_int4(W->w4, buf, d->n_out, K4, st); e != cudaSuccess) return cuda_status(e);
+        w4e = buf;
+    }
+    return cuda_status(launch_mixed_gemm_tiles(T, d->n_out, d->K, d->r, reinterpret_cast<const int8_t*>(u8), x4e, s_x8,
+                                               s_x4, W->w8, w4e, W->s_w8, W->s_w4,
+                                               d->w_scale_dtype == RESQ_SCALE_FP16, Y, y_dtype, dbg8, dbg4, st, z_x8,
+                                               z_x4, wsum8, wsum4));
+}
+
+// The tile kernel serves every T here, so the workspace is carved as for T > 16.
+static Workspace carve_asym(const resq_layer_desc_t* d, int T, bool has_P, bool has_w4_i8) {
+    return carve(d->K, d->n_out, d->r, T > kDecodeMaxT ? T : kDecodeMaxT + 1, has_P, has_w4_i8);
+}
+
+int resq_mixed_gemm_asym(const resq_layer_desc_t* d, int T, const uint8_t* u8, const uint8_t* u4, const uint8_t* u4_u8,
+                         const float* s_x8, const float* s_x4, const float* z_x8, const float* z_x4,
+                         const resq_weights_t* W, const int32_t* wsum8, const int32_t* wsum4, void* Y, int y_dtype,
+                         int32_t* dbg_acc8, int32_t* dbg_acc4, void* workspace, size_t workspace_bytes, void* stream) {
+    if (int e = check_desc(d)) return e;
+    if (T < 1 || (y_dtype != RESQ_Y_BF16 && y_dtype != RESQ_Y_FP32)) return RESQ_ERR_SHAPE;
+    if (!u8 || !s_x8 || !s_x4 || !z_x8 || !z_x4 || !wsum8 || !wsum4 || !Y || (!u4 && !u4_u8)) return RESQ_ERR_NULL;
+    if ((dbg_acc8 == nullptr) != (dbg_acc4 == nullptr)) return RESQ_ERR_NULL;
+    if (int e = check_weights(W)) return e;
+    if (!aligned16(u8) || !aligned16(u4) || !aligned16(u4_u8) || !aligned16(s_x8) || !aligned16(s_x4) ||
+        !aligned16(z_x8) || !aligned16(z_x4) || !aligned16(wsum8) || !aligned16(wsum4) || !aligned16(Y) ||
+        !aligned16(dbg_acc8) || !aligned16(dbg_acc4) || !aligned16(workspace))
+        return RESQ_ERR_ALIGN;
+    const Workspace map = carve_asym(d, T, false, W->w4_i8 != nullptr);
+    if (!workspace || workspace_bytes < map.total) return RESQ_ERR_WORKSPACE;
+    if (int e = check_arch()) return e;
+    return mixed_gemm_asym_impl(d, T, u8, u4, u4_u8, s_x8, s_x4, z_x8, z_x4, W, wsum8, wsum4, Y, y_dtype, dbg_acc8,
+                                dbg_acc4, static_cast<char*>(workspace), map, static_cast<cudaStream_t>(stream));
+}
+
+int resq_linear_asym(const resq_layer_desc_t* d, int T, const void* X, const void* P, const resq_weights_t* W,
+                     const int32_t* wsum8, const int32_t* wsum4, void* Y, int y_dtype, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    if (int e = check_desc(d)) return e;
+    if (T < 1 || (y_dtype != RESQ_Y_BF16 && y_dtype != RESQ_Y_FP32)) return RESQ_ERR_SHAPE;
+    if (!X || !Y || !wsum8 || !wsum4) return RESQ_ERR_NULL;
+    if (int e = check_weights(W)) return e;
+    if (!aligned16(X) || !aligned16(P) || !aligned16(Y) || !aligned16(wsum8) || !aligned16(wsum4) ||
+        !aligned16(workspace))
+        return RESQ_ERR_ALIGN;
+    const Workspace map = carve_asym(d, T, P != nullptr, W->w4_i8 != nullptr);
+    if (!workspace || workspace_bytes < map.total) return RESQ_ERR_WORKSPACE;
+    if (int e = check_arch()) return e;
+    char* ws = static_cast<char*>(workspace);
+    uint8_t* u8 = reinterpret_cast<uint8_t*>(ws + map.x8);
+    uint8_t* u4e = reinterpret_cast<uint8_t*>(ws + map.x4e);
+    float* s_x8 = reinterpret_cast<float*>(ws + map.sx8);
+    float* s_x4 = reinterpret_cast<float*>(ws + map.sx4);
+    float* z_x8 = reinterpret_cast<float*>(ws + map.zx8);
+    float* z_x4 = reinterpret_cast<float*>(ws + map.zx4);
+    if (int e = resq_project_quantize_asym(X, P, T, d->K, d->r, u8, nullptr, s_x8, s_x4, z_x8, z_x4, u4e, ws + map.panel,
+                                           workspace_bytes - map.panel, stream))
+        return e;
+    return mixed_gemm_asym_impl(d, T, u8, nullptr, u4e, s_x8, s_x4, z_x8, z_x4, W, wsum8, wsum4, Y, y_dtype, nullptr,
+                                nullptr, ws, map, static_cast<cudaStream_t>(stream));
+}
+
+size_t resq_workspace_bytes_asym(const resq_layer_desc_t* d, int T, int has_P, int has_w4_i8) {
+    if (check_desc(d) || T < 1) return 0;
+    return carve_asym(d, T, has_P != 0, has_w4_i8 != 0).total;
 }
 
 int resq_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, void* stream) {

@@ -21,13 +21,28 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
                                   uint8_t* q4, void* s8, void* s4, bool scale_fp16, int8_t* q4_i8,
                                   size_t in_row_stride, cudaStream_t st);
 
-cudaError_t launch_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, cudaStream_t st);
+// codes_unsigned: the nibbles are 0..15 (asymmetric activation codes) instead of two's complement.
+cudaError_t launch_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, cudaStream_t st,
+                               bool codes_unsigned = false);
 
 // Many-token tile kernel on tcgen05 kind::i8.  x4e / w4e are the INT4 codes one per byte.
 cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8, const int8_t* x4e,
                                     const float* s_x8, const float* s_x4, const int8_t* w8, const int8_t* w4e,
                                     const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
-                                    int32_t* dbg8, int32_t* dbg4, cudaStream_t st);
+                                    int32_t* dbg8, int32_t* dbg4, cudaStream_t st, const float* z_x8 = nullptr,
+                                    const float* z_x4 = nullptr, const int32_t* wsum8 = nullptr,
+                                    const int32_t* wsum4 = nullptr);
+// z_x8 != NULL selects asymmetric activations: x8 / x4e then hold UNSIGNED codes (0..255, 0..15) and the
+// epilogue adds z_x8[t] * s_w8[n] * wsum8[n] + z_x4[t] * s_w4[n] * wsum4[n].
+
+// Asymmetric split quantization (Eq. 1, second form) of the rows of a [rows][K] matrix.  Returns
+// cudaErrorNotSupported for rows wider than 200 KB.
+cudaError_t launch_split_quantize_asym(const void* in, bool in_is_f32, size_t rows, int K, int r, uint8_t* u8,
+                                       uint8_t* u4, float* s8, float* s4, float* z8, float* z4, uint8_t* u4_u8,
+                                       size_t in_row_stride_bytes, cudaStream_t st);
+// wsum8[n] = sum_j w8[n][j], wsum4[n] = sum_j w4[n][j] (packed codes).
+cudaError_t launch_weight_row_sums(const int8_t* w8, const uint8_t* w4, int N, int K, int r, int32_t* wsum8,
+                                   int32_t* wsum4, cudaStream_t st);
 
 // Few-token (T <= 16) weight-streaming split-K kernel.  scratch: see decode_scratch_bytes().
 size_t decode_scratch_bytes(int T, int N);

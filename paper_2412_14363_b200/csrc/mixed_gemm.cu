@@ -50,6 +50,11 @@ struct Params {
     const void* s_w8;
     const void* s_w4;
     int w_fp16;
+    // asymmetric activations only: per-token zero-points and per-channel row sums of the weight codes
+    const float* z_x8;
+    const float* z_x4;
+    const int32_t* wsum8;
+    const int32_t* wsum4;
     void* Y;
     int y_dtype;
     int32_t* dbg8;
@@ -68,6 +73,8 @@ struct __align__(8) Shared {
     int epi_stop;
     float sw8[BN];
     float sw4[BN];
+    float zc8[BN];  // asymmetric activations: (float)wsum8[n] * sw8[n], the column factor of the zero-point term
+    float zc4[BN];
 };
 
 constexpr size_t kSmemBytes = 1024 + STAGES * (A_BYTES + B_BYTES) + sizeof(Shared);
@@ -78,6 +85,9 @@ __device__ __forceinline__ float load_scale(const void* p, int i, int fp16) {
 
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
+// ASYM: the activation codes are unsigned (u8 x s8 products) and every output gets the rank-one
+// zero-point terms z_x8[t] * s_w8[n] * wsum8[n] + z_x4[t] * s_w4[n] * wsum4[n] (Eq. 1, second form).
+template <bool ASYM>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constant__ CUtensorMap tmA4,
                   const __grid_constant__ CUtensorMap tmB8, const __grid_constant__ CUtensorMap tmB4,
@@ -154,7 +164,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (even CTA only)
         if (lane == 0 && rank == 0) {
-            const uint32_t idesc = make_idesc_i8(2 * BM, p.bn);
+            const uint32_t idesc = ASYM ? make_idesc_u8s8(2 * BM, p.bn) : make_idesc_i8(2 * BM, p.bn);
             int stage = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
@@ -201,8 +211,14 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             const int n_end = min(p.N, n0 + p.bn);  // first column past this tile
             {
                 const int n = n0 + et;
-                sh->sw8[et] = n < n_end ? load_scale(p.s_w8, n, p.w_fp16) : 0.f;
-                sh->sw4[et] = n < n_end ? load_scale(p.s_w4, n, p.w_fp16) : 0.f;
+                const float w8s = n < n_end ? load_scale(p.s_w8, n, p.w_fp16) : 0.f;
+                const float w4s = n < n_end ? load_scale(p.s_w4, n, p.w_fp16) : 0.f;
+                sh->sw8[et] = w8s;
+                sh->sw4[et] = w4s;
+                if (ASYM) {
+                    sh->zc8[et] = n < n_end ? static_cast<float>(p.wsum8[n]) * w8s : 0.f;
+                    sh->zc4[et] = n < n_end ? static_cast<float>(p.wsum4[n]) * w4s : 0.f;
+                }
             }
             epi_barrier();
             if (sh->epi_stop) break;
@@ -210,6 +226,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             const bool row_ok = row < p.T;
             const float sx8 = row_ok ? __ldg(p.s_x8 + row) : 0.f;
             const float sx4 = row_ok ? __ldg(p.s_x4 + row) : 0.f;
+            const float zx8 = ASYM && row_ok ? __ldg(p.z_x8 + row) : 0.f;
+            const float zx4 = ASYM && row_ok ? __ldg(p.z_x4 + row) : 0.f;
             if (!mbar_wait(&sh->acc_full, acc_phase, abort_flag)) continue;  // flag is set; leave at the next sample
             acc_phase ^= 1;
             tc_fence_after();
@@ -248,6 +266,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                         const float t8 = static_cast<float>(static_cast<int>(a8[j])) * (sx8 * sh->sw8[cb + j]);
                         const float t4 = static_cast<float>(static_cast<int>(a4c[j])) * (sx4 * sh->sw4[cb + j]);
                         y[j] = t8 + t4;
+                        if (ASYM) y[j] += zx8 * sh->zc8[cb + j] + zx4 * sh->zc4[cb + j];
                     }
                     if (p.y_dtype == RESQ_Y_BF16) {
                         __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.Y) + off;
@@ -316,13 +335,18 @@ int pick_tile_width(int /*m_tiles*/, int /*N*/, int /*sms*/) { return 256; }
 cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8, const int8_t* x4e,
                                     const float* s_x8, const float* s_x4, const int8_t* w8, const int8_t* w4e,
                                     const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
-                                    int32_t* dbg8, int32_t* dbg4, cudaStream_t st) {
+                                    int32_t* dbg8, int32_t* dbg4, cudaStream_t st, const float* z_x8,
+                                    const float* z_x4, const int32_t* wsum8, const int32_t* wsum4) {
+    const bool asym = z_x8 != nullptr;  // then x8 / x4e hold unsigned codes
     static bool attr_set[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 64 && !attr_set[dev]) {
-        e = cudaFuncSetAttribute(mixed_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(mixed_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kSmemBytes));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(mixed_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kSmemBytes));
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
@@ -343,11 +367,13 @@ cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8
     p.kb4 = (K4 + BK - 1) / BK;
     p.s_x8 = s_x8; p.s_x4 = s_x4; p.s_w8 = s_w8; p.s_w4 = s_w4;
     p.w_fp16 = w_scale_fp16 ? 1 : 0;
+    p.z_x8 = z_x8; p.z_x4 = z_x4; p.wsum8 = wsum8; p.wsum4 = wsum4;
     p.Y = Y; p.y_dtype = y_dtype; p.dbg8 = dbg8; p.dbg4 = dbg8 ? dbg4 : nullptr;
     p.status = device_status_ptr();
     const int tiles = p.m_tiles * p.n_tiles;
     const int pairs = tiles < sms / 2 ? tiles : sms / 2;
-    mixed_gemm_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
+    if (asym) mixed_gemm_kernel<true><<<2 * pairs, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
+    else mixed_gemm_kernel<false><<<2 * pairs, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
     return cudaGetLastError();
 }
 

@@ -329,6 +329,7 @@ split_quantize_fast_kernel(const void* __restrict__ in, size_t in_row_bytes, siz
     }
 }
 
+template <bool UNSIGNED>
 __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* __restrict__ out, size_t nwords) {
     // one 32-bit packed word (8 codes) per thread -> 8 bytes
     for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < nwords;
@@ -338,7 +339,7 @@ __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* _
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             int v = static_cast<int>((w >> (4 * k)) & 0xFu);
-            v = (v ^ 8) - 8;  // sign-extend the nibble
+            if (!UNSIGNED) v = (v ^ 8) - 8;  // sign-extend the nibble
             o[k >> 2] |= (static_cast<uint32_t>(v) & 0xFFu) << (8 * (k & 3));
         }
         reinterpret_cast<uint2*>(out)[i] = make_uint2(o[0], o[1]);
@@ -384,12 +385,14 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
     return cudaGetLastError();
 }
 
-cudaError_t launch_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, cudaStream_t st) {
+cudaError_t launch_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, cudaStream_t st,
+                               bool codes_unsigned) {
     const size_t nwords = rows * cols / 8;
     if (nwords == 0) return cudaSuccess;
     size_t blocks = (nwords + 255) / 256;
     if (blocks > 148 * 32) blocks = 148 * 32;
-    unpack_int4_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(packed, out, nwords);
+    if (codes_unsigned) unpack_int4_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, st>>>(packed, out, nwords);
+    else unpack_int4_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, st>>>(packed, out, nwords);
     return cudaGetLastError();
 }
 

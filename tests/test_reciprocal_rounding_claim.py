@@ -50,3 +50,38 @@ def test_product_rounding_agrees_outside_guard_band():
                 else:
                     fallbacks += 1
     assert checked > 10000 and fallbacks > 1000  # both branches were exercised
+
+
+def test_asymmetric_product_rounding_agrees_outside_guard_band():
+    """Same claim for the asymmetric quantizer: d = fl(x - z), code = rint(fl(d / s)) against
+    rint(d * RN(1 / s)); quotients reach 255, so the guard band is 2^-14."""
+    guard = Fraction(1, 2) - Fraction(1, 2 ** 14)
+    rng = np.random.default_rng(4)
+    checked = fallbacks = 0
+    for bits, qmax in ((8, 255), (4, 15)):
+        for _ in range(40):
+            lo = np.float32(rng.uniform(-10, 10))
+            rng_w = np.float32(np.exp(rng.uniform(-12, 12)))
+            hi = np.float32(lo + rng_w)
+            s = np.float32(np.float32(hi - lo) / np.float32(qmax))
+            inv = np.float32(np.float32(1.0) / s)
+            k = rng.integers(0, qmax, 200).astype(np.float32) + np.float32(0.5)
+            near = (np.float32(lo) + (k * s).astype(np.float32)).astype(np.float32)
+            near = (near.view(np.int32) + rng.integers(-4, 5, 200).astype(np.int32)).view(np.float32)
+            x = np.concatenate([near, rng.uniform(lo, hi, 200).astype(np.float32)])
+            x = x[(x >= lo) & (x <= hi)]
+            row = np.concatenate([[lo, hi], x]).astype(np.float32)
+            pad = np.tile(row, 2)[None, :]                      # both segments hold the same data
+            out = oracle.split_quantize_asym(pad, row.size)
+            codes = out[0 if bits == 8 else 1][0, 2:]
+            assert out[2 if bits == 8 else 3][0] == s and out[4 if bits == 8 else 5][0] == lo
+            for xv, code in zip(x, codes):
+                d = np.float32(xv - lo)
+                p = Fraction(float(d)) * Fraction(float(inv))
+                n = _rint_half_even(p)
+                if abs(p - n) < guard:
+                    assert n == int(code), (float(xv), float(s), n, int(code))
+                    checked += 1
+                else:
+                    fallbacks += 1
+    assert checked > 10000 and fallbacks > 500
