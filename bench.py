@@ -230,6 +230,62 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
     return out
 
 
+# --------------------------------------------------------------------------------------- asymmetric leg
+def asym_leg(resq, torch, dev, layers, T, steps):
+    """One pass of the block with asymmetric per-token activation codes (unsigned codes + zero-points,
+    u8 x s8 products, rank-one zero-point terms in the epilogue); the weights are those of the main leg."""
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    bufs = []
+    for L in layers:
+        K4 = L.K - L.r
+        z = lambda *shape, dt=torch.float32: torch.empty(shape, dtype=dt, device=dev)
+        bufs.append(dict(ws8=None, u8=z(T, L.r, dt=torch.uint8), u4e=z(T, K4, dt=torch.uint8), sx8=z(T), sx4=z(T),
+                         zx8=z(T), zx4=z(T), wsp=resq.alloc_workspace_asym(L.desc, T, L.online, True, device=dev)))
+        bufs[-1]["ws8"], bufs[-1]["ws4"] = resq.resq_weight_row_sums(L.W)
+
+    def step(events=None):
+        for L, b in zip(layers, bufs):
+            e0 = ev() if events is not None else None
+            resq.resq_project_quantize_asym(L.X, L.P, L.r, b["u8"], None, b["sx8"], b["sx4"], b["zx8"], b["zx4"], b["u4e"],
+                                            b["wsp"] if L.online else None)
+            e1 = ev() if events is not None else None
+            resq.resq_mixed_gemm_asym(L.W, b["ws8"], b["ws4"], b["u8"], None, b["sx8"], b["sx4"], b["zx8"], b["zx4"], L.Y,
+                                      b["wsp"], u4_u8=b["u4e"])
+            if events is not None:
+                events.append((L, e0, e1, ev()))
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    events = []
+    t0 = ev()
+    for _ in range(steps):
+        step(events)
+    t1 = ev()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / steps
+    per_layer, ops, g_ms = {}, 0.0, 0.0
+    for L in layers:
+        q = statistics.mean(e0.elapsed_time(e1) for l, e0, e1, _ in events if l is L)
+        g = statistics.mean(e1.elapsed_time(e2) for l, _, e1, e2 in events if l is L)
+        per_layer[L.name] = {"quantize_ms": round(q, 4), "mixed_gemm_ms": round(g, 4),
+                             "mixed_gemm_tops": round(2.0 * T * L.K * L.N / (g * 1e-3) / 1e12, 1)}
+        ops += 2.0 * T * L.K * L.N
+        g_ms += g
+    st = resq.resq_device_status()
+    if st != resq.OK:
+        raise SystemExit(f"device status {st}: {resq.status_string(st)}")
+    return {"workload": WORKLOAD + "-asymmetric-activations", "steps": steps, "ms_per_step": round(ms, 4),
+            "tokens_per_s": round(T / (ms * 1e-3), 1), "mixed_gemm_tops": round(ops / (g_ms * 1e-3) / 1e12, 1),
+            "per_layer": per_layer}
+
+
 # --------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import numpy as np
@@ -445,6 +501,11 @@ def run_ours(args):
     if st != resq.OK:
         raise SystemExit(f"device status {st}: {resq.status_string(st)}")
 
+    # ---- the same prefill block with asymmetric per-token activations (the paper's experimental setting)
+    asym = None
+    if not args.no_asym and not only:
+        asym = asym_leg(resq, torch, dev, layers, T, max(5, min(args.steps, 10)))
+
     # ---- decode variant of the same block (this rank only; reported by rank 0)
     decode = None
     if not args.no_decode and not only:
@@ -492,7 +553,7 @@ def run_ours(args):
             "mixed_gemm_frac_of_int8_peak": {"vs_measured_bf16_x2": kernels["mixed_gemm"]["frac"],
                                              "vs_nominal_4500": kernels["mixed_gemm"]["frac_of_nominal_4500"]},
             "per_layer": per_layer,
-            "roofline": roofline, "decode": decode, "e2e": e2e, "cpu_baseline": cpu_baseline, "parity_spot_check": parity,
+            "roofline": roofline, "decode": decode, "asymmetric": asym, "e2e": e2e, "cpu_baseline": cpu_baseline, "parity_spot_check": parity,
             "gpu_launches": LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
         }
         print(json.dumps(line))
@@ -540,6 +601,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--no-asym", action="store_true", help="skip the asymmetric-activation leg (profiling runs)")
     ap.add_argument("--no-decode", action="store_true", help="skip the few-token leg (profiling runs)")
     ap.add_argument("--decode-only", action="store_true", help="run only the few-token leg (profiling runs)")
     ap.add_argument("--layers", default="", help="comma-separated subset of qkv,o,gate_up,down (profiling runs)")
