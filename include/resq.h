@@ -157,8 +157,8 @@ int resq_linear(const resq_layer_desc_t* desc, int T, const void* X, const void*
  *     Y[t][n] = s_x8[t]*s_w8[n]*sum_j u8[t][j]*w8[n][j] + z_x8[t]*s_w8[n]*wsum8[n]
  *             + s_x4[t]*s_w4[n]*sum_j u4[t][j]*w4[n][j] + z_x4[t]*s_w4[n]*wsum4[n],
  * wsum8[n] = sum_j w8[n][j] and wsum4[n] = sum_j w4[n][j] being the integer row sums of the weight codes
- * (computed once per layer by resq_weight_row_sums).  The products run as u8 x s8 on the same tensor-core
- * tile kernel for every T >= 1.  Unsigned INT4 codes pack like the signed ones (code 2i in the low nibble).
+ * (computed once per layer by resq_weight_row_sums).  The products run as u8 x s8: on the weight-streaming
+ * kernel for T <= 16 when the packed codes u4 are given, on the tensor-core tile kernel otherwise.  Unsigned INT4 codes pack like the signed ones (code 2i in the low nibble).
  * The epilogue is fp32: (float)acc*(s_x*s_w) per segment plus z_x*((float)wsum*s_w) per segment.
  * K * 4 bytes (a staged fp32 row) must not exceed 200 KB, else RESQ_ERR_SHAPE.
  */

@@ -304,6 +304,14 @@ static int mixed_gemm_asym_impl(const resq_layer_desc_t* d, int T, const uint8_t
                                 void* Y, int y_dtype, int32_t* dbg8, int32_t* dbg4, char* ws, const Workspace& map,
                                 cudaStream_t st) {
     const size_t K4 = static_cast<size_t>(d->K - d->r);
+    if (T <= kDecodeMaxT && u4) {
+        // Few tokens and packed codes at hand: the weight-streaming kernel (falls through if it cannot stage them).
+        const cudaError_t e = launch_mixed_gemm_stream(T, d->n_out, d->K, d->r, reinterpret_cast<const int8_t*>(u8), u4,
+                                                       s_x8, s_x4, W->w8, W->w4, W->s_w8, W->s_w4,
+                                                       d->w_scale_dtype == RESQ_SCALE_FP16, Y, y_dtype, dbg8, dbg4, st,
+                                                       z_x8, z_x4, wsum8, wsum4);
+        if (e != cudaErrorNotSupported) return cuda_status(e);
+    }
     const int8_t* x4e = reinterpret_cast<const int8_t*>(u4e_ready);
     if (!x4e) {
         int8_t* buf = reinterpret_cast<int8_t*>(ws + map.x4e);
@@ -367,10 +375,12 @@ int resq_linear_asym(const resq_layer_desc_t* d, int T, const void* X, const voi
     float* s_x4 = reinterpret_cast<float*>(ws + map.sx4);
     float* z_x8 = reinterpret_cast<float*>(ws + map.zx8);
     float* z_x4 = reinterpret_cast<float*>(ws + map.zx4);
-    if (int e = resq_project_quantize_asym(X, P, T, d->K, d->r, u8, nullptr, s_x8, s_x4, z_x8, z_x4, u4e, ws + map.panel,
+    // Few tokens: the streaming kernel wants the packed codes as well (the tile kernel, its fallback, the others).
+    uint8_t* u4 = T <= kDecodeMaxT ? reinterpret_cast<uint8_t*>(ws + map.x4) : nullptr;
+    if (int e = resq_project_quantize_asym(X, P, T, d->K, d->r, u8, u4, s_x8, s_x4, z_x8, z_x4, u4e, ws + map.panel,
                                            workspace_bytes - map.panel, stream))
         return e;
-    return mixed_gemm_asym_impl(d, T, u8, nullptr, u4e, s_x8, s_x4, z_x8, z_x4, W, wsum8, wsum4, Y, y_dtype, nullptr,
+    return mixed_gemm_asym_impl(d, T, u8, u4, u4e, s_x8, s_x4, z_x8, z_x4, W, wsum8, wsum4, Y, y_dtype, nullptr,
                                 nullptr, ws, map, static_cast<cudaStream_t>(stream));
 }
 

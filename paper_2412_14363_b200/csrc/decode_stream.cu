@@ -71,6 +71,11 @@ struct Params {
     const void* s_w8;
     const void* s_w4;
     int w_fp16;
+    // asymmetric activations only (unsigned codes): zero-points per token, row sums of the weight codes
+    const float* z_x8;
+    const float* z_x4;
+    const int32_t* wsum8;
+    const int32_t* wsum4;
     void* Y;
     int y_dtype;
     int32_t* dbg8;
@@ -86,12 +91,20 @@ struct __align__(16) Control {
 };
 static_assert(sizeof(Control) <= kControlBytes, "control block");
 
+// AU: the 16-row operand (the tokens) holds unsigned bytes.
+template <bool AU>
 __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    if constexpr (AU)
+        asm volatile(
+            "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile(
+            "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -108,7 +121,11 @@ __device__ __forceinline__ float2 load_scale2(const void* p, int n, int fp16) {
 // kSplit: the INT4 activations are staged already split into their even / odd codes times 16 (twice
 //         the shared memory, a third of the logic operations); otherwise they stay packed and are
 //         split when used.
-template <int TT, int CS, bool kSplit>
+// ASYM:   asymmetric activations: the codes are unsigned (0..255, 0..15; Eq. 1, second form).  The INT4
+//         activations then enter as their even / odd codes themselves (no factor 16), so
+//         acc4 = accO / 16 + accE - 8 * S_even[t], and the epilogue adds the zero-point terms
+//         z_x8[t] * s_w8[n] * wsum8[n] + z_x4[t] * s_w4[n] * wsum4[n].
+template <int TT, int CS, bool kSplit, bool ASYM>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_constant__ CUtensorMap tmW4,
                          const Params p) {
@@ -175,6 +192,8 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
     // Token scales of the two accumulator rows this thread holds.
     const float sx8a = g < p.T ? p.s_x8[g] : 0.f, sx4a = g < p.T ? p.s_x4[g] : 0.f;
     const float sx8b = g + 8 < p.T ? p.s_x8[g + 8] : 0.f, sx4b = g + 8 < p.T ? p.s_x4[g + 8] : 0.f;
+    const float zx8a = ASYM && g < p.T ? p.z_x8[g] : 0.f, zx4a = ASYM && g < p.T ? p.z_x4[g] : 0.f;
+    const float zx8b = ASYM && g + 8 < p.T ? p.z_x8[g + 8] : 0.f, zx4b = ASYM && g + 8 < p.T ? p.z_x4[g + 8] : 0.f;
     // Stage the activation codes: zero padded to the pitch, zero rows for tokens >= T.  The first
     // batch of INT8 and of INT4 vectors is loaded before anything is stored (one round trip to L2 for
     // the usual sizes); the rest of the ring goes out right behind those loads.
@@ -217,7 +236,11 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                 if (i >= n4) continue;
                 const int t = i / v4, o = i - t * v4;
                 uint8_t* dst = act4 + static_cast<size_t>(t) * p.pitch4 + (o << 4);
-                if (kSplit) {
+                if (kSplit && ASYM) {
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(v[b].x & kLo, v[b].y & kLo, v[b].z & kLo, v[b].w & kLo);
+                    *reinterpret_cast<uint4*>(dst + static_cast<size_t>(TP) * p.pitch4) =
+                        make_uint4((v[b].x >> 4) & kLo, (v[b].y >> 4) & kLo, (v[b].z >> 4) & kLo, (v[b].w >> 4) & kLo);
+                } else if (kSplit) {
                     *reinterpret_cast<uint4*>(dst) =
                         make_uint4((v[b].x << 4) & kHi, (v[b].y << 4) & kHi, (v[b].z << 4) & kHi, (v[b].w << 4) & kHi);
                     *reinterpret_cast<uint4*>(dst + static_cast<size_t>(TP) * p.pitch4) =
@@ -255,8 +278,11 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             const uint8_t* row = act4 + static_cast<size_t>(t) * p.pitch4;
             for (int i = lane; i < (p.pitch4 >> 4); i += 32) {
                 uint4 v = *reinterpret_cast<const uint4*>(row + (i << 4));
-                if (!kSplit) v = make_uint4((v.x << 4) & kHi, (v.y << 4) & kHi, (v.z << 4) & kHi, (v.w << 4) & kHi);
-                se = __dp4a(static_cast<int>(v.x), 0x01010101, se);
+                if (!kSplit) {
+                    if (ASYM) v = make_uint4(v.x & kLo, v.y & kLo, v.z & kLo, v.w & kLo);
+                    else v = make_uint4((v.x << 4) & kHi, (v.y << 4) & kHi, (v.z << 4) & kHi, (v.w << 4) & kHi);
+                }
+                se = __dp4a(static_cast<int>(v.x), 0x01010101, se);  // the lanes are < 128 when unsigned
                 se = __dp4a(static_cast<int>(v.y), 0x01010101, se);
                 se = __dp4a(static_cast<int>(v.z), 0x01010101, se);
                 se = __dp4a(static_cast<int>(v.w), 0x01010101, se);
@@ -264,7 +290,7 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
-        if (lane == 0) ctl->s_even[t] = se >> 4;  // the lanes held 16 x the codes
+        if (lane == 0) ctl->s_even[t] = ASYM ? se : se >> 4;  // signed codes: the lanes held 16 x the codes
     }
     __syncthreads();
     const int sev_a = ctl->s_even[g], sev_b = TT == 2 ? ctl->s_even[g + 8] : 0;
@@ -286,11 +312,16 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         const int n0 = ub * kUnitRows + 2 * tig;  // first of this thread's two channels in half 0
         // Channel scales, fetched now and used after the reduction.
         float2 sw8[2], sw4[2];
+        int2 ws8[2] = {}, ws4[2] = {};
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int n = h < halves ? n0 + 8 * h : n0;
             sw8[h] = load_scale2(p.s_w8, n, p.w_fp16);
             sw4[h] = load_scale2(p.s_w4, n, p.w_fp16);
+            if (ASYM) {
+                ws8[h] = *reinterpret_cast<const int2*>(p.wsum8 + n);
+                ws4[h] = *reinterpret_cast<const int2*>(p.wsum4 + n);
+            }
         }
         int acc8[2][4], accO[2][4], accE[2][4];
 #pragma unroll
@@ -311,10 +342,10 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                     if (TT == 2) y = *reinterpret_cast<const uint4*>(xa + 8 * p.pitch8 + 64 * s);
                     const uint4 wa = *reinterpret_cast<const uint4*>(w0 + 64 * s);
                     const uint4 wb = *reinterpret_cast<const uint4*>(w1 + 64 * s);
-                    mma_s8(acc8[0], x.x, y.x, x.y, y.y, wa.x, wa.y);
-                    mma_s8(acc8[1], x.x, y.x, x.y, y.y, wb.x, wb.y);
-                    mma_s8(acc8[0], x.z, y.z, x.w, y.w, wa.z, wa.w);
-                    mma_s8(acc8[1], x.z, y.z, x.w, y.w, wb.z, wb.w);
+                    mma_s8<ASYM>(acc8[0], x.x, y.x, x.y, y.y, wa.x, wa.y);
+                    mma_s8<ASYM>(acc8[1], x.x, y.x, x.y, y.y, wb.x, wb.y);
+                    mma_s8<ASYM>(acc8[0], x.z, y.z, x.w, y.w, wa.z, wa.w);
+                    mma_s8<ASYM>(acc8[1], x.z, y.z, x.w, y.w, wb.z, wb.w);
                 }
             } else {
                 const uint8_t* xa = a4row + (c - p.c8) * kChunkBytes;
@@ -341,8 +372,13 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                         const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            xe[j] = (xs[j] << 4) & kHi; xo[j] = xs[j] & kHi;
-                            ye[j] = (ys[j] << 4) & kHi; yo[j] = ys[j] & kHi;
+                            if (ASYM) {
+                                xe[j] = xs[j] & kLo; xo[j] = (xs[j] >> 4) & kLo;
+                                ye[j] = ys[j] & kLo; yo[j] = (ys[j] >> 4) & kLo;
+                            } else {
+                                xe[j] = (xs[j] << 4) & kHi; xo[j] = xs[j] & kHi;
+                                ye[j] = (ys[j] << 4) & kHi; yo[j] = ys[j] & kHi;
+                            }
                         }
                     }
                     const uint4 wa = *reinterpret_cast<const uint4*>(w0 + 64 * s);
@@ -350,10 +386,10 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                     const uint32_t was[4] = {wa.x, wa.y, wa.z, wa.w}, wbs[4] = {wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
                     for (int j = 0; j < 4; j += 2) {
-                        mma_s8(accO[0], xo[j], yo[j], xo[j + 1], yo[j + 1], was[j] & kHi, was[j + 1] & kHi);
-                        mma_s8(accE[0], xe[j], ye[j], xe[j + 1], ye[j + 1], (was[j] ^ kFlip) & kLo, (was[j + 1] ^ kFlip) & kLo);
-                        mma_s8(accO[1], xo[j], yo[j], xo[j + 1], yo[j + 1], wbs[j] & kHi, wbs[j + 1] & kHi);
-                        mma_s8(accE[1], xe[j], ye[j], xe[j + 1], ye[j + 1], (wbs[j] ^ kFlip) & kLo, (wbs[j + 1] ^ kFlip) & kLo);
+                        mma_s8<ASYM>(accO[0], xo[j], yo[j], xo[j + 1], yo[j + 1], was[j] & kHi, was[j + 1] & kHi);
+                        mma_s8<ASYM>(accE[0], xe[j], ye[j], xe[j + 1], ye[j + 1], (was[j] ^ kFlip) & kLo, (was[j + 1] ^ kFlip) & kLo);
+                        mma_s8<ASYM>(accO[1], xo[j], yo[j], xo[j + 1], yo[j + 1], wbs[j] & kHi, wbs[j + 1] & kHi);
+                        mma_s8<ASYM>(accE[1], xe[j], ye[j], xe[j + 1], ye[j + 1], (wbs[j] ^ kFlip) & kLo, (wbs[j + 1] ^ kFlip) & kLo);
                     }
                 }
             }
@@ -374,7 +410,7 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 part[h][0][i] = acc8[h][i];
-                part[h][1][i] = (accO[h][i] >> 8) + (accE[h][i] >> 4);
+                part[h][1][i] = ASYM ? (accO[h][i] >> 4) + accE[h][i] : (accO[h][i] >> 8) + (accE[h][i] >> 4);
             }
         const int item_begin = item * nchunks, item_end = item_begin + nchunks;
         bool finish = true;
@@ -426,8 +462,13 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                     const int sev = 8 * (tr ? sev_b : sev_a);
                     const int a8x = part[h][0][2 * tr], a8y = part[h][0][2 * tr + 1];
                     const int a4x = part[h][1][2 * tr] - sev, a4y = part[h][1][2 * tr + 1] - sev;
-                    const float yx = static_cast<float>(a8x) * (sx8 * sw8[h].x) + static_cast<float>(a4x) * (sx4 * sw4[h].x);
-                    const float yy = static_cast<float>(a8y) * (sx8 * sw8[h].y) + static_cast<float>(a4y) * (sx4 * sw4[h].y);
+                    float yx = static_cast<float>(a8x) * (sx8 * sw8[h].x) + static_cast<float>(a4x) * (sx4 * sw4[h].x);
+                    float yy = static_cast<float>(a8y) * (sx8 * sw8[h].y) + static_cast<float>(a4y) * (sx4 * sw4[h].y);
+                    if (ASYM) {
+                        const float zx8 = tr ? zx8b : zx8a, zx4 = tr ? zx4b : zx4a;
+                        yx += zx8 * (static_cast<float>(ws8[h].x) * sw8[h].x) + zx4 * (static_cast<float>(ws4[h].x) * sw4[h].x);
+                        yy += zx8 * (static_cast<float>(ws8[h].y) * sw8[h].y) + zx4 * (static_cast<float>(ws4[h].y) * sw4[h].y);
+                    }
                     const size_t o = static_cast<size_t>(t) * p.N + n0 + 8 * h;
                     if (p.y_dtype == RESQ_Y_BF16)
                         *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(p.Y) + o) = __floats2bfloat162_rn(yx, yy);
@@ -477,10 +518,10 @@ bool make_map_rows(CUtensorMap* m, const void* base, uint64_t rows, uint64_t row
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int TT, int CS, bool SPLIT>
+template <int TT, int CS, bool SPLIT, bool ASYM>
 cudaError_t launch_variant(const CUtensorMap& t8, const CUtensorMap& t4, const Params& p, int grid, size_t smem,
                            cudaStream_t st) {
-    auto kern = mixed_gemm_stream_kernel<TT, CS, SPLIT>;
+    auto kern = mixed_gemm_stream_kernel<TT, CS, SPLIT, ASYM>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -512,7 +553,9 @@ void set_decode_early_weights(int on) { g_early_weights = on ? 1 : 0; }
 cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x8, const uint8_t* x4,
                                      const float* s_x8, const float* s_x4, const int8_t* w8, const uint8_t* w4,
                                      const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
-                                     int32_t* dbg8, int32_t* dbg4, cudaStream_t st) {
+                                     int32_t* dbg8, int32_t* dbg4, cudaStream_t st, const float* z_x8,
+                                     const float* z_x4, const int32_t* wsum8, const int32_t* wsum4) {
+    const bool asym = z_x8 != nullptr;  // then x8 / x4 hold unsigned codes
     Params p;
     p.T = T; p.N = N; p.r = r; p.row4 = (K - r) / 2;
     p.units = N / kUnitRows;
@@ -552,6 +595,7 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
     p.early_weights = g_early_weights;
     p.x8 = x8; p.x4 = x4; p.s_x8 = s_x8; p.s_x4 = s_x4; p.s_w8 = s_w8; p.s_w4 = s_w4;
     p.w_fp16 = w_scale_fp16 ? 1 : 0;
+    p.z_x8 = z_x8; p.z_x4 = z_x4; p.wsum8 = wsum8; p.wsum4 = wsum4;
     p.Y = Y; p.y_dtype = y_dtype; p.dbg8 = dbg8; p.dbg4 = dbg8 ? dbg4 : nullptr;
     p.status = device_status_ptr();
     const size_t smem = fixed + static_cast<size_t>(kWarps) * nstages * kItemRows * 64 * cs;
@@ -564,16 +608,23 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int grid = p.units < sms ? p.units : sms;
     const int variant = (TT == 2 ? 4 : 0) + (cs == 5 ? 2 : 0) + split;
+#define RESQ_STREAM_CASE(v, tt, c, sp)                                                               \
+    case v:                                                                                          \
+        return asym ? launch_variant<tt, c, sp, true>(t8, t4, p, grid, smem, st)                     \
+                    : launch_variant<tt, c, sp, false>(t8, t4, p, grid, smem, st);
     switch (variant) {
-        case 0: return launch_variant<1, 3, false>(t8, t4, p, grid, smem, st);
-        case 1: return launch_variant<1, 3, true>(t8, t4, p, grid, smem, st);
-        case 2: return launch_variant<1, 5, false>(t8, t4, p, grid, smem, st);
-        case 3: return launch_variant<1, 5, true>(t8, t4, p, grid, smem, st);
-        case 4: return launch_variant<2, 3, false>(t8, t4, p, grid, smem, st);
-        case 5: return launch_variant<2, 3, true>(t8, t4, p, grid, smem, st);
-        case 6: return launch_variant<2, 5, false>(t8, t4, p, grid, smem, st);
-        default: return launch_variant<2, 5, true>(t8, t4, p, grid, smem, st);
+        RESQ_STREAM_CASE(0, 1, 3, false)
+        RESQ_STREAM_CASE(1, 1, 3, true)
+        RESQ_STREAM_CASE(2, 1, 5, false)
+        RESQ_STREAM_CASE(3, 1, 5, true)
+        RESQ_STREAM_CASE(4, 2, 3, false)
+        RESQ_STREAM_CASE(5, 2, 3, true)
+        RESQ_STREAM_CASE(6, 2, 5, false)
+        default:
+            return asym ? launch_variant<2, 5, true, true>(t8, t4, p, grid, smem, st)
+                        : launch_variant<2, 5, true, false>(t8, t4, p, grid, smem, st);
     }
+#undef RESQ_STREAM_CASE
 }
 
 }  // namespace resq

@@ -57,7 +57,9 @@ cudaError_t launch_mixed_gemm_decode(int T, int N, int K, int r, const int8_t* x
 cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x8, const uint8_t* x4,
                                      const float* s_x8, const float* s_x4, const int8_t* w8, const uint8_t* w4,
                                      const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
-                                     int32_t* dbg8, int32_t* dbg4, cudaStream_t st);
+                                     int32_t* dbg8, int32_t* dbg4, cudaStream_t st, const float* z_x8 = nullptr,
+                                     const float* z_x4 = nullptr, const int32_t* wsum8 = nullptr,
+                                     const int32_t* wsum4 = nullptr);  // z_x8 != NULL: asymmetric, unsigned codes
 void set_decode_early_weights(int on);
 
 // Online projection C = X·P (bf16 x bf16 -> fp32) on tcgen05 kind::f16, CTA pairs; writes fp32 C [T][K].

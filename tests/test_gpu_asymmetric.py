@@ -177,3 +177,37 @@ def test_asym_online_projection(resq):
     g8, g4 = host(u8).astype(np.int32), host(u4e).astype(np.int32)
     assert np.abs(g8 - o8).max() <= 1 and np.abs(g4 - o4).max() <= 1
     assert ((g8 != o8).sum() + (g4 != o4).sum()) / float(T * K) <= 1e-3
+
+
+@pytest.mark.parametrize("T,K,N,r,fp16", [
+    (1, 4096, 4096, 512, True),      # o_proj shape, one token: streaming kernel, split staging
+    (4, 4096, 1024, 512, True),
+    (16, 4096, 6144, 512, True),     # packed staging (T > 8)
+    (9, 2048, 264, 256, False),
+    (3, 1056, 72, 96, False),        # segment lengths that are not multiples of a step
+    (16, 14336, 256, 1792, True),    # down_proj reduction length
+    (2, 4096, 8, 512, False),        # a single unit
+])
+def test_asym_decode_bit_exact(resq, T, K, N, r, fp16):
+    """T <= 16 with packed codes: the weight-streaming kernel with unsigned activation codes."""
+    C_bits = _shifted(T, K, 980 + T)
+    _, Wp = synthetic_folded(2, K, N, r, seed_shift=40 + T)
+    pw = oracle.pack_weights(Wp, r, scale_fp16=fp16)
+    res = oracle.linear_asym(C_bits, None, pw)
+    desc = resq.layer_desc(K, N, r, resq.SCALE_FP16 if fp16 else resq.SCALE_FP32)
+    sdt = torch.float16 if fp16 else torch.float32
+    W = resq.Weights(desc, dev(pw.q8), dev(pw.w4_packed), dev(pw.s8).to(sdt), dev(pw.s4).to(sdt), None)
+    ws8, ws4 = resq.resq_weight_row_sums(W)
+    wsp = resq.alloc_workspace_asym(desc, T, False, False)
+    y32 = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+    a8 = torch.full((T, N), -1, dtype=torch.int32, device="cuda")
+    a4 = torch.full((T, N), -1, dtype=torch.int32, device="cuda")
+    resq.resq_mixed_gemm_asym(W, ws8, ws4, dev(res.u8), dev(res.u4_packed), dev(res.s_x8), dev(res.s_x4),
+                              dev(res.z_x8), dev(res.z_x4), y32, wsp, a8, a4)
+    ybf = torch.zeros((T, N), dtype=torch.bfloat16, device="cuda")
+    resq.resq_mixed_gemm_asym(W, ws8, ws4, dev(res.u8), dev(res.u4_packed), dev(res.s_x8), dev(res.s_x4),
+                              dev(res.z_x8), dev(res.z_x4), ybf, wsp)
+    assert resq.resq_device_status() == resq.OK
+    assert (host(a8) == res.acc8).all()
+    assert (host(a4) == res.acc4).all()
+    _check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))
