@@ -25,7 +25,7 @@
  *    segment; s = a / qmax as an IEEE fp32 division (qmax = 127 or 7); if the scale is stored as
  *    fp16 it is rounded to fp16 first and the rounded value is the one used; code =
  *    clamp(round-half-even(x / s)) with an IEEE fp32 division; a == 0 gives s = 0 and codes 0.
- *  - Shape rules: r % 32 == 0, (K - r) % 32 == 0, 0 < r < K, n_out % 8 == 0, T >= 1.
+ *  - Shape rules: r % 32 == 0, (K - r) % 32 == 0, 0 <= r < K (r = 0: uniform INT4), n_out % 8 == 0, T >= 1.
  *    Data pointers must be 16-byte aligned.
  *  - Every function returns a resq_status_t (0 = success).  Arguments are validated on the host
  *    before anything is launched; on a non-zero return nothing was enqueued.  Waits inside the
@@ -111,6 +111,19 @@ int resq_pack_weights(const resq_layer_desc_t* desc, const float* W_proj, int8_t
 int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int8_t* x8, uint8_t* x4,
                           float* s_x8, float* s_x4, int8_t* x4_i8, void* workspace,
                           size_t workspace_bytes, void* stream);
+
+/*
+ * The paper's own down_proj input path (Section 4.3): U_D is a Hadamard matrix, so the projection that cannot
+ * be folded is a fast transform, and the down_proj weights and activations are quantized uniformly to 4 bits
+ * (r = 0; a mixed split r > 0 is accepted as well).  C = X·H_K / sqrt(K) is formed in fp32 per token in shared
+ * memory and quantized at once (Eq. 1, Eq. 2) without ever being written out.  H_K = Sylvester(2^k) (x) H_m with
+ * coefficient index a·m + b; m = 1, or m = 12 / 28 by Paley's second construction (q = 5 / 13) -- the paper
+ * names no construction; K = 8192, 14336 and 28672 are covered.  Other K, or K·4 bytes > 200 KB, give
+ * RESQ_ERR_SHAPE.  Outputs as resq_project_quantize (x8 may be NULL when r = 0).  The weights to pair with it are
+ * resq_pack_weights of (H_K^T W / sqrt(K))^T.  Every entry point accepts r = 0 (then w8 / x8 may be NULL).
+ */
+int resq_hadamard_quantize(const void* X, int T, int K, int r, int8_t* x8, uint8_t* x4, float* s_x8, float* s_x4,
+                           int8_t* x4_i8, void* stream);
 
 /*
  * The online projection alone (Section 4.3, U_D): C = X·P with X bf16 [T][K], P bf16 [K][K] (row i =

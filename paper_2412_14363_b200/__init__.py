@@ -22,7 +22,7 @@ Y_BF16, Y_FP32 = 0, 1
 
 EXPORTS = [
     "resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_bytes", "resq_workspace_bytes",
-    "resq_pack_weights", "resq_project", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
+    "resq_pack_weights", "resq_project", "resq_hadamard_quantize", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
     "resq_unpack_int4", "resq_set_option",
     "resq_weight_row_sums", "resq_project_quantize_asym", "resq_mixed_gemm_asym", "resq_linear_asym",
     "resq_workspace_bytes_asym",
@@ -61,6 +61,7 @@ lib.resq_workspace_bytes.restype = _sz
 lib.resq_workspace_bytes.argtypes = [_dp, _i, _i, _i]
 lib.resq_pack_weights.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_project.argtypes = [_vp, _vp, _i, _i, _vp, _vp]
+lib.resq_hadamard_quantize.argtypes = [_vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_project_quantize.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 lib.resq_project_quantize_static.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_mixed_gemm.argtypes = [_dp, _i, _vp, _vp, _vp, _vp, _vp, ctypes.POINTER(WeightsStruct), _vp, _i, _vp, _vp,
@@ -156,6 +157,13 @@ def resq_project(X, P, C):
     _check(lib.resq_project(_ptr(X), _ptr(P), T, K, _ptr(C), _stream()), "resq_project")
 
 
+def resq_hadamard_quantize(X, r: int, x8, x4, s_x8, s_x4, x4_i8=None):
+    """X bf16 [T][K] -> codes and scales of X·H_K/sqrt(K) (Hadamard U_D, Section 4.3); r = 0: uniform INT4."""
+    T, K = X.shape
+    _check(lib.resq_hadamard_quantize(_ptr(X), T, K, r, _ptr(x8), _ptr(x4), _ptr(s_x8), _ptr(s_x4), _ptr(x4_i8),
+                                      _stream()), "resq_hadamard_quantize")
+
+
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -171,7 +179,7 @@ def resq_project_quantize_static(X, P, r: int, x8, x4, s_x8, s_x4, x4_i8=None):
 
 def resq_mixed_gemm(W: Weights, x8, x4, s_x8, s_x4, Y, workspace, dbg_acc8=None, dbg_acc4=None, x4_i8=None):
     import torch
-    T = x8.shape[0]
+    T = s_x8.shape[0]  # x8 may be None for a uniform INT4 layer (r = 0)
     y_dtype = Y_BF16 if Y.dtype == torch.bfloat16 else Y_FP32
     ws = W.struct()
     _check(lib.resq_mixed_gemm(ctypes.byref(W.desc), T, _ptr(x8), _ptr(x4), _ptr(x4_i8), _ptr(s_x8), _ptr(s_x4),
@@ -237,7 +245,7 @@ def resq_project_quantize_asym(X, P, r: int, u8, u4, s_x8, s_x4, z_x8, z_x4, u4_
 def resq_mixed_gemm_asym(W: Weights, wsum8, wsum4, u8, u4, s_x8, s_x4, z_x8, z_x4, Y, workspace, dbg_acc8=None,
                          dbg_acc4=None, u4_u8=None):
     import torch
-    T = u8.shape[0]
+    T = s_x8.shape[0]
     y_dtype = Y_BF16 if Y.dtype == torch.bfloat16 else Y_FP32
     ws = W.struct()
     _check(lib.resq_mixed_gemm_asym(ctypes.byref(W.desc), T, _ptr(u8), _ptr(u4), _ptr(u4_u8), _ptr(s_x8), _ptr(s_x4),

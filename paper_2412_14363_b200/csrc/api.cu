@@ -42,7 +42,7 @@ inline size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 int check_shape(int K, int n_out, int r) {
-    if (K <= 0 || r <= 0 || r >= K || n_out <= 0) return RESQ_ERR_SHAPE;
+    if (K <= 0 || r < 0 || r >= K || n_out <= 0) return RESQ_ERR_SHAPE;  // r == 0: uniform INT4 (Section 4.3, down_proj)
     if (r % 32 != 0 || (K - r) % 32 != 0 || n_out % 8 != 0) return RESQ_ERR_SHAPE;
     return RESQ_OK;
 }
@@ -116,7 +116,7 @@ size_t resq_workspace_bytes(const resq_layer_desc_t* d, int T, int has_P, int ha
 int resq_pack_weights(const resq_layer_desc_t* d, const float* W_proj, int8_t* w8, uint8_t* w4, void* s_w8,
                       void* s_w4, int8_t* w4_i8, void* stream) {
     if (int e = check_desc(d)) return e;
-    if (!W_proj || !w8 || !w4 || !s_w8 || !s_w4) return RESQ_ERR_NULL;
+    if (!W_proj || (!w8 && d->r > 0) || !w4 || !s_w8 || !s_w4) return RESQ_ERR_NULL;
     if (!aligned16(W_proj) || !aligned16(w8) || !aligned16(w4) || !aligned16(s_w8) || !aligned16(s_w4) ||
         !aligned16(w4_i8))
         return RESQ_ERR_ALIGN;
@@ -130,7 +130,7 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
                           float* s_x4, int8_t* x4_i8, void* workspace, size_t workspace_bytes, void* stream) {
     if (T < 1) return RESQ_ERR_SHAPE;
     if (int e = check_shape(K, 8, r)) return e;
-    if (!X || !x8 || !s_x8 || !s_x4 || (!x4 && !x4_i8)) return RESQ_ERR_NULL;
+    if (!X || (!x8 && r > 0) || !s_x8 || !s_x4 || (!x4 && !x4_i8)) return RESQ_ERR_NULL;
     if (!aligned16(X) || !aligned16(P) || !aligned16(x8) || !aligned16(x4) || !aligned16(s_x8) ||
         !aligned16(s_x4) || !aligned16(x4_i8) || !aligned16(workspace))
         return RESQ_ERR_ALIGN;
@@ -160,6 +160,18 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
     return RESQ_OK;
 }
 
+int resq_hadamard_quantize(const void* X, int T, int K, int r, int8_t* x8, uint8_t* x4, float* s_x8, float* s_x4,
+                           int8_t* x4_i8, void* stream) {
+    if (T < 1) return RESQ_ERR_SHAPE;
+    if (int e = check_shape(K, 8, r)) return e;
+    if (!X || (!x8 && r > 0) || !s_x8 || !s_x4 || (!x4 && !x4_i8)) return RESQ_ERR_NULL;
+    if (!aligned16(X) || !aligned16(x8) || !aligned16(x4) || !aligned16(s_x8) || !aligned16(s_x4) || !aligned16(x4_i8))
+        return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    const cudaError_t e = launch_hadamard_quantize(X, T, K, r, x8, x4, s_x8, s_x4, x4_i8, static_cast<cudaStream_t>(stream));
+    return e == cudaErrorNotSupported ? RESQ_ERR_SHAPE : cuda_status(e);
+}
+
 int resq_project(const void* X, const void* P, int T, int K, float* C, void* stream) {
     if (T < 1 || K <= 0 || K % 8 != 0) return RESQ_ERR_SHAPE;
     if (!X || !P || !C) return RESQ_ERR_NULL;
@@ -178,6 +190,7 @@ static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, 
         const cudaError_t e = launch_mixed_gemm_stream(T, d->n_out, d->K, d->r, x8, x4, s_x8, s_x4, W->w8, W->w4,
                                                        W->s_w8, W->s_w4, fp16, Y, y_dtype, dbg8, dbg4, st);
         if (e != cudaErrorNotSupported) return cuda_status(e);
+        if (d->r == 0) return RESQ_ERR_SHAPE;  // the cluster split-K fallback needs an INT8 segment
     }
     if (T <= kDecodeMaxT)
         return cuda_status(launch_mixed_gemm_decode(T, d->n_out, d->K, d->r, x8, x4, s_x8, s_x4, W->w8, W->w4,
@@ -199,8 +212,8 @@ static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, 
                                                W->s_w4, fp16, Y, y_dtype, dbg8, dbg4, st));
 }
 
-static int check_weights(const resq_weights_t* W) {
-    if (!W || !W->w8 || !W->w4 || !W->s_w8 || !W->s_w4) return RESQ_ERR_NULL;
+static int check_weights(const resq_weights_t* W, int r) {
+    if (!W || (!W->w8 && r > 0) || !W->w4 || !W->s_w8 || !W->s_w4) return RESQ_ERR_NULL;
     if (!aligned16(W->w8) || !aligned16(W->w4) || !aligned16(W->s_w8) || !aligned16(W->s_w4) ||
         !aligned16(W->w4_i8))
         return RESQ_ERR_ALIGN;
@@ -212,10 +225,10 @@ int resq_mixed_gemm(const resq_layer_desc_t* d, int T, const int8_t* x8, const u
                     int32_t* dbg_acc8, int32_t* dbg_acc4, void* workspace, size_t workspace_bytes, void* stream) {
     if (int e = check_desc(d)) return e;
     if (T < 1 || (y_dtype != RESQ_Y_BF16 && y_dtype != RESQ_Y_FP32)) return RESQ_ERR_SHAPE;
-    if (!x8 || !s_x8 || !s_x4 || !Y) return RESQ_ERR_NULL;
+    if ((!x8 && d->r > 0) || !s_x8 || !s_x4 || !Y) return RESQ_ERR_NULL;
     if (!x4 && (!x4_i8 || T <= kDecodeMaxT)) return RESQ_ERR_NULL;
     if ((dbg_acc8 == nullptr) != (dbg_acc4 == nullptr)) return RESQ_ERR_NULL;
-    if (int e = check_weights(W)) return e;
+    if (int e = check_weights(W, d->r)) return e;
     if (!aligned16(x8) || !aligned16(x4) || !aligned16(x4_i8) || !aligned16(s_x8) || !aligned16(s_x4) ||
         !aligned16(Y) || !aligned16(dbg_acc8) || !aligned16(dbg_acc4) || !aligned16(workspace))
         return RESQ_ERR_ALIGN;
@@ -231,7 +244,7 @@ int resq_linear(const resq_layer_desc_t* d, int T, const void* X, const void* P,
     if (int e = check_desc(d)) return e;
     if (T < 1 || (y_dtype != RESQ_Y_BF16 && y_dtype != RESQ_Y_FP32)) return RESQ_ERR_SHAPE;
     if (!X || !Y) return RESQ_ERR_NULL;
-    if (int e = check_weights(W)) return e;
+    if (int e = check_weights(W, d->r)) return e;
     if (!aligned16(X) || !aligned16(P) || !aligned16(Y) || !aligned16(workspace)) return RESQ_ERR_ALIGN;
     const Workspace map = carve(d->K, d->n_out, d->r, T, P != nullptr, W->w4_i8 != nullptr);
     if (!workspace || workspace_bytes < map.total) return RESQ_ERR_WORKSPACE;
@@ -255,7 +268,7 @@ int resq_linear(const resq_layer_desc_t* d, int T, const void* X, const void* P,
 int resq_weight_row_sums(const resq_layer_desc_t* d, const resq_weights_t* W, int32_t* wsum8, int32_t* wsum4,
                          void* stream) {
     if (int e = check_desc(d)) return e;
-    if (int e = check_weights(W)) return e;
+    if (int e = check_weights(W, d->r)) return e;
     if (!wsum8 || !wsum4) return RESQ_ERR_NULL;
     if (!aligned16(wsum8) || !aligned16(wsum4)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
@@ -268,7 +281,7 @@ int resq_project_quantize_asym(const void* X, const void* P, int T, int K, int r
                                size_t workspace_bytes, void* stream) {
     if (T < 1) return RESQ_ERR_SHAPE;
     if (int e = check_shape(K, 8, r)) return e;
-    if (!X || !u8 || !s_x8 || !s_x4 || !z_x8 || !z_x4 || (!u4 && !u4_u8)) return RESQ_ERR_NULL;
+    if (!X || (!u8 && r > 0) || !s_x8 || !s_x4 || !z_x8 || !z_x4 || (!u4 && !u4_u8)) return RESQ_ERR_NULL;
     if (!aligned16(X) || !aligned16(P) || !aligned16(u8) || !aligned16(u4) || !aligned16(s_x8) || !aligned16(s_x4) ||
         !aligned16(z_x8) || !aligned16(z_x4) || !aligned16(u4_u8) || !aligned16(workspace))
         return RESQ_ERR_ALIGN;
@@ -341,9 +354,9 @@ int resq_mixed_gemm_asym(const resq_layer_desc_t* d, int T, const uint8_t* u8, c
                          int32_t* dbg_acc8, int32_t* dbg_acc4, void* workspace, size_t workspace_bytes, void* stream) {
     if (int e = check_desc(d)) return e;
     if (T < 1 || (y_dtype != RESQ_Y_BF16 && y_dtype != RESQ_Y_FP32)) return RESQ_ERR_SHAPE;
-    if (!u8 || !s_x8 || !s_x4 || !z_x8 || !z_x4 || !wsum8 || !wsum4 || !Y || (!u4 && !u4_u8)) return RESQ_ERR_NULL;
+    if ((!u8 && d->r > 0) || !s_x8 || !s_x4 || !z_x8 || !z_x4 || !wsum8 || !wsum4 || !Y || (!u4 && !u4_u8)) return RESQ_ERR_NULL;
     if ((dbg_acc8 == nullptr) != (dbg_acc4 == nullptr)) return RESQ_ERR_NULL;
-    if (int e = check_weights(W)) return e;
+    if (int e = check_weights(W, d->r)) return e;
     if (!aligned16(u8) || !aligned16(u4) || !aligned16(u4_u8) || !aligned16(s_x8) || !aligned16(s_x4) ||
         !aligned16(z_x8) || !aligned16(z_x4) || !aligned16(wsum8) || !aligned16(wsum4) || !aligned16(Y) ||
         !aligned16(dbg_acc8) || !aligned16(dbg_acc4) || !aligned16(workspace))
@@ -361,7 +374,7 @@ int resq_linear_asym(const resq_layer_desc_t* d, int T, const void* X, const voi
     if (int e = check_desc(d)) return e;
     if (T < 1 || (y_dtype != RESQ_Y_BF16 && y_dtype != RESQ_Y_FP32)) return RESQ_ERR_SHAPE;
     if (!X || !Y || !wsum8 || !wsum4) return RESQ_ERR_NULL;
-    if (int e = check_weights(W)) return e;
+    if (int e = check_weights(W, d->r)) return e;
     if (!aligned16(X) || !aligned16(P) || !aligned16(Y) || !aligned16(wsum8) || !aligned16(wsum4) ||
         !aligned16(workspace))
         return RESQ_ERR_ALIGN;

@@ -601,7 +601,12 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
     const size_t smem = fixed + static_cast<size_t>(kWarps) * nstages * kItemRows * 64 * cs;
 
     CUtensorMap t8, t4;
-    if (!make_map_rows(&t8, w8, N, r, 64 * cs) || !make_map_rows(&t4, w4, N, p.row4, 64 * cs)) return cudaErrorInvalidValue;
+    if (!make_map_rows(&t4, w4, N, p.row4, 64 * cs)) return cudaErrorInvalidValue;
+    if (r > 0) {
+        if (!make_map_rows(&t8, w8, N, r, 64 * cs)) return cudaErrorInvalidValue;
+    } else {
+        t8 = t4;  // uniform INT4: no INT8 chunks are ever requested
+    }
     int dev = 0, sms = 148;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;

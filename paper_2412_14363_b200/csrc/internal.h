@@ -21,6 +21,11 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
                                   uint8_t* q4, void* s8, void* s4, bool scale_fp16, int8_t* q4_i8,
                                   size_t in_row_stride, cudaStream_t st);
 
+// Hadamard transform of the bf16 rows (H_K / sqrt(K), K = 2^k * {1, 12, 28}) fused with the split quantizer
+// (r may be 0).  Returns cudaErrorNotSupported for other K or rows wider than 200 KB of fp32.
+cudaError_t launch_hadamard_quantize(const void* X, size_t rows, int K, int r, int8_t* q8, uint8_t* q4, float* s8,
+                                     float* s4, int8_t* q4_i8, cudaStream_t st);
+
 // codes_unsigned: the nibbles are 0..15 (asymmetric activation codes) instead of two's complement.
 cudaError_t launch_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, cudaStream_t st,
                                bool codes_unsigned = false);

@@ -245,6 +245,10 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                 uint32_t a8[16];
                 tmem_ld16(lane_addr + c * 16, a8);
                 tmem_ld_wait();
+                if (p.kb8 == 0) {  // uniform INT4: the INT8 accumulator was never written
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) a8[j] = 0;
+                }
                 const int cb = ch * (BN / 2) + c * 16;  // first column of the chunk inside the tile
                 const int nb = n0 + cb;
                 const uint32_t* a4c = &a4[c >> 1][(c & 1) * 16];
@@ -353,9 +357,13 @@ cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8
     }
     const int K4 = K - r;
     CUtensorMap tA8, tA4, tB8, tB4;
-    if (!make_map_u8(&tA8, x8, T, r, BM) || !make_map_u8(&tA4, x4e, T, K4, BM) ||
-        !make_map_u8(&tB8, w8, N, r, BN_HALF) || !make_map_u8(&tB4, w4e, N, K4, BN_HALF))
-        return cudaErrorInvalidValue;
+    if (!make_map_u8(&tA4, x4e, T, K4, BM) || !make_map_u8(&tB4, w4e, N, K4, BN_HALF)) return cudaErrorInvalidValue;
+    if (r > 0) {
+        if (!make_map_u8(&tA8, x8, T, r, BM) || !make_map_u8(&tB8, w8, N, r, BN_HALF)) return cudaErrorInvalidValue;
+    } else {  // uniform INT4: no INT8 segment, its maps are never used
+        tA8 = tA4;
+        tB8 = tB4;
+    }
     Params p;
     p.T = T; p.N = N; p.r = r; p.K4 = K4;
     int sms = 148;

@@ -4,6 +4,7 @@
 // keeps up to kMaxChunks of them in registers so the row is read from memory once, reduces the two
 // per-segment absmax values with warp shuffles + one shared-memory step, then emits int8 codes
 // (8-byte stores) and packed int4 codes (4-byte stores).
+#include <cmath>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -346,6 +347,186 @@ __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* _
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Hadamard basis for the down_proj input (Section 4.3: U_D is a Hadamard matrix so that the projection
+// that cannot be folded costs a fast transform instead of a dense product), fused with the per-token
+// quantizer: C = X * H_K / sqrt(K), H_K = Sylvester(2^k) (x) H_m with coefficient index a * m + b, m = 1, or
+// m = 12 / 28 with Paley's second construction (q = 5 / 13).  One CTA per row: the row is widened to fp32
+// in shared memory, multiplied group-wise by the small factor (constant memory), run through the
+// Sylvester butterflies three index bits per pass (eight values in registers, conflict-free strides),
+// scaled, and then quantized exactly as in the fast path above (absmax per segment, reciprocal-product
+// rounding with the exact fallback).  r = 0 gives the paper's uniform INT4 down_proj input.
+__constant__ float c_paley12[12 * 12];
+__constant__ float c_paley28[28 * 28];
+
+template <int M>
+__device__ __forceinline__ const float* small_factor() {
+    return M == 12 ? c_paley12 : c_paley28;
+}
+
+template <int M>
+__global__ void __launch_bounds__(kThreads)
+hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K, int kbits, int r, float inv_sqrt_k,
+                         int8_t* __restrict__ q8, uint8_t* __restrict__ q4, float* __restrict__ s8_out,
+                         float* __restrict__ s4_out, int8_t* __restrict__ q4e) {
+    extern __shared__ __align__(16) float hrow[];  // [K]
+    __shared__ float red[2][kThreads / 32];
+    const int tid = threadIdx.x;
+    const int nchunks = K >> 3, rchunks = r >> 3;
+    const int K4 = K - r;
+    const uint8_t* srow = reinterpret_cast<const uint8_t*>(hrow);
+    for (size_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        // 1. widen the bf16 row
+        const uint4* xp = reinterpret_cast<const uint4*>(X + row * static_cast<size_t>(K));
+        for (int c = tid; c < nchunks; c += kThreads) {
+            const uint4 u = __ldg(xp + c);
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+            float4 a, b;
+            a.x = __uint_as_float(w[0] << 16); a.y = __uint_as_float(w[0] & 0xFFFF0000u);
+            a.z = __uint_as_float(w[1] << 16); a.w = __uint_as_float(w[1] & 0xFFFF0000u);
+            b.x = __uint_as_float(w[2] << 16); b.y = __uint_as_float(w[2] & 0xFFFF0000u);
+            b.z = __uint_as_float(w[3] << 16); b.w = __uint_as_float(w[3] & 0xFFFF0000u);
+            reinterpret_cast<float4*>(hrow)[2 * c] = a;
+            reinterpret_cast<float4*>(hrow)[2 * c + 1] = b;
+        }
+        __syncthreads();
+        // 2. the small factor, one group of M consecutive coefficients per thread, in place
+        if constexpr (M > 1) {
+            const float* H = small_factor<M>();
+            for (int a = tid; a < (K / M); a += kThreads) {
+                float x[M], y[M];
+#pragma unroll
+                for (int i = 0; i < M; ++i) x[i] = hrow[a * M + i];
+#pragma unroll
+                for (int j = 0; j < M; ++j) {
+                    float acc = 0.f;
+#pragma unroll
+                    for (int i = 0; i < M; ++i) acc = fmaf(x[i], H[i * M + j], acc);
+                    y[j] = acc;
+                }
+#pragma unroll
+                for (int j = 0; j < M; ++j) hrow[a * M + j] = y[j];
+            }
+            __syncthreads();
+        }
+        // 3. Sylvester butterflies over the index bits of a, three bits per pass
+        for (int s = 0; s < kbits; s += 3) {
+            const int nb = kbits - s < 3 ? kbits - s : 3;
+            const int count = K >> nb;
+            const int stride = M << s;
+            for (int i = tid; i < count; i += kThreads) {
+                const int arest = i / M, b = i - arest * M;
+                const int a0 = ((arest >> s) << (s + nb)) | (arest & ((1 << s) - 1));
+                float* base = hrow + a0 * M + b;
+                float v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = j < (1 << nb) ? base[j * stride] : 0.f;
+#pragma unroll
+                for (int bit = 0; bit < 3; ++bit) {
+                    if (bit < nb) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (!(j & (1 << bit))) {
+                                const float lo = v[j], hi = v[j | (1 << bit)];
+                                v[j] = lo + hi;
+                                v[j | (1 << bit)] = lo - hi;
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (j < (1 << nb)) base[j * stride] = v[j];
+            }
+            __syncthreads();
+        }
+        // 4. scale by 1 / sqrt(K) and take the two absmax values
+        float a8 = 0.f, a4 = 0.f;
+        for (int c = tid; c < nchunks; c += kThreads) {
+            float4* p = reinterpret_cast<float4*>(hrow) + 2 * c;
+            float4 a = p[0], b = p[1];
+            a.x *= inv_sqrt_k; a.y *= inv_sqrt_k; a.z *= inv_sqrt_k; a.w *= inv_sqrt_k;
+            b.x *= inv_sqrt_k; b.y *= inv_sqrt_k; b.z *= inv_sqrt_k; b.w *= inv_sqrt_k;
+            p[0] = a; p[1] = b;
+            const float m = fmaxf(fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))),
+                                  fmaxf(fmaxf(fabsf(b.x), fabsf(b.y)), fmaxf(fabsf(b.z), fabsf(b.w))));
+            if (c < rchunks) a8 = fmaxf(a8, m);
+            else a4 = fmaxf(a4, m);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            a8 = fmaxf(a8, __shfl_xor_sync(0xffffffffu, a8, o));
+            a4 = fmaxf(a4, __shfl_xor_sync(0xffffffffu, a4, o));
+        }
+        if ((tid & 31) == 0) {
+            red[0][tid >> 5] = a8;
+            red[1][tid >> 5] = a4;
+        }
+        __syncthreads();  // also: every thread's scaled values are in place
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) {
+            a8 = fmaxf(a8, red[0][w]);
+            a4 = fmaxf(a4, red[1][w]);
+        }
+        // 5. codes
+        const float s8 = __fdiv_rn(a8, 127.f), s4 = __fdiv_rn(a4, 7.f);
+        const float inv8 = s8 > 0.f ? __frcp_rn(s8) : 0.f, inv4 = s4 > 0.f ? __frcp_rn(s4) : 0.f;
+        const bool exact8 = s8 > 0.f && !(inv8 >= 1.1754944e-38f && inv8 <= 3.0e38f);
+        const bool exact4 = s4 > 0.f && !(inv4 >= 1.1754944e-38f && inv4 <= 3.0e38f);
+        if (tid == 0) {
+            s8_out[row] = s8;
+            s4_out[row] = s4;
+        }
+        int8_t* q8row = q8 + row * static_cast<size_t>(r);
+        uint8_t* q4row = q4 ? q4 + row * static_cast<size_t>(K4 >> 1) : nullptr;
+        int8_t* q4e_row = q4e ? q4e + row * static_cast<size_t>(K4) : nullptr;
+        for (int c = tid; c < nchunks; c += kThreads) {
+            uint32_t t[8];
+            const bool seg8 = c < rchunks;
+            const float s = seg8 ? s8 : s4;
+            if (s > 0.f) fast_codes(lds_chunk<true>(srow, c), s, seg8 ? inv8 : inv4, seg8 ? exact8 : exact4, t);
+            else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) t[k] = 0;
+            }
+            const uint32_t w0 = pack_low_bytes(t[0], t[1], t[2], t[3]), w1 = pack_low_bytes(t[4], t[5], t[6], t[7]);
+            if (seg8) {
+                *reinterpret_cast<uint2*>(q8row + c * 8) = make_uint2(w0, w1);
+            } else {
+                const int jj = (c - rchunks) * 8;
+                if (q4e_row) *reinterpret_cast<uint2*>(q4e_row + jj) = make_uint2(w0, w1);
+                if (q4row) {
+                    uint32_t packed = 0;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) packed |= (t[k] & 0xFu) << (4 * k);
+                    *reinterpret_cast<uint32_t*>(q4row + (jj >> 1)) = packed;
+                }
+            }
+        }
+        __syncthreads();  // the row buffer is reused by the next row
+    }
+}
+
+// Paley's second construction for a prime q = 1 (mod 4): a Hadamard matrix of order 2 (q + 1) from the
+// quadratic character chi of GF(q): S = [[0, 1^T], [1, chi(i - j)]], H = S (x) [[1,1],[1,-1]] + I (x) [[1,-1],[-1,-1]].
+void paley2(int q, float* H /* [2(q+1)]^2 */) {
+    const int n = q + 1, N = 2 * n;
+    auto chi = [q](int a) {
+        a = ((a % q) + q) % q;
+        if (a == 0) return 0;
+        for (int x = 1; x < q; ++x)
+            if ((x * x) % q == a) return 1;
+        return -1;
+    };
+    auto S = [&](int i, int j) { return i == 0 ? (j == 0 ? 0 : 1) : (j == 0 ? 1 : chi((i - 1) - (j - 1))); };
+    const int A[2][2] = {{1, 1}, {1, -1}}, B[2][2] = {{1, -1}, {-1, -1}};
+    for (int i = 0; i < n; ++i)
+        for (int j = 0; j < n; ++j)
+            for (int u = 0; u < 2; ++u)
+                for (int v = 0; v < 2; ++v)
+                    H[(2 * i + u) * N + 2 * j + v] = static_cast<float>(S(i, j) * A[u][v] + (i == j ? B[u][v] : 0));
+}
+
 }  // namespace
 
 cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, int K, int r, int8_t* q8,
@@ -393,6 +574,54 @@ cudaError_t launch_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, 
     if (blocks > 148 * 32) blocks = 148 * 32;
     if (codes_unsigned) unpack_int4_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, st>>>(packed, out, nwords);
     else unpack_int4_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, st>>>(packed, out, nwords);
+    return cudaGetLastError();
+}
+
+
+// K = 2^k * m with m in {28, 12, 1} (largest first); false if K has no such form.
+bool hadamard_factor(int K, int* kbits, int* m) {
+    for (int mm : {28, 12, 1}) {
+        if (K % mm) continue;
+        const int a = K / mm;
+        if (a & (a - 1)) continue;
+        int kb = 0;
+        while ((1 << kb) < a) ++kb;
+        *kbits = kb;
+        *m = mm;
+        return true;
+    }
+    return false;
+}
+
+cudaError_t launch_hadamard_quantize(const void* X, size_t rows, int K, int r, int8_t* q8, uint8_t* q4, float* s8,
+                                     float* s4, int8_t* q4_i8, cudaStream_t st) {
+    if (rows == 0) return cudaSuccess;
+    int kbits = 0, m = 0;
+    if (!hadamard_factor(K, &kbits, &m)) return cudaErrorNotSupported;
+    const size_t smem = static_cast<size_t>(K) * 4;
+    if (smem > 200u * 1024u) return cudaErrorNotSupported;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    static bool ready[64] = {};
+    if (dev < 64 && !ready[dev]) {
+        // Once per device: the two small factors into constant memory, the shared-memory limit of the kernels.
+        static float h12[12 * 12], h28[28 * 28];
+        paley2(5, h12);
+        paley2(13, h28);
+        if ((e = cudaMemcpyToSymbol(c_paley12, h12, sizeof(h12))) != cudaSuccess) return e;
+        if ((e = cudaMemcpyToSymbol(c_paley28, h28, sizeof(h28))) != cudaSuccess) return e;
+        for (auto k : {hadamard_quantize_kernel<1>, hadamard_quantize_kernel<12>, hadamard_quantize_kernel<28>})
+            if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess)
+                return e;
+        ready[dev] = true;
+    }
+    const float inv_sqrt_k = static_cast<float>(1.0 / sqrt(static_cast<double>(K)));
+    const unsigned grid = static_cast<unsigned>(rows < 148u * 16u ? rows : 148u * 16u);
+    const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(X);
+    if (m == 1) hadamard_quantize_kernel<1><<<grid, kThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
+    else if (m == 12) hadamard_quantize_kernel<12><<<grid, kThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
+    else hadamard_quantize_kernel<28><<<grid, kThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
     return cudaGetLastError();
 }
 

@@ -64,13 +64,17 @@ def test_host_validation_happens_before_any_launch(resq):
     ws = resq.WeightsStruct(fake, fake, fake, fake, None)
     W = ctypes.byref(ws)
     # shape rules
-    for K, N, r in ((512, 512, 0), (512, 512, 512), (512, 512, 48), (500, 512, 64), (512, 508, 64), (0, 8, 0)):
+    for K, N, r in ((512, 512, -32), (512, 512, 512), (512, 512, 48), (500, 512, 64), (512, 508, 64), (0, 8, 0)):
         bad = resq.layer_desc(K, N, r)
         assert L.resq_mixed_gemm(ctypes.byref(bad), 16, fake, fake, None, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
         assert L.resq_pack_weights(ctypes.byref(bad), fake, fake, fake, fake, fake, None, None) == resq.ERR_SHAPE
     assert L.resq_mixed_gemm(ctypes.byref(good), 0, fake, fake, None, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
     assert L.resq_mixed_gemm(ctypes.byref(good), 16, fake, fake, None, fake, fake, W, fake, 7, None, None, fake, 1 << 30, None) == resq.ERR_SHAPE
     assert L.resq_project_quantize(fake, None, 16, 512, 60, fake, fake, fake, fake, None, None, 0, None) == resq.ERR_SHAPE
+    # the Hadamard path: a width with no construction here, a misaligned input, a missing output
+    assert L.resq_hadamard_quantize(fake, 4, 1000, 0, None, fake, fake, fake, None, None) == resq.ERR_SHAPE
+    assert L.resq_hadamard_quantize(fake + 2, 4, 1024, 0, None, fake, fake, fake, None, None) == resq.ERR_ALIGN
+    assert L.resq_hadamard_quantize(fake, 4, 1024, 128, None, fake, fake, fake, None, None) == resq.ERR_NULL
     # null pointers
     assert L.resq_mixed_gemm(None, 16, fake, fake, None, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_NULL
     assert L.resq_mixed_gemm(ctypes.byref(good), 16, None, fake, None, fake, fake, W, fake, 0, None, None, fake, 1 << 30, None) == resq.ERR_NULL
