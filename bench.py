@@ -286,6 +286,52 @@ def asym_leg(resq, torch, dev, layers, T, steps):
             "per_layer": per_layer}
 
 
+# --------------------------------------------------------------------------------------- Hadamard leg
+def hadamard_leg(resq, torch, dev, L, T, steps, peaks):
+    """down_proj as the paper runs it (Section 4.3): Hadamard transform fused with uniform INT4 quantization of
+    the input, uniform INT4 weights (r = 0), instead of the dense bf16 projection with a mixed 8/4 split."""
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    desc = resq.layer_desc(L.K, L.N, 0)
+    W = resq.resq_pack_weights(desc, L.W_proj, with_w4_i8=True)   # stands in for (H^T W / sqrt(K))^T: same distribution
+    x4e = torch.empty((T, L.K), dtype=torch.int8, device=dev)
+    s8 = torch.empty(T, dtype=torch.float32, device=dev)
+    s4 = torch.empty(T, dtype=torch.float32, device=dev)
+    ws = resq.alloc_workspace(desc, T, False, True, device=dev)
+
+    def step(events=None):
+        e0 = ev() if events is not None else None
+        resq.resq_hadamard_quantize(L.X, 0, None, None, s8, s4, x4e)
+        e1 = ev() if events is not None else None
+        resq.resq_mixed_gemm(W, None, None, s8, s4, L.Y, ws, x4_i8=x4e)
+        if events is not None:
+            events.append((e0, e1, ev()))
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    events = []
+    for _ in range(steps):
+        step(events)
+    torch.cuda.synchronize()
+    q = statistics.mean(a.elapsed_time(b) for a, b, _ in events)
+    g = statistics.mean(b.elapsed_time(c) for _, b, c in events)
+    st = resq.resq_device_status()
+    if st != resq.OK:
+        raise SystemExit(f"device status {st}: {resq.status_string(st)}")
+    bytes_q = T * (2.0 * L.K + L.K + 8)   # read bf16, write one code per byte + scales
+    return {"workload": f"down_proj {L.K}->{L.N}, T={T}: Hadamard U_D + uniform INT4 (r = 0)", "steps": steps,
+            "hadamard_quantize_ms": round(q, 4), "hadamard_quantize_gbs": round(bytes_q / (q * 1e-3) / 1e9, 1),
+            "hadamard_quantize_frac_of_hbm_peak": round(bytes_q / (q * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+            "int4_gemm_ms": round(g, 4), "int4_gemm_tops": round(2.0 * T * L.K * L.N / (g * 1e-3) / 1e12, 1),
+            "layer_ms": round(q + g, 4)}
+
+
 # --------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import numpy as np
@@ -506,6 +552,11 @@ def run_ours(args):
     if not args.no_asym and not only:
         asym = asym_leg(resq, torch, dev, layers, T, max(5, min(args.steps, 10)))
 
+    # ---- the paper's own down_proj path: Hadamard U_D + uniform INT4 (r = 0)
+    had = None
+    if not args.no_asym and online:
+        had = hadamard_leg(resq, torch, dev, online[0], T, max(5, min(args.steps, 10)), peaks)
+
     # ---- decode variant of the same block (this rank only; reported by rank 0)
     decode = None
     if not args.no_decode and not only:
@@ -553,7 +604,7 @@ def run_ours(args):
             "mixed_gemm_frac_of_int8_peak": {"vs_measured_bf16_x2": kernels["mixed_gemm"]["frac"],
                                              "vs_nominal_4500": kernels["mixed_gemm"]["frac_of_nominal_4500"]},
             "per_layer": per_layer,
-            "roofline": roofline, "decode": decode, "asymmetric": asym, "e2e": e2e, "cpu_baseline": cpu_baseline, "parity_spot_check": parity,
+            "roofline": roofline, "decode": decode, "asymmetric": asym, "hadamard_down_proj": had, "e2e": e2e, "cpu_baseline": cpu_baseline, "parity_spot_check": parity,
             "gpu_launches": LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
         }
         print(json.dumps(line))

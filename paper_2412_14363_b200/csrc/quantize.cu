@@ -394,18 +394,25 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
         if constexpr (M > 1) {
             const float* H = small_factor<M>();
             for (int a = tid; a < (K / M); a += kThreads) {
+                // M * 4 bytes is a multiple of 16: the group moves as float4s (conflict-free at this stride)
+                float4* gp = reinterpret_cast<float4*>(hrow + a * M);
                 float x[M], y[M];
 #pragma unroll
-                for (int i = 0; i < M; ++i) x[i] = hrow[a * M + i];
-#pragma unroll
-                for (int j = 0; j < M; ++j) {
-                    float acc = 0.f;
-#pragma unroll
-                    for (int i = 0; i < M; ++i) acc = fmaf(x[i], H[i * M + j], acc);
-                    y[j] = acc;
+                for (int i = 0; i < M / 4; ++i) {
+                    const float4 v = gp[i];
+                    x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
                 }
 #pragma unroll
-                for (int j = 0; j < M; ++j) hrow[a * M + j] = y[j];
+                for (int i = 0; i < M; ++i) asm volatile("" : "+f"(x[i]));  // keep the group in registers
+#pragma unroll
+                for (int j = 0; j < M; ++j) y[j] = 0.f;
+#pragma unroll
+                for (int i = 0; i < M; ++i) {
+#pragma unroll
+                    for (int j = 0; j < M; ++j) y[j] = fmaf(x[i], H[i * M + j], y[j]);
+                }
+#pragma unroll
+                for (int i = 0; i < M / 4; ++i) gp[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
             }
             __syncthreads();
         }
