@@ -48,6 +48,23 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
 
 
+# --------------------------------------------------------------------------------------- ranks
+def max_over_ranks(ms: float, device) -> float:
+    """The slowest rank's time: replicas run independently, the job is as fast as its slowest replica."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank processes `tokens_per_rank` tokens per step (weak scaling)."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 # --------------------------------------------------------------------------------------- clocks
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -414,12 +431,9 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop()
     ms_total = t_start.elapsed_time(t_end)
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dev)
     ms_per_step = ms_total / args.steps
-    value = world * T / (ms_per_step * 1e-3)
+    value = job_value(T, world, ms_per_step)
 
     # ---- per-kernel times (this rank), averaged over the timed steps
     kq = {L.name: [] for L in layers}
@@ -537,11 +551,8 @@ def run_ours(args):
         s1 = ev()
         barrier()
         e_ms = s0.elapsed_time(s1)
-        if world > 1:
-            t = torch.tensor([e_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        e2e = {"value": round(world * T / (e_ms / e_steps * 1e-3), 1), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e_ms = max_over_ranks(e_ms, dev)
+        e2e = {"value": round(job_value(T, world, e_ms / e_steps), 1), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": round(e_ms / e_steps, 4), "steps": e_steps}
     st = resq.resq_device_status()
     if st != resq.OK:

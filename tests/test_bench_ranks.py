@@ -1,0 +1,47 @@
+"""The N > 1 path of bench.py on CPU: two gloo ranks, each with its own step time; the job's time is the
+slowest rank's and its throughput counts every rank's tokens (replicas, no data-path collective).  Also:
+the reference arm leaves all work to rank 0."""
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms = bench.max_over_ranks(2.0 + 3.0 * rank, torch.device("cpu"))      # rank 0: 2 ms, rank 1: 5 ms
+    out[rank] = (ms, bench.job_value(4096, world, ms))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_take_the_slowest_time_and_sum_the_tokens():
+    world = 2
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_worker, args=(world, 29500 + os.getpid() % 2000, out), nprocs=world, join=True)
+        res = dict(out)
+    assert res[0][0] == res[1][0] == 5.0
+    assert abs(res[0][1] - 2 * 4096 / 5e-3) < 1e-6
+
+
+def test_single_process_is_identity():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(1.25, torch.device("cpu")) == 1.25
+    assert bench.job_value(4096, 1, 2.0) == 4096 / 2e-3
+
+
+def test_reference_arm_other_ranks_do_no_work():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1"],
+                       env=env, capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0 and r.stdout.strip() == ""
