@@ -262,7 +262,7 @@ def asym_leg(resq, torch, dev, layers, T, steps):
     for L in layers:
         K4 = L.K - L.r
         z = lambda *shape, dt=torch.float32: torch.empty(shape, dtype=dt, device=dev)
-        bufs.append(dict(ws8=None, u8=z(T, L.r, dt=torch.uint8), u4e=z(T, K4, dt=torch.uint8), sx8=z(T), sx4=z(T),
+        bufs.append(dict(ws8=None, Y=torch.empty_like(L.Y), u8=z(T, L.r, dt=torch.uint8), u4e=z(T, K4, dt=torch.uint8), sx8=z(T), sx4=z(T),
                          zx8=z(T), zx4=z(T), wsp=resq.alloc_workspace_asym(L.desc, T, L.online, True, device=dev)))
         bufs[-1]["ws8"], bufs[-1]["ws4"] = resq.resq_weight_row_sums(L.W)
 
@@ -272,7 +272,7 @@ def asym_leg(resq, torch, dev, layers, T, steps):
             resq.resq_project_quantize_asym(L.X, L.P, L.r, b["u8"], None, b["sx8"], b["sx4"], b["zx8"], b["zx4"], b["u4e"],
                                             b["wsp"] if L.online else None)
             e1 = ev() if events is not None else None
-            resq.resq_mixed_gemm_asym(L.W, b["ws8"], b["ws4"], b["u8"], None, b["sx8"], b["sx4"], b["zx8"], b["zx4"], L.Y,
+            resq.resq_mixed_gemm_asym(L.W, b["ws8"], b["ws4"], b["u8"], None, b["sx8"], b["sx4"], b["zx8"], b["zx4"], b["Y"],
                                       b["wsp"], u4_u8=b["u4e"])
             if events is not None:
                 events.append((L, e0, e1, ev()))
@@ -320,12 +320,13 @@ def hadamard_leg(resq, torch, dev, L, T, steps, peaks):
     s8 = torch.empty(T, dtype=torch.float32, device=dev)
     s4 = torch.empty(T, dtype=torch.float32, device=dev)
     ws = resq.alloc_workspace(desc, T, False, True, device=dev)
+    Y = torch.empty_like(L.Y)  # the main leg's outputs stay untouched for the parity spot check
 
     def step(events=None):
         e0 = ev() if events is not None else None
         resq.resq_hadamard_quantize(L.X, 0, None, None, s8, s4, x4e)
         e1 = ev() if events is not None else None
-        resq.resq_mixed_gemm(W, None, None, s8, s4, L.Y, ws, x4_i8=x4e)
+        resq.resq_mixed_gemm(W, None, None, s8, s4, Y, ws, x4_i8=x4e)
         if events is not None:
             events.append((e0, e1, ev()))
 
