@@ -1,0 +1,91 @@
+"""Parity at the full sizes of the Llama-3-8B and Llama-3-70B prefill configurations, in the launch configuration
+the benchmark times (all token rows, whole layers, the tile kernels), checked on sampled token rows that the
+oracle can afford: for those rows everything the layer produces is compared -- codes, scales, the fp32 output
+of every output channel."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from tests.gpu_util import host
+from tests.test_gpu_parity import check_output
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def resq():
+    import paper_2412_14363_b200 as m
+    return m
+
+
+def _bits(t):
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def _sample_rows(T):
+    return np.unique(np.array([0, 1, 127, 128, 255, 256, T // 2 - 1, T // 2, T - 257, T - 129, T - 2, T - 1]))
+
+
+@pytest.mark.parametrize("T,K,N", [
+    (4096, 4096, 28672),    # 8B gate|up: the widest layer of the benchmark
+    (4096, 4096, 6144),     # 8B q|k|v
+    (8192, 8192, 10240),    # 70B q|k|v (8192 + 2 x 1024 output channels)
+    (8192, 8192, 28672),    # 70B gate (one of the two halves; both together are the same kernel, twice the tiles)
+])
+def test_folded_layer_full_size_sampled_rows(resq, T, K, N):
+    r = K // 8
+    dev = torch.device("cuda")
+    X = synth.t_activations(T, K, dev, "t4", seed=21)
+    Wp = synth.t_projected_weights_direct(N, K, dev, seed=22)
+    desc = resq.layer_desc(K, N, r)
+    W = resq.resq_pack_weights(desc, Wp, with_w4_i8=True)
+    pw = oracle.pack_weights(Wp.cpu().numpy(), r)
+    del Wp
+    assert (host(W.w8) == pw.q8).all() and (host(W.w4) == pw.w4_packed).all()
+    assert (host(W.s_w8).view(np.uint32) == pw.s8.view(np.uint32)).all()
+    ws = resq.alloc_workspace(desc, T, False, True)
+    Y = torch.empty((T, N), dtype=torch.float32, device=dev)
+    resq.resq_linear(W, X, None, Y, ws)
+    assert resq.resq_device_status() == resq.OK
+    rows = _sample_rows(T)
+    res = oracle.linear(_bits(X[torch.from_numpy(rows).to(dev)]), None, pw)
+    check_output(res, pw, host(Y[torch.from_numpy(rows).to(dev)]))
+
+
+@pytest.mark.parametrize("T,K,N", [(4096, 14336, 4096), (8192, 28672, 8192)])
+def test_down_proj_full_size_sampled_rows(resq, T, K, N):
+    """down_proj with the online projection at full size: the kernel's codes on the sampled rows lie within +-1 of
+    the oracle's on <= 0.1 %, and its output is exact given its own codes."""
+    r = K // 8
+    K4 = K - r
+    dev = torch.device("cuda")
+    X = synth.t_activations(T, K, dev, "t4", seed=31)
+    P = synth.t_kron_orthogonal_bf16(K, dev)
+    Wp = synth.t_projected_weights_direct(N, K, dev, seed=32)
+    desc = resq.layer_desc(K, N, r)
+    W = resq.resq_pack_weights(desc, Wp, with_w4_i8=True)
+    pw = oracle.pack_weights(Wp.cpu().numpy(), r)
+    del Wp
+    ws = resq.alloc_workspace(desc, T, True, True)
+    x8 = torch.empty((T, r), dtype=torch.int8, device=dev)
+    x4e = torch.empty((T, K4), dtype=torch.int8, device=dev)
+    s8 = torch.empty(T, dtype=torch.float32, device=dev)
+    s4 = torch.empty(T, dtype=torch.float32, device=dev)
+    resq.resq_project_quantize(X, P, r, x8, None, s8, s4, x4e, ws)
+    Y = torch.empty((T, N), dtype=torch.float32, device=dev)
+    resq.resq_mixed_gemm(W, x8, None, s8, s4, Y, ws, x4_i8=x4e)
+    assert resq.resq_device_status() == resq.OK
+    rows = _sample_rows(T)[::3]
+    idx = torch.from_numpy(rows).to(dev)
+    C = oracle.project(_bits(X[idx]), _bits(P))
+    q8, q4, o8, o4 = oracle.split_quantize(C, r)
+    g8, g4 = host(x8[idx]), host(x4e[idx])
+    assert np.abs(g8.astype(np.int32) - q8).max() <= 1 and np.abs(g4.astype(np.int32) - q4).max() <= 1
+    assert ((g8 != q8).sum() + (g4 != q4).sum()) / float(rows.size * K) <= 1e-3
+    gs8, gs4 = host(s8[idx]), host(s4[idx])
+    acc8, acc4 = oracle.int_gemm(g8, pw.q8), oracle.int_gemm(g4, pw.q4)
+    y32, ybf = oracle.epilogue(acc8, acc4, gs8, gs4, pw.s8, pw.s4)
+    res = oracle.LayerResult(None, g8, g4, oracle.pack_nibbles(g4), gs8, gs4, acc8, acc4, y32, ybf)
+    check_output(res, pw, host(Y[idx]))
