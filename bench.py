@@ -228,6 +228,33 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
             step(i)
         t1 = ev()
         torch.cuda.synchronize()
+        # The same GEMV chain with asymmetric activation codes (unsigned codes, zero-points, weight row sums).
+        ab = []
+        for (L, desc, copies), b in zip(sets, bufs):
+            K4 = L.K - L.r
+            z = lambda *shape, dt=torch.float32: torch.empty(shape, dtype=dt, device=dev)
+            a = dict(u8=z(T, L.r, dt=torch.uint8), u4=z(T, K4 // 2, dt=torch.uint8), sx8=z(T), sx4=z(T), zx8=z(T),
+                     zx4=z(T), wsp=resq.alloc_workspace_asym(desc, T, False, False, device=dev))
+            a["ws8"], a["ws4"] = resq.resq_weight_row_sums(copies[0])
+            Xc = b["X"] if not L.online else L.X[:T, :L.K].contiguous()   # codes of raw rows: same cost, no projection
+            resq.resq_project_quantize_asym(Xc, None, L.r, a["u8"], a["u4"], a["sx8"], a["sx4"], a["zx8"], a["zx4"])
+            ab.append(a)
+
+        def asym_chain(i):
+            for (L, desc, copies), b, a in zip(sets, bufs, ab):
+                resq.resq_mixed_gemm_asym(copies[i % DECODE_COPIES], a["ws8"], a["ws4"], a["u8"], a["u4"], a["sx8"],
+                                          a["sx4"], a["zx8"], a["zx4"], b["Y"], a["wsp"])
+
+        for i in range(3):
+            asym_chain(i)
+        torch.cuda.synchronize()
+        torch.cuda._sleep(HOST_LEAD_CYCLES)
+        a0 = ev()
+        for i in range(steps):
+            asym_chain(i)
+        a1 = ev()
+        torch.cuda.synchronize()
+        gemv_asym = a0.elapsed_time(a1) / steps
         gemv = c0.elapsed_time(c1) / steps
         total = t0.elapsed_time(t1) / steps
         gbs = weight_bytes / (gemv * 1e-3) / 1e9
@@ -235,6 +262,8 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
                         "weight_stream_gbs": round(gbs, 1),
                         "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
                         "frac_of_nominal_8000": round(gbs / 8000.0, 4),
+                        "asymmetric_mixed_gemv_us": round(gemv_asym * 1e3, 2),
+                        "asymmetric_weight_stream_gbs": round(weight_bytes / (gemv_asym * 1e-3) / 1e9, 1),
                         "folded_quantize_us": round(quant * 1e3, 2),
                         "online_projection_us": round(proj * 1e3, 2),
                         "online_projection_p_stream_gbs": round(p_bytes / (proj * 1e-3) / 1e9, 1) if proj > 0 else None,

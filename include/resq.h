@@ -121,6 +121,8 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
  * names no construction; K = 8192, 14336 and 28672 are covered.  Other K, or K·4 bytes > 200 KB, give
  * RESQ_ERR_SHAPE.  Outputs as resq_project_quantize (x8 may be NULL when r = 0).  The weights to pair with it are
  * resq_pack_weights of (H_K^T W / sqrt(K))^T.  Every entry point accepts r = 0 (then w8 / x8 may be NULL).
+ * The first call on each device uploads the two small factors to constant memory with a blocking copy: make it
+ * outside any stream capture.
  */
 int resq_hadamard_quantize(const void* X, int T, int K, int r, int8_t* x8, uint8_t* x4, float* s_x8, float* s_x4,
                            int8_t* x4_i8, void* stream);
