@@ -164,6 +164,11 @@ void oracle_epilogue(const int32_t* acc8, const int32_t* acc4, const float* s_x8
  * ==================================================================================================== */
 void oracle_quantize_vector_asym(const float* x, long n, int bits, uint8_t* code, float* s_out, float* z_out) {
     const float qmax = (float)((1 << bits) - 1);
+    if (n == 0) { /* an empty segment (r = 0): nothing to quantize, s = 0 and z = 0 */
+        *s_out = 0.0f;
+        *z_out = 0.0f;
+        return;
+    }
     float lo = x[0], hi = x[0];
     for (long j = 1; j < n; ++j) {
         if (x[j] < lo) lo = x[j];

@@ -142,6 +142,7 @@ split_quantize_asym_kernel(const void* __restrict__ in, size_t in_row_bytes, siz
         }
     }
     if (!live) return;
+    if (rchunks == 0) lo8 = hi8 = 0.f;  // uniform 4-bit layer: the empty INT8 segment has s = 0, z = 0
 
     // ---- scales, zero-points
     const size_t row = row0 + grp;

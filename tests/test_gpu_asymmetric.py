@@ -140,9 +140,10 @@ def test_asym_extreme_codes(resq):
     assert (np.abs(host(y).astype(np.float64) - y32) <= 1e-5 * (np.abs(acc8 * 0.5 * 0.01) + np.abs(acc4 * 2.0 * 0.1) + mag)).all()
 
 
-@pytest.mark.parametrize("T", [5, 200])
-def test_asym_linear_end_to_end(resq, T):
-    K, N, r = 2048, 512, 256
+@pytest.mark.parametrize("T,r", [(5, 256), (200, 256), (3, 0), (130, 0)])
+def test_asym_linear_end_to_end(resq, T, r):
+    """Whole layer; r = 0 is the uniform 4-bit layer (empty INT8 segment: s = 0, z = 0)."""
+    K, N = 2048, 512
     C_bits = _shifted(T, K, 950 + T)
     _, Wp = synthetic_folded(2, K, N, r, seed_shift=3)
     pw = oracle.pack_weights(Wp, r)

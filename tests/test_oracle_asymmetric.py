@@ -118,3 +118,14 @@ def test_asymmetric_beats_symmetric_on_shifted_activations():
     e_asym = np.linalg.norm(oracle.linear_asym_from_coeff(C, pw).y32 - exact)
     e_sym = np.linalg.norm(oracle.linear_from_coeff(C, pw).y32 - exact)
     assert e_asym < e_sym
+
+
+def test_empty_high_precision_segment():
+    """r = 0 (uniform 4-bit): the INT8 segment is empty, its scale and zero-point are 0 and it adds nothing."""
+    rng = np.random.default_rng(9)
+    C = (rng.standard_normal((3, 64)) + 2.0).astype(np.float32)
+    u8, u4, s8, s4, z8, z4 = oracle.split_quantize_asym(C, 0)
+    assert u8.shape == (3, 0) and (s8 == 0).all() and (z8 == 0).all() and (s4 > 0).all()
+    pw = oracle.pack_weights(rng.standard_normal((8, 64)).astype(np.float32), 0)
+    res = oracle.linear_asym_from_coeff(C, pw)
+    assert np.isfinite(res.y32).all() and (res.acc8 == 0).all()
