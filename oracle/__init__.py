@@ -93,6 +93,16 @@ def split_quantize(C, r: int, scale_fp16: bool = False):
     return q8, q4, s8, s4
 
 
+def quantize_rows(X, bits: int):
+    """Uniform-precision symmetric quantizer of Eq. 1 on each row of X [rows][n]: (codes int8, scales fp32 [rows])."""
+    X = _chk(X, np.float32)
+    rows, n = X.shape
+    code = np.empty((rows, n), np.int8)
+    s = np.empty(rows, np.float32)
+    _c().oracle_quantize_rows(_p(X), ctypes.c_long(rows), int(n), int(bits), _p(code), _p(s))
+    return code, s
+
+
 def pack_nibbles(code):
     code = _chk(code, np.int8)
     assert code.shape[-1] % 2 == 0

@@ -86,6 +86,12 @@ void oracle_split_quantize(const float* C, long rows, int K, int r, int scale_fp
     }
 }
 
+/* Uniform-precision form of Eq. 1 on every row of a [rows][n] matrix (one scale per row). */
+void oracle_quantize_rows(const float* x, long rows, int n, int bits, int8_t* code, float* s) {
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < rows; ++t) s[t] = oracle_quantize_vector(x + t * n, n, bits, 0, code + t * n);
+}
+
 /* Canonical nibble packing: byte i holds code 2i in bits 0..3 and code 2i+1 in bits 4..7, two's complement. */
 void oracle_pack_nibbles(const int8_t* code, long n, uint8_t* packed) {
     for (long i = 0; i < n / 2; ++i)
