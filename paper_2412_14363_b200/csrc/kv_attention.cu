@@ -1,0 +1,471 @@
+// Single-query attention over the mixed-precision KV cache (Section 4.3, Eq. 8; Section 5.1).  HBM-bound: every
+// 5632-byte cache block (32 positions of one KV head: key and value codes, scales, zero-points) is read once.
+//
+// Work.  Blocks are numbered in (sequence, KV head, block) order; the 148 x 8 warps of the persistent grid
+// each take an equal contiguous run of that list.  A warp owns a ring of four block-sized stages filled by
+// bulk copies that its lane 0 issues (one copy per block, completion on the warp's own mbarriers), so no
+// CTA-wide barrier exists after start-up.  Whenever the run leaves a (sequence, head) the warp writes one
+// partial record (running maximum, sum of weights, unnormalised output) for the query heads of that KV head;
+// a second small kernel merges the records of each (sequence, query head).
+//
+// Arithmetic.  The codes never become dequantized values.  With q8/q4 the two segments of a query head,
+//     q . k_hat = s8 (q8 . c8) + z8 sum(q8) + s4 (q4 . c4) + z4 sum(q4),
+//     sum_j p_j v_hat_j = sum_j (p_j s_j) c_j + sum_j p_j z_j          (per segment),
+// so both products contract fp16 queries / weights with integer codes on mma.sync m16n8k16 (codes are exact
+// in half: 1024 + c and 64 + c are built with one logic op on the packed bytes or nibbles and the offset is
+// subtracted exactly).  Positions are the M rows of the score product (8 query heads of a group as N) and the
+// K rows of the output product (16 coefficients as M), so the score accumulators only need an 8x8 transpose
+// (movmatrix) to become the second product's B fragments.  Scores, the running softmax and all sums are
+// fp32; the weights p_j s_j are scaled by a power of two taken from the value scales so that they stay in
+// half's range whatever the magnitude of V.
+#include <cuda_fp16.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+#include "../../include/resq_kv.h"
+
+namespace resq {
+namespace {
+
+constexpr int kD = 128;
+constexpr int kWarps = 8;
+constexpr int kStages = 4;
+constexpr int kBlk = RESQ_KV_BLOCK_BYTES;
+constexpr int kOffK8 = 0, kOffK4 = 512, kOffKM = 2304, kOffV8 = 2816, kOffV4 = 3328, kOffVM = 5120;
+constexpr int kRecFloats = 8 * (kD + 2);  // per query head of the group: m, l, 128 outputs
+constexpr float kLog2eOverSqrtD = 0.12751743f;  // log2(e) / sqrt(128)
+
+struct AttnParams {
+    const uint8_t* cache;
+    const __half* q;
+    const int32_t* seq_lens;
+    float* partial;
+    float* out;
+    int* status;
+    int n_seqs, n_kv_heads, group, capacity, n_warps_total;
+};
+
+__device__ __forceinline__ int clamped_len(const int32_t* seq_lens, int b, int capacity) {
+    const int len = seq_lens[b];
+    return len < 0 ? 0 : (len > capacity ? capacity : len);
+}
+
+// Whole warp: returns the number of blocks per head summed over all sequences.  If target >= 0, also finds the
+// sequence that holds global block `target` (the list has n_kv_heads times the per-head blocks of each
+// sequence) and the per-head blocks of all sequences before it.
+__device__ __forceinline__ long long scan_blocks(const AttnParams& p, int lane, long long target, int* b_out,
+                                                 long long* before_out) {
+    long long base = 0;
+    bool found = false;
+    for (int b0 = 0; b0 < p.n_seqs; b0 += 32) {
+        const int b = b0 + lane;
+        const int t = b < p.n_seqs ? (clamped_len(p.seq_lens, b, p.capacity) + 31) >> 5 : 0;
+        int incl = t;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (target >= 0 && !found) {
+            const unsigned m = __ballot_sync(0xffffffffu, (base + incl) * p.n_kv_heads > target);
+            if (m) {
+                const int l = __ffs(m) - 1;
+                *b_out = b0 + l;
+                *before_out = base + __shfl_sync(0xffffffffu, incl - t, l);
+                found = true;
+            }
+        }
+        base += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    return base;
+}
+
+struct Cursor {  // one block of the global list
+    int b, h, blk, nblk, len;
+};
+__device__ __forceinline__ void advance(Cursor& cu, const AttnParams& p) {
+    if (++cu.blk < cu.nblk) return;
+    cu.blk = 0;
+    if (++cu.h < p.n_kv_heads) return;
+    cu.h = 0;
+    do {
+        if (++cu.b >= p.n_seqs) { cu.nblk = 0; cu.len = 0; return; }
+        cu.len = clamped_len(p.seq_lens, cu.b, p.capacity);
+        cu.nblk = (cu.len + 31) >> 5;
+    } while (cu.nblk == 0);
+}
+
+__device__ __forceinline__ uint32_t sub_h2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("sub.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// Two codes held in bits 0-3 / 16-19 (lo) or 4-7 / 20-23 (hi) of w as an exact half2.
+__device__ __forceinline__ uint32_t nib_lo(uint32_t w) { return sub_h2((w & 0x000F000Fu) | 0x64006400u, 0x64006400u); }
+__device__ __forceinline__ uint32_t nib_hi(uint32_t w) { return sub_h2((w & 0x00F000F0u) | 0x54005400u, 0x54005400u); }
+// Two bytes of w (picked by SEL, with 0x64 as the upper byte of each half) as an exact half2.
+template <uint32_t SEL>
+__device__ __forceinline__ uint32_t bytes_h2(uint32_t w) { return sub_h2(__byte_perm(w, 0x64646464u, SEL), 0x64006400u); }
+
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(x));
+    return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ uint32_t lds32(const uint8_t* p) { return *reinterpret_cast<const uint32_t*>(p); }
+__device__ __forceinline__ uint32_t lds16(const uint8_t* p) { return *reinterpret_cast<const uint16_t*>(p); }
+
+// Coefficient index behind entry e (k = 2c, 2c + 1, 2c + 8, 2c + 9) of contraction step j of the score product,
+// as the key-side extraction delivers them: step 0 is the 8-bit segment (bytes 4c..4c+3 of the position's 16),
+// steps 1-6 take two steps per 32-bit word c + 4i of the 4-bit codes (nibbles (0,4),(1,5) then (2,6),(3,7)),
+// step 7 the nibbles (0,2),(1,3) of half-word 24 + c.
+__device__ __forceinline__ int kdim(int j, int c, int e) {
+    if (j == 0) return 4 * c + e;
+    if (j == 7) return 112 + 4 * c + ((e & 1) << 1) + (e >> 1);
+    const int i = (j - 1) >> 1, sub = (j - 1) & 1;
+    return 16 + 8 * (c + 4 * i) + 2 * sub + ((e & 1) << 2) + (e >> 1);
+}
+
+struct ValueScale {  // per position: scales times 2^-E, zero-points, 2^-E, E (E from the larger value scale)
+    float sn8, sn4, z8, z4, i2e, e;
+};
+__device__ __forceinline__ ValueScale value_scale(const uint8_t* vm, int tok, bool valid) {
+    const float4 m = *reinterpret_cast<const float4*>(vm + tok * 16);
+    uint32_t eb = __float_as_uint(fmaxf(m.x, m.z)) & 0x7F800000u;
+    eb = min(max(eb, 63u << 23), 191u << 23);  // 2^-64 .. 2^64
+    ValueScale v;
+    v.i2e = __uint_as_float((254u << 23) - eb);
+    v.e = static_cast<float>(static_cast<int>(eb >> 23) - 127);
+    v.sn8 = valid ? m.x * v.i2e : 0.f;
+    v.sn4 = valid ? m.z * v.i2e : 0.f;
+    v.z8 = valid ? m.y : 0.f;
+    v.z4 = valid ? m.w : 0.f;
+    return v;
+}
+
+__global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const AttnParams p) {
+    extern __shared__ __align__(128) uint8_t rings[];
+    __shared__ uint64_t full_s[kWarps][kStages];
+    __shared__ int abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+    uint8_t* ring = rings + static_cast<size_t>(warp) * kStages * kBlk;
+    uint64_t* full = full_s[warp];
+    if (lane == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(&full[s], 1);
+        fence_mbar_init();
+    }
+    if (threadIdx.x == 0) abort_flag = 0;
+    __syncthreads();
+
+    // ---- this warp's run of the global block list
+    const long long wg = static_cast<long long>(blockIdx.x) * kWarps + warp;
+    int b_first = 0;
+    long long before = 0;
+    const long long total = scan_blocks(p, lane, -1, &b_first, &before) * p.n_kv_heads;
+    const long long start = total * wg / p.n_warps_total, end = total * (wg + 1) / p.n_warps_total, n = end - start;
+    if (n <= 0) return;
+    scan_blocks(p, lane, start, &b_first, &before);
+    Cursor cons;
+    cons.b = b_first;
+    cons.len = clamped_len(p.seq_lens, b_first, p.capacity);
+    cons.nblk = (cons.len + 31) >> 5;
+    {
+        const long long local = start - before * p.n_kv_heads;
+        cons.h = static_cast<int>(local / cons.nblk);
+        cons.blk = static_cast<int>(local - static_cast<long long>(cons.h) * cons.nblk);
+    }
+    Cursor prod = cons;
+    const int blocks_cap = p.capacity / RESQ_KV_BLOCK;
+    auto issue = [&](int stage) {  // lane 0 copies the producer cursor's block; every lane moves the cursor
+        if (lane == 0) {
+            const uint8_t* src = p.cache + ((static_cast<long long>(prod.b) * p.n_kv_heads + prod.h) * blocks_cap + prod.blk) * kBlk;
+            mbar_arrive_expect_tx(&full[stage], kBlk);
+            bulk_load(ring + stage * kBlk, src, kBlk, &full[stage]);
+        }
+        advance(prod, p);
+    };
+    long long issued = 0;
+    for (; issued < n && issued < kStages; ++issued) issue(static_cast<int>(issued));
+
+    uint32_t qf[8][2];
+    float kq8[2], kq4[2], m_run[2], l[2], z8[2], z4[2], acc[8][4];
+    bool fresh = true, ok = true;
+    long long i = 0;
+    for (; i < n; ++i) {
+        const int stage = static_cast<int>(i % kStages);
+        const uint32_t phase = static_cast<uint32_t>(i / kStages) & 1u;
+        if (fresh) {  // a new (sequence, KV head): query fragments of its group, empty running state
+            fresh = false;
+            const __half* qrow = p.q + (static_cast<long long>(cons.b) * p.n_kv_heads * p.group + cons.h * p.group + g) * kD;
+            float s8 = 0.f, s4 = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    __half2 v = __floats2half2_rn(0.f, 0.f);
+                    if (g < p.group) v = __halves2half2(qrow[kdim(j, c, 2 * hf)], qrow[kdim(j, c, 2 * hf + 1)]);
+                    qf[j][hf] = *reinterpret_cast<const uint32_t*>(&v);
+                    const float2 f = __half22float2(v);
+                    if (j == 0) s8 += f.x + f.y; else s4 += f.x + f.y;
+                }
+            s8 += __shfl_xor_sync(0xffffffffu, s8, 1); s8 += __shfl_xor_sync(0xffffffffu, s8, 2);
+            s4 += __shfl_xor_sync(0xffffffffu, s4, 1); s4 += __shfl_xor_sync(0xffffffffu, s4, 2);
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {  // the score fragment's columns are heads 2c, 2c + 1
+                kq8[e] = kLog2eOverSqrtD * __shfl_sync(0xffffffffu, s8, 4 * (2 * c + e));
+                kq4[e] = kLog2eOverSqrtD * __shfl_sync(0xffffffffu, s4, 4 * (2 * c + e));
+                m_run[e] = -INFINITY; l[e] = z8[e] = z4[e] = 0.f;
+            }
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
+        }
+        if (!mbar_wait(&full[stage], phase, &abort_flag)) { ok = false; break; }
+        const uint8_t* st = ring + stage * kBlk;
+        const int valid = min(RESQ_KV_BLOCK, cons.len - RESQ_KV_BLOCK * cons.blk);
+
+        // ---- scores of the 32 positions (two 16-row products), in log2 units, plus the value-scale exponent
+        float sc[2][4];
+        ValueScale vs[2][2];
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            const int tokA = 16 * m + 2 * g, tokB = tokA + 1;  // rows g and g + 8 of the product
+            float d8[4] = {0.f, 0.f, 0.f, 0.f}, d4[4] = {0.f, 0.f, 0.f, 0.f};
+            {
+                const uint32_t wa = lds32(st + kOffK8 + tokA * 16 + 4 * c), wb = lds32(st + kOffK8 + tokB * 16 + 4 * c);
+                mma_f16(d8, bytes_h2<0x4140>(wa), bytes_h2<0x4140>(wb), bytes_h2<0x4342>(wa), bytes_h2<0x4342>(wb),
+                        qf[0][0], qf[0][1]);
+            }
+#pragma unroll
+            for (int i3 = 0; i3 < 3; ++i3) {
+                uint32_t wa = lds32(st + kOffK4 + tokA * 56 + 4 * (c + 4 * i3)), wb = lds32(st + kOffK4 + tokB * 56 + 4 * (c + 4 * i3));
+                mma_f16(d4, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[1 + 2 * i3][0], qf[1 + 2 * i3][1]);
+                wa >>= 8; wb >>= 8;
+                mma_f16(d4, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[2 + 2 * i3][0], qf[2 + 2 * i3][1]);
+            }
+            {
+                uint32_t xa = lds16(st + kOffK4 + tokA * 56 + 48 + 2 * c), xb = lds16(st + kOffK4 + tokB * 56 + 48 + 2 * c);
+                xa |= xa << 8; xb |= xb << 8;
+                mma_f16(d4, nib_lo(xa), nib_lo(xb), nib_hi(xa), nib_hi(xb), qf[7][0], qf[7][1]);
+            }
+            const float4 kmA = *reinterpret_cast<const float4*>(st + kOffKM + tokA * 16);
+            const float4 kmB = *reinterpret_cast<const float4*>(st + kOffKM + tokB * 16);
+            const bool vA = tokA < valid, vB = tokB < valid;
+            vs[m][0] = value_scale(st + kOffVM, tokA, vA);
+            vs[m][1] = value_scale(st + kOffVM, tokB, vB);
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const float sA = kLog2eOverSqrtD * (kmA.x * d8[e] + kmA.z * d4[e]) + kmA.y * kq8[e] + kmA.w * kq4[e] + vs[m][0].e;
+                const float sB = kLog2eOverSqrtD * (kmB.x * d8[2 + e] + kmB.z * d4[2 + e]) + kmB.y * kq8[e] + kmB.w * kq4[e] + vs[m][1].e;
+                sc[m][e] = vA ? sA : -INFINITY;
+                sc[m][2 + e] = vB ? sB : -INFINITY;
+            }
+        }
+        // ---- running maximum per head (columns 2c, 2c + 1), shared by the 8 lanes with this c
+        float mn[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            float mx = fmaxf(fmaxf(sc[0][e], sc[0][2 + e]), fmaxf(sc[1][e], sc[1][2 + e]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            mn[e] = fmaxf(m_run[e], mx);
+        }
+        if (__any_sync(0xffffffffu, mn[0] != m_run[0] || mn[1] != m_run[1])) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const float a = ex2(m_run[e] - mn[e]);
+                l[e] *= a; z8[e] *= a; z4[e] *= a;
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) { acc[mt][e] *= a; acc[mt][2 + e] *= a; }
+                m_run[e] = mn[e];
+            }
+        }
+        // ---- weights, their transposes as B fragments, and the output products
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            float p8[2][2], p4[2][2];
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const ValueScale& v = vs[m][t];
+                    const float pw = ex2(sc[m][2 * t + e] - m_run[e]);
+                    const float w = pw * v.i2e;
+                    l[e] += w; z8[e] = fmaf(w, v.z8, z8[e]); z4[e] = fmaf(w, v.z4, z4[e]);
+                    p8[t][e] = pw * v.sn8; p4[t][e] = pw * v.sn4;
+                }
+            const uint32_t b80 = movmatrix_trans(pack_h2(p8[0][0], p8[0][1])), b81 = movmatrix_trans(pack_h2(p8[1][0], p8[1][1]));
+            const uint32_t b40 = movmatrix_trans(pack_h2(p4[0][0], p4[0][1])), b41 = movmatrix_trans(pack_h2(p4[1][0], p4[1][1]));
+            const int t0 = 16 * m + 4 * c;  // contraction entries 2c, 2c+1, 2c+8, 2c+9 are positions t0, t0+2, t0+1, t0+3
+            {
+                const uint8_t* v8 = st + kOffV8 + t0 * 16 + 2 * g;
+                const uint32_t w02 = lds16(v8) | (lds16(v8 + 32) << 16), w13 = lds16(v8 + 16) | (lds16(v8 + 48) << 16);
+                mma_f16(acc[0], bytes_h2<0x4240>(w02), bytes_h2<0x4341>(w02), bytes_h2<0x4240>(w13), bytes_h2<0x4341>(w13), b80, b81);
+            }
+#pragma unroll
+            for (int i3 = 0; i3 < 3; ++i3) {
+                const uint8_t* v4 = st + kOffV4 + t0 * 56 + 2 * (g + 8 * i3);
+                uint32_t w02 = lds16(v4) | (lds16(v4 + 112) << 16), w13 = lds16(v4 + 56) | (lds16(v4 + 168) << 16);
+                mma_f16(acc[1 + 2 * i3], nib_lo(w02), nib_hi(w02), nib_lo(w13), nib_hi(w13), b40, b41);
+                w02 >>= 8; w13 >>= 8;
+                mma_f16(acc[2 + 2 * i3], nib_lo(w02), nib_hi(w02), nib_lo(w13), nib_hi(w13), b40, b41);
+            }
+            {
+                const uint8_t* v4 = st + kOffV4 + t0 * 56 + 48 + g;
+                const uint32_t w02 = v4[0] | (static_cast<uint32_t>(v4[112]) << 16), w13 = v4[56] | (static_cast<uint32_t>(v4[168]) << 16);
+                mma_f16(acc[7], nib_lo(w02), nib_hi(w02), nib_lo(w13), nib_hi(w13), b40, b41);
+            }
+        }
+        __syncwarp();
+        if (issued < n) {  // refill the stage just read
+            issue(stage);
+            ++issued;
+        }
+        // ---- leaving this (sequence, head), or the run: one partial record
+        if (cons.blk == cons.nblk - 1 || i == n - 1) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1) {
+                    l[e] += __shfl_xor_sync(0xffffffffu, l[e], o);
+                    z8[e] += __shfl_xor_sync(0xffffffffu, z8[e], o);
+                    z4[e] += __shfl_xor_sync(0xffffffffu, z4[e], o);
+                }
+            float* rec = p.partial + (wg + static_cast<long long>(cons.b) * p.n_kv_heads + cons.h) * kRecFloats;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                if (2 * c + e >= p.group) continue;
+                float* r = rec + (2 * c + e) * (kD + 2);
+                if (g == 0) { r[0] = m_run[e]; r[1] = l[e]; }
+                r += 2;
+                r[2 * g] = acc[0][e] + z8[e];
+                r[2 * g + 1] = acc[0][2 + e] + z8[e];
+#pragma unroll
+                for (int i3 = 0; i3 < 3; ++i3) {
+                    const int d0 = 16 + 4 * (g + 8 * i3);
+                    r[d0] = acc[1 + 2 * i3][e] + z4[e];
+                    r[d0 + 1] = acc[1 + 2 * i3][2 + e] + z4[e];
+                    r[d0 + 2] = acc[2 + 2 * i3][e] + z4[e];
+                    r[d0 + 3] = acc[2 + 2 * i3][2 + e] + z4[e];
+                }
+                r[112 + 2 * g] = acc[7][e] + z4[e];
+                r[113 + 2 * g] = acc[7][2 + e] + z4[e];
+            }
+            fresh = true;
+        }
+        advance(cons, p);
+    }
+    if (!ok) {  // a wait ran out: let this warp's copies in flight land (bounded), then report
+        for (long long k = i; k < issued; ++k) {
+            const int stage = static_cast<int>(k % kStages);
+            const uint32_t phase = static_cast<uint32_t>(k / kStages) & 1u;
+            for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&full[stage], phase); ++spin) {}
+        }
+        if (lane == 0) atomicOr(p.status, RESQ_ERR_TIMEOUT);
+    }
+}
+
+// Merges the partial records of one (sequence, query head): out = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i.
+// The warps that hold a record of this (sequence, KV head) are those whose runs meet its range of the block list.
+__global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams p) {
+    __shared__ long long red[2][kD / 32];
+    const int n_q_heads = p.n_kv_heads * p.group;
+    const int b = blockIdx.x / n_q_heads, hq = blockIdx.x - b * n_q_heads;
+    const int hk = hq / p.group, hg = hq - hk * p.group, d = threadIdx.x;
+    long long before = 0, total = 0;
+    for (int i = d; i < p.n_seqs; i += kD) {
+        const int len = p.seq_lens[i];
+        if (hq == 0 && b == 0 && (len < 0 || len > p.capacity)) atomicOr(p.status, RESQ_ERR_INDEX);
+        const int t = (clamped_len(p.seq_lens, i, p.capacity) + 31) >> 5;
+        total += t;
+        if (i < b) before += t;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        before += __shfl_xor_sync(0xffffffffu, before, o);
+        total += __shfl_xor_sync(0xffffffffu, total, o);
+    }
+    if ((d & 31) == 0) { red[0][d >> 5] = before; red[1][d >> 5] = total; }
+    __syncthreads();
+    before = red[0][0] + red[0][1] + red[0][2] + red[0][3];
+    total = (red[1][0] + red[1][1] + red[1][2] + red[1][3]) * p.n_kv_heads;
+    float* out = p.out + (static_cast<long long>(b) * n_q_heads + hq) * kD;
+    const int nblk = (clamped_len(p.seq_lens, b, p.capacity) + 31) >> 5;
+    if (nblk == 0) {  // empty sequence
+        out[d] = 0.f;
+        return;
+    }
+    const long long lo = before * p.n_kv_heads + static_cast<long long>(hk) * nblk, hi = lo + nblk;  // [lo, hi)
+    const long long nw = p.n_warps_total;
+    const long long w_first = ((lo + 1) * nw - 1) / total, w_last = (hi * nw - 1) / total;
+    const long long s = static_cast<long long>(b) * p.n_kv_heads + hk;
+    float M = -INFINITY;
+    for (long long w = w_first; w <= w_last; ++w) {
+        const long long rs = total * w / nw, re = total * (w + 1) / nw;
+        if (re <= rs || re <= lo || rs >= hi) continue;  // empty run, or no block of this range
+        M = fmaxf(M, p.partial[(w + s) * kRecFloats + hg * (kD + 2)]);
+    }
+    float num = 0.f, den = 0.f;
+    for (long long w = w_first; w <= w_last; ++w) {
+        const long long rs = total * w / nw, re = total * (w + 1) / nw;
+        if (re <= rs || re <= lo || rs >= hi) continue;
+        const float* r = p.partial + (w + s) * kRecFloats + hg * (kD + 2);
+        const float f = ex2(r[0] - M);
+        den = fmaf(f, r[1], den);
+        num = fmaf(f, r[2 + d], num);
+    }
+    out[d] = num / den;
+}
+
+}  // namespace
+
+size_t attention_scratch_bytes(int n_seqs, int n_kv_heads) {
+    return (static_cast<size_t>(148) * kWarps + static_cast<size_t>(n_seqs) * n_kv_heads) * kRecFloats * sizeof(float);
+}
+
+cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q16, int n_q_heads, const int32_t* seq_lens,
+                                    float* out, void* scratch, cudaStream_t st) {
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaError_t e = cudaGetDevice(&dev); e != cudaSuccess) return e;
+    constexpr int kSmem = kWarps * kStages * kBlk;
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        if (cudaError_t e = cudaFuncSetAttribute(attention_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+            e != cudaSuccess)
+            return e;
+        configured[dev] = true;
+    }
+    AttnParams p{};
+    p.cache = static_cast<const uint8_t*>(cache.data);
+    p.q = static_cast<const __half*>(q16);
+    p.seq_lens = seq_lens;
+    p.partial = static_cast<float*>(scratch);
+    p.out = out;
+    p.status = device_status_ptr();
+    p.n_seqs = cache.n_seqs;
+    p.n_kv_heads = cache.n_kv_heads;
+    p.group = n_q_heads / cache.n_kv_heads;
+    p.capacity = cache.capacity;
+    p.n_warps_total = 148 * kWarps;
+    attention_decode_kernel<<<148, kWarps * 32, kSmem, st>>>(p);
+    if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
+    attention_combine_kernel<<<cache.n_seqs * n_q_heads, kD, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace resq
