@@ -51,7 +51,9 @@ typedef enum resq_status {
     RESQ_ERR_WORKSPACE = 4,  /* workspace missing or smaller than resq_workspace_bytes() */
     RESQ_ERR_ARCH = 5,       /* current device is not compute capability 10.x */
     RESQ_ERR_CUDA = 6,       /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
-    RESQ_ERR_TIMEOUT = 7     /* reported by resq_device_status: a bounded device wait ran out */
+    RESQ_ERR_TIMEOUT = 7,    /* reported by resq_device_status: a bounded device wait ran out */
+    RESQ_ERR_INDEX = 8       /* reported by resq_device_status: an index read on the device (cache slot, sequence
+                                length) was out of range; the element was skipped or clamped (resq_kv.h) */
 } resq_status_t;
 
 /* Weight-scale storage type. */
@@ -238,7 +240,8 @@ int resq_set_option(int option, int value);
 int resq_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t cols, void* stream);
 
 /* Synchronizes `stream`, then reads and clears the device status word of the current device:
- * RESQ_OK, RESQ_ERR_TIMEOUT, or RESQ_ERR_CUDA if the stream reported an error. */
+ * RESQ_OK, RESQ_ERR_TIMEOUT, RESQ_ERR_INDEX (a timeout wins if both happened), or RESQ_ERR_CUDA if the stream
+ * reported an error. */
 int resq_device_status(void* stream);
 
 /* The CUDA runtime's description of the error behind the latest RESQ_ERR_CUDA that any entry point of

@@ -10,7 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libresq.so")
-SOURCES = ["api.cu", "quantize.cu", "quantize_asym.cu", "mixed_gemm.cu", "decode.cu", "decode_stream.cu", "project.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "quantize.cu", "quantize_asym.cu", "mixed_gemm.cu", "decode.cu", "decode_stream.cu", "project.cu", "static_scratch.cu",
+           "kv_cache.cu", "kv_attention.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -426,9 +426,69 @@ int resq_device_status(void* stream) {
     if (v != 0) {
         int zero = 0;
         cudaMemcpy(p, &zero, sizeof(int), cudaMemcpyHostToDevice);
-        return RESQ_ERR_TIMEOUT;
+        return (v & RESQ_ERR_TIMEOUT) ? RESQ_ERR_TIMEOUT : RESQ_ERR_INDEX;  // kernels OR 7 or 8 into the word
     }
     return RESQ_OK;
+}
+
+// ---- attention-block path (resq_kv.h) ----
+size_t resq_kv_cache_bytes(int n_seqs, int n_kv_heads, int d_head, int capacity) {
+    if (n_seqs < 1 || n_kv_heads < 1 || d_head != 128 || capacity < RESQ_KV_BLOCK || capacity % RESQ_KV_BLOCK != 0) return 0;
+    return static_cast<size_t>(n_seqs) * n_kv_heads * (capacity / RESQ_KV_BLOCK) * RESQ_KV_BLOCK_BYTES;
+}
+
+static int check_cache(const resq_kv_cache_t* c) {
+    if (!c) return RESQ_ERR_NULL;
+    if (resq_kv_cache_bytes(c->n_seqs, c->n_kv_heads, c->d_head, c->capacity) == 0) return RESQ_ERR_SHAPE;
+    if (!c->data) return RESQ_ERR_NULL;
+    return aligned16(c->data) ? RESQ_OK : RESQ_ERR_ALIGN;
+}
+
+int resq_uc_quantize(const float* W_C, int d_head, int8_t* wq, float* s_u, void* stream) {
+    if (d_head != 128) return RESQ_ERR_SHAPE;
+    if (!W_C || !wq || !s_u) return RESQ_ERR_NULL;
+    if (!aligned16(W_C) || !aligned16(wq) || !aligned16(s_u)) return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_uc_quantize(W_C, wq, s_u, static_cast<cudaStream_t>(stream)));
+}
+
+int resq_query_project(const void* q, int64_t rows, int d_head, const int8_t* wq, const float* s_u, void* q_out,
+                       void* stream) {
+    if (d_head != 128 || rows < 0) return RESQ_ERR_SHAPE;
+    if (!q || !wq || !s_u || !q_out) return RESQ_ERR_NULL;
+    if (!aligned16(q) || !aligned16(wq) || !aligned16(s_u) || !aligned16(q_out)) return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_query_project(q, rows, wq, s_u, q_out, static_cast<cudaStream_t>(stream)));
+}
+
+int resq_kv_append(const resq_kv_cache_t* cache, const void* k, const void* v, int64_t T, const int32_t* seq_ids,
+                   const int32_t* positions, const int8_t* wq, const float* s_u, void* stream) {
+    if (int e = check_cache(cache)) return e;
+    if (T < 0) return RESQ_ERR_SHAPE;
+    if (!k || !v || !seq_ids || !positions || !wq || !s_u) return RESQ_ERR_NULL;
+    if (!aligned16(k) || !aligned16(v) || !aligned16(wq) || !aligned16(s_u)) return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_kv_append(*cache, k, v, T, seq_ids, positions, wq, s_u, static_cast<cudaStream_t>(stream)));
+}
+
+size_t resq_attention_workspace_bytes(int n_seqs, int n_q_heads, int n_kv_heads, int d_head) {
+    if (n_seqs < 1 || n_kv_heads < 1 || d_head != 128 || n_q_heads < n_kv_heads || n_q_heads % n_kv_heads != 0 ||
+        n_q_heads / n_kv_heads > 8)
+        return 0;
+    return attention_scratch_bytes(n_seqs, n_kv_heads);
+}
+
+int resq_attention_decode(const resq_kv_cache_t* cache, const void* q16, int n_q_heads, const int32_t* seq_lens,
+                          float* out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (int e = check_cache(cache)) return e;
+    const size_t need = resq_attention_workspace_bytes(cache->n_seqs, n_q_heads, cache->n_kv_heads, cache->d_head);
+    if (need == 0) return RESQ_ERR_SHAPE;
+    if (!q16 || !seq_lens || !out) return RESQ_ERR_NULL;
+    if (!workspace || workspace_bytes < need) return RESQ_ERR_WORKSPACE;
+    if (!aligned16(q16) || !aligned16(out) || !aligned16(workspace)) return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_attention_decode(*cache, q16, n_q_heads, seq_lens, out, workspace,
+                                               static_cast<cudaStream_t>(stream)));
 }
 
 const char* resq_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
@@ -443,6 +503,7 @@ const char* resq_status_string(int s) {
         case RESQ_ERR_ARCH: return "device is not compute capability 10.x";
         case RESQ_ERR_CUDA: return "CUDA call failed";
         case RESQ_ERR_TIMEOUT: return "bounded device wait ran out";
+        case RESQ_ERR_INDEX: return "device-side index out of range";
         default: return "unknown status";
     }
 }

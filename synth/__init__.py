@@ -159,6 +159,26 @@ def kron_orthogonal_bf16(K: int, seed: int = SEED_P, inner: int = 128) -> np.nda
     return out
 
 
+SEED_ATTN = 7
+
+
+def haar_orthogonal(n: int, seed: int = SEED_ATTN, stream: int = 0) -> np.ndarray:
+    """n x n Haar-distributed orthogonal matrix (sign-fixed Q of a seeded Gaussian matrix), float64: a stand-in
+    for a per-layer head basis such as U_C, which the method obtains from calibration data that is not here."""
+    q, rr = np.linalg.qr(gaussian_matrix(n, seed, stream))
+    return q * np.sign(np.diag(rr))
+
+
+def head_vectors(T: int, H: int, d: int, seed: int = SEED_ATTN, stream: int = 1, lead: float = 4.0,
+                 scale: float = 1.0, shift: float = 0.0) -> np.ndarray:
+    """bf16-valued float32 [T][H][d] head vectors: iid N(0, 1) entries times `scale`, the first d/8 coefficients
+    of every head `lead` times larger (a basis ordered by variance puts its high-variance coefficients
+    first), plus `shift`."""
+    x = normal(seed, stream, T * H * d).reshape(T, H, d) * scale
+    x[:, :, : d // 8] *= lead
+    return to_bf16_values((x + shift).astype(np.float32))
+
+
 # ----------------------------------------------------------------------------
 # The same counter-based streams on a torch device, for full-size workloads (hundreds of millions
 # of draws).  The integer stream is identical to the numpy one; log/cos may differ in the last ulp.

@@ -17,8 +17,8 @@ def resq():
     return m
 
 
-def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "resq.h")).read()
+def _declared_functions(header="resq.h"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(resq_[a-z0-9_]+)\s*\(", text)))
 
@@ -29,6 +29,45 @@ def test_library_exports_every_declared_symbol(resq):
     for n in names:
         assert hasattr(resq.lib, n), n
     assert sorted(resq.EXPORTS) == names
+
+
+def test_every_header_is_covered():
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["resq.h", "resq_kv.h"]
+
+
+def test_library_exports_every_kv_symbol(resq):
+    from paper_2412_14363_b200 import kv
+    names = _declared_functions("resq_kv.h")
+    assert "resq_attention_decode" in names and "resq_kv_append" in names
+    for n in names:
+        assert hasattr(resq.lib, n), n
+    assert sorted(kv.KV_EXPORTS) == names
+
+
+def test_kv_host_validation(resq):
+    """Geometry, NULL and alignment checks of the attention-block entry points (nothing is launched)."""
+    import ctypes
+    from paper_2412_14363_b200 import kv
+    L = resq.lib
+    assert L.resq_kv_cache_bytes(2, 8, 128, 64) == 2 * 8 * 2 * 5632
+    assert L.resq_kv_cache_bytes(2, 8, 64, 64) == 0 and L.resq_kv_cache_bytes(2, 8, 128, 48) == 0
+    assert L.resq_kv_cache_bytes(0, 8, 128, 64) == 0
+    assert L.resq_attention_workspace_bytes(4, 32, 8, 128) > 0
+    assert L.resq_attention_workspace_bytes(4, 30, 8, 128) == 0      # not a multiple of the KV heads
+    assert L.resq_attention_workspace_bytes(4, 72, 8, 128) == 0      # more than 8 query heads per KV head
+    fake = 1 << 20
+    c = kv.KvCacheStruct(2, 8, 128, 64, fake)
+    assert L.resq_uc_quantize(fake, 64, fake, fake, None) == resq.ERR_SHAPE
+    assert L.resq_uc_quantize(None, 128, fake, fake, None) == resq.ERR_NULL
+    assert L.resq_query_project(fake, 5, 128, fake, fake + 4, fake, None) == resq.ERR_ALIGN
+    assert L.resq_query_project(fake, -1, 128, fake, fake, fake, None) == resq.ERR_SHAPE
+    assert L.resq_kv_append(None, fake, fake, 1, fake, fake, fake, fake, None) == resq.ERR_NULL
+    assert L.resq_kv_append(ctypes.byref(c), fake, None, 1, fake, fake, fake, fake, None) == resq.ERR_NULL
+    bad = kv.KvCacheStruct(2, 8, 128, 40, fake)
+    assert L.resq_kv_append(ctypes.byref(bad), fake, fake, 1, fake, fake, fake, fake, None) == resq.ERR_SHAPE
+    assert L.resq_attention_decode(ctypes.byref(c), fake, 32, fake, fake, fake, 16, None) == resq.ERR_WORKSPACE
+    assert L.resq_attention_decode(ctypes.byref(c), fake, 12, fake, fake, fake, 1 << 30, None) == resq.ERR_SHAPE
+    assert "index" in resq.status_string(kv.ERR_INDEX)
 
 
 def test_status_strings(resq):
