@@ -379,6 +379,86 @@ def hadamard_leg(resq, torch, dev, L, T, steps, peaks):
             "layer_ms": round(q + g, 4)}
 
 
+# --------------------------------------------------------------------------------------- attention-block leg
+KV_HQ, KV_HKV, KV_D = 32, 8, 128   # Llama-3-8B attention geometry
+
+
+def kv_leg(resq, torch, dev, peaks, steps, n_seqs=16, seq_len=8192, prefill_T=4096):
+    """The attention-block path (Section 4.3, Eq. 8; Section 5.1): 8-bit U_C projection of query and key, the
+    per-head 8/4-bit KV cache, and single-query attention over it for `n_seqs` sequences of `seq_len` cached
+    positions.  Two cache copies (each larger than L2) are cycled so that every timed byte comes from DRAM."""
+    import numpy as np
+    import synth
+    from paper_2412_14363_b200 import kv
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    def timed(fn, n):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        t0 = ev()
+        for i in range(n):
+            fn(i)
+        t1 = ev()
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / n
+
+    W_C = torch.from_numpy(np.ascontiguousarray(synth.haar_orthogonal(KV_D).T.astype(np.float32))).to(dev)
+    wq, s_u = kv.resq_uc_quantize(W_C)
+    caches = [kv.KvCache(n_seqs, KV_HKV, seq_len, device=dev) for _ in range(2)]
+    pos = torch.arange(seq_len, dtype=torch.int32, device=dev)
+    for b in range(n_seqs):   # fill through the library's own append (checked against the oracle in the tests)
+        k = synth.t_head_vectors(seq_len, KV_HKV, KV_D, dev, stream=1000 + b, lead=1.0, scale=1.5)
+        v = synth.t_head_vectors(seq_len, KV_HKV, KV_D, dev, stream=2000 + b, lead=4.0, shift=0.2)
+        ids = torch.full((seq_len,), b, dtype=torch.int32, device=dev)
+        for c in caches:
+            kv.resq_kv_append(c, k, v, ids, pos, wq, s_u)
+    q = synth.t_head_vectors(n_seqs, KV_HQ, KV_D, dev, stream=3000, lead=1.0, scale=1.5)
+    q16 = torch.empty((n_seqs, KV_HQ, KV_D), dtype=torch.float16, device=dev)
+    out = torch.empty((n_seqs, KV_HQ, KV_D), dtype=torch.float32, device=dev)
+    lens = torch.full((n_seqs,), seq_len, dtype=torch.int32, device=dev)
+    ws = kv.attention_workspace(caches[0], KV_HQ)
+    kv.resq_query_project(q, wq, s_u, q16)
+    attn_ms = timed(lambda i: kv.resq_attention_decode(caches[i % 2], q16, lens, out, ws), steps)
+    cache_bytes = caches[0].nbytes
+    # one generation step's cache update and query projection (launch-latency sized)
+    k1 = synth.t_head_vectors(n_seqs, KV_HKV, KV_D, dev, stream=3001, lead=1.0)
+    v1 = synth.t_head_vectors(n_seqs, KV_HKV, KV_D, dev, stream=3002)
+    ids1 = torch.arange(n_seqs, dtype=torch.int32, device=dev)
+    pos1 = torch.full((n_seqs,), seq_len - 1, dtype=torch.int32, device=dev)
+    app1_ms = timed(lambda i: kv.resq_kv_append(caches[i % 2], k1, v1, ids1, pos1, wq, s_u), steps)
+    qp1_ms = timed(lambda i: kv.resq_query_project(q, wq, s_u, q16), steps)
+    # prefill-sized update: prefill_T tokens of one sequence
+    T = min(prefill_T, seq_len)
+    kp = synth.t_head_vectors(T, KV_HKV, KV_D, dev, stream=3003, lead=1.0)
+    vp = synth.t_head_vectors(T, KV_HKV, KV_D, dev, stream=3004)
+    qp = synth.t_head_vectors(T, KV_HQ, KV_D, dev, stream=3005, lead=1.0)
+    qp16 = torch.empty((T, KV_HQ, KV_D), dtype=torch.float16, device=dev)
+    idsp = torch.zeros(T, dtype=torch.int32, device=dev)
+    appp_ms = timed(lambda i: kv.resq_kv_append(caches[i % 2], kp, vp, idsp, pos[:T], wq, s_u), steps)
+    qpp_ms = timed(lambda i: kv.resq_query_project(qp, wq, s_u, qp16), steps)
+    app_bytes = T * KV_HKV * (2 * 2 * KV_D + 2 * 88)
+    qp_bytes = T * KV_HQ * (2 * KV_D + 2 * KV_D)
+    st = resq.resq_device_status()
+    if st != resq.OK:
+        raise SystemExit(f"device status {st}: {resq.status_string(st)}")
+    gbs = cache_bytes / (attn_ms * 1e-3) / 1e9
+    return {"workload": f"llama3-8b attention, {KV_HQ} query / {KV_HKV} KV heads x {KV_D}: {n_seqs} sequences x {seq_len} cached positions",
+            "steps": steps, "cache_bytes": cache_bytes, "bytes_per_head_vector": 88, "vs_bf16_cache": round(256 / 88, 2),
+            "attention_decode_us": round(attn_ms * 1e3, 2), "attention_cache_stream_gbs": round(gbs, 1),
+            "attention_frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
+            "decode_step_kv_append_us": round(app1_ms * 1e3, 2), "decode_step_query_project_us": round(qp1_ms * 1e3, 2),
+            "prefill_tokens": T, "prefill_kv_append_us": round(appp_ms * 1e3, 2),
+            "prefill_kv_append_gbs": round(app_bytes / (appp_ms * 1e-3) / 1e9, 1),
+            "prefill_query_project_us": round(qpp_ms * 1e3, 2),
+            "prefill_query_project_gbs": round(qp_bytes / (qpp_ms * 1e-3) / 1e9, 1)}
+
+
 # --------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import numpy as np
@@ -437,6 +517,10 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    if args.kv_only:  # profiling runs: the attention-block leg alone
+        print(json.dumps({"kv_cache_path": kv_leg(resq, torch, dev, peaks, max(5, min(args.steps, 20)), args.kv_seqs,
+                                                  args.kv_len)}))
+        return
     if args.decode_only:  # profiling runs: the few-token leg alone
         print(json.dumps({"decode": decode_leg(resq, torch, dev, peaks, layers, max(5, min(args.steps, 20)))}))
         return
@@ -608,6 +692,15 @@ def run_ours(args):
                                            "ms_per_step": round(k["mixed_gemv_us"] * 1e-3, 5),
                                            "frac": k["frac_of_hbm_peak"]}
 
+    # ---- the attention-block path: U_C projection, mixed-precision KV cache, single-query attention
+    kvp = None
+    if not args.no_kv and not only:
+        kvp = kv_leg(resq, torch, dev, peaks, max(5, min(args.steps, 20)), args.kv_seqs, args.kv_len)
+        kernels["attention_decode"] = {"bound": "hbm", "dtype": "f16", "achieved": kvp["attention_cache_stream_gbs"],
+                                       "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                       "ms_per_step": round(kvp["attention_decode_us"] * 1e-3, 5),
+                                       "frac": kvp["attention_frac_of_hbm_peak"]}
+
     # ---- CPU baseline: the oracle on a row sample, rank 0 at N = 1 only; also a parity spot check
     cpu_baseline, parity = None, None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -645,7 +738,7 @@ def run_ours(args):
             "mixed_gemm_frac_of_int8_peak": {"vs_measured_bf16_x2": kernels["mixed_gemm"]["frac"],
                                              "vs_nominal_4500": kernels["mixed_gemm"]["frac_of_nominal_4500"]},
             "per_layer": per_layer,
-            "roofline": roofline, "decode": decode, "asymmetric": asym, "hadamard_down_proj": had, "e2e": e2e, "cpu_baseline": cpu_baseline, "parity_spot_check": parity,
+            "roofline": roofline, "decode": decode, "asymmetric": asym, "hadamard_down_proj": had, "kv_cache_path": kvp, "e2e": e2e, "cpu_baseline": cpu_baseline, "parity_spot_check": parity,
             "gpu_launches": LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
         }
         print(json.dumps(line))
@@ -696,6 +789,10 @@ def main():
     ap.add_argument("--no-asym", action="store_true", help="skip the asymmetric-activation leg (profiling runs)")
     ap.add_argument("--no-decode", action="store_true", help="skip the few-token leg (profiling runs)")
     ap.add_argument("--decode-only", action="store_true", help="run only the few-token leg (profiling runs)")
+    ap.add_argument("--no-kv", action="store_true", help="skip the attention-block leg (profiling runs)")
+    ap.add_argument("--kv-only", action="store_true", help="run only the attention-block leg (profiling runs)")
+    ap.add_argument("--kv-seqs", type=int, default=16, help="sequences in the attention-block leg")
+    ap.add_argument("--kv-len", type=int, default=8192, help="cached positions per sequence in the attention-block leg")
     ap.add_argument("--layers", default="", help="comma-separated subset of qkv,o,gate_up,down (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -264,3 +264,12 @@ def t_kron_orthogonal_bf16(K: int, device, seed: int = SEED_P, inner: int = 128)
     for i in range(a):
         out[i * inner:(i + 1) * inner] = torch.kron(qa[i:i + 1, :], qb).to(torch.float32).to(torch.bfloat16)
     return out
+
+
+def t_head_vectors(T: int, H: int, d: int, device, seed: int = SEED_ATTN, stream: int = 1, lead: float = 4.0,
+                   scale: float = 1.0, shift: float = 0.0):
+    """torch.bfloat16 [T][H][d] on `device`; same recipe as head_vectors()."""
+    import torch
+    x = t_normal(seed, stream, T * H * d, 0, device).reshape(T, H, d) * scale
+    x[:, :, : d // 8] *= lead
+    return (x + shift).to(torch.float32).to(torch.bfloat16)
