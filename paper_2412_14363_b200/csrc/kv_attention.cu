@@ -1,8 +1,8 @@
 // Single-query attention over the mixed-precision KV cache (Section 4.3, Eq. 8; Section 5.1).  HBM-bound: every
 // 5632-byte cache block (32 positions of one KV head: key and value codes, scales, zero-points) is read once.
 //
-// Work.  Blocks are numbered in (sequence, KV head, block) order; the 148 x 8 warps of the persistent grid
-// each take an equal contiguous run of that list.  A warp owns a ring of four block-sized stages filled by
+// Work.  Blocks are numbered in (sequence, KV head, block) order; the 148 x 12 warps of the persistent grid
+// each take an equal contiguous run of that list.  A warp owns a ring of three block-sized stages filled by
 // bulk copies that its lane 0 issues (one copy per block, completion on the warp's own mbarriers), so no
 // CTA-wide barrier exists after start-up.  Whenever the run leaves a (sequence, head) the warp writes one
 // partial record (running maximum, sum of weights, unnormalised output) for the query heads of that KV head;
@@ -12,8 +12,8 @@
 //     q . k_hat = s8 (q8 . c8) + z8 sum(q8) + s4 (q4 . c4) + z4 sum(q4),
 //     sum_j p_j v_hat_j = sum_j (p_j s_j) c_j + sum_j p_j z_j          (per segment),
 // so both products contract fp16 queries / weights with integer codes on mma.sync m16n8k16 (codes are exact
-// in half: 1024 + c and 64 + c are built with one logic op on the packed bytes or nibbles and the offset is
-// subtracted exactly).  Positions are the M rows of the score product (8 query heads of a group as N) and the
+// in half: 1024 + c and 64 + c are built with one logic op on the packed bytes or nibbles; the offsets are
+// removed from the fp32 sums afterwards).  Positions are the M rows of the score product (8 query heads of a group as N) and the
 // K rows of the output product (16 coefficients as M), so the score accumulators only need an 8x8 transpose
 // (movmatrix) to become the second product's B fragments.  Scores, the running softmax and all sums are
 // fp32; the weights p_j s_j are scaled by a power of two taken from the value scales so that they stay in
@@ -28,10 +28,11 @@ namespace resq {
 namespace {
 
 constexpr int kD = 128;
-constexpr int kWarps = 8;
-constexpr int kStages = 4;
+constexpr int kWarps = 12;
+constexpr int kStages = 3;
 constexpr int kBlk = RESQ_KV_BLOCK_BYTES;
 constexpr int kOffK8 = 0, kOffK4 = 512, kOffKM = 2304, kOffV8 = 2816, kOffV4 = 3328, kOffVM = 5120;
+constexpr int kNumWarps = 148 * kWarps;  // the grid is always 148 CTAs
 constexpr int kRecFloats = 8 * (kD + 2);  // per query head of the group: m, l, 128 outputs
 constexpr float kLog2eOverSqrtD = 0.12751743f;  // log2(e) / sqrt(128)
 
@@ -42,8 +43,11 @@ struct AttnParams {
     float* partial;
     float* out;
     int* status;
-    int n_seqs, n_kv_heads, group, capacity, n_warps_total;
+    int n_seqs, n_kv_heads, group, capacity;
 };
+
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ int clamped_len(const int32_t* seq_lens, int b, int capacity) {
     const int len = seq_lens[b];
@@ -95,17 +99,17 @@ __device__ __forceinline__ void advance(Cursor& cu, const AttnParams& p) {
     } while (cu.nblk == 0);
 }
 
-__device__ __forceinline__ uint32_t sub_h2(uint32_t a, uint32_t b) {
-    uint32_t d;
-    asm("sub.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
-}
-// Two codes held in bits 0-3 / 16-19 (lo) or 4-7 / 20-23 (hi) of w as an exact half2.
-__device__ __forceinline__ uint32_t nib_lo(uint32_t w) { return sub_h2((w & 0x000F000Fu) | 0x64006400u, 0x64006400u); }
-__device__ __forceinline__ uint32_t nib_hi(uint32_t w) { return sub_h2((w & 0x00F000F0u) | 0x54005400u, 0x54005400u); }
-// Two bytes of w (picked by SEL, with 0x64 as the upper byte of each half) as an exact half2.
+// Codes as half2 operands WITH an offset: one logic op puts a code into the mantissa of 1024.0 (ulp 1) or of
+// 64.0 (ulp 1/16, for a nibble sitting in bits 4-7), giving 1024 + c or 64 + c exactly.  The offsets are not
+// subtracted per element: they add offset * sum(other operand) to a product, which is removed once per
+// position (scores) or once per record (outputs, via a product with an all-ones operand).
+constexpr float kOffLo = 1024.f, kOffHi = 64.f;
+// Two codes held in bits 0-3 / 16-19 (lo) or 4-7 / 20-23 (hi) of w.
+__device__ __forceinline__ uint32_t nib_lo(uint32_t w) { return (w & 0x000F000Fu) | 0x64006400u; }
+__device__ __forceinline__ uint32_t nib_hi(uint32_t w) { return (w & 0x00F000F0u) | 0x54005400u; }
+// Two bytes of w (picked by SEL), each with 0x64 as the upper byte of its half: 1024 + c.
 template <uint32_t SEL>
-__device__ __forceinline__ uint32_t bytes_h2(uint32_t w) { return sub_h2(__byte_perm(w, 0x64646464u, SEL), 0x64006400u); }
+__device__ __forceinline__ uint32_t bytes_h2(uint32_t w) { return __byte_perm(w, 0x64646464u, SEL); }
 
 __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                         uint32_t b1) {
@@ -144,17 +148,17 @@ __device__ __forceinline__ int kdim(int j, int c, int e) {
 struct ValueScale {  // per position: scales times 2^-E, zero-points, 2^-E, E (E from the larger value scale)
     float sn8, sn4, z8, z4, i2e, e;
 };
-__device__ __forceinline__ ValueScale value_scale(const uint8_t* vm, int tok, bool valid) {
+__device__ __forceinline__ ValueScale value_scale(const uint8_t* vm, int tok) {
     const float4 m = *reinterpret_cast<const float4*>(vm + tok * 16);
     uint32_t eb = __float_as_uint(fmaxf(m.x, m.z)) & 0x7F800000u;
     eb = min(max(eb, 63u << 23), 191u << 23);  // 2^-64 .. 2^64
     ValueScale v;
     v.i2e = __uint_as_float((254u << 23) - eb);
     v.e = static_cast<float>(static_cast<int>(eb >> 23) - 127);
-    v.sn8 = valid ? m.x * v.i2e : 0.f;
-    v.sn4 = valid ? m.z * v.i2e : 0.f;
-    v.z8 = valid ? m.y : 0.f;
-    v.z4 = valid ? m.w : 0.f;
+    v.sn8 = m.x * v.i2e;
+    v.sn4 = m.z * v.i2e;
+    v.z8 = m.y;
+    v.z4 = m.w;
     return v;
 }
 
@@ -171,13 +175,14 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
     }
     if (threadIdx.x == 0) abort_flag = 0;
     __syncthreads();
+    griddep_launch_dependents();  // the merge kernel may be scheduled as SMs free up; it waits for this grid itself
 
     // ---- this warp's run of the global block list
     const long long wg = static_cast<long long>(blockIdx.x) * kWarps + warp;
     int b_first = 0;
     long long before = 0;
     const long long total = scan_blocks(p, lane, -1, &b_first, &before) * p.n_kv_heads;
-    const long long start = total * wg / p.n_warps_total, end = total * (wg + 1) / p.n_warps_total, n = end - start;
+    const long long start = total * wg / kNumWarps, end = total * (wg + 1) / kNumWarps, n = end - start;
     if (n <= 0) return;
     scan_blocks(p, lane, start, &b_first, &before);
     Cursor cons;
@@ -203,7 +208,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
     for (; issued < n && issued < kStages; ++issued) issue(static_cast<int>(issued));
 
     uint32_t qf[8][2];
-    float kq8[2], kq4[2], m_run[2], l[2], z8[2], z4[2], acc[8][4];
+    float kq8[2], kq4[2], ko8[2], ko4[2], m_run[2], l[2], z8[2], z4[2], acc[8][4], ones8[2], ones4[2];
     bool fresh = true, ok = true;
     long long i = 0;
     for (; i < n; ++i) {
@@ -212,7 +217,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
         if (fresh) {  // a new (sequence, KV head): query fragments of its group, empty running state
             fresh = false;
             const __half* qrow = p.q + (static_cast<long long>(cons.b) * p.n_kv_heads * p.group + cons.h * p.group + g) * kD;
-            float s8 = 0.f, s4 = 0.f;
+            float s8 = 0.f, s4 = 0.f, o4 = 0.f;  // sums of q over the segments; offset-weighted sum of the 4-bit part
 #pragma unroll
             for (int j = 0; j < 8; ++j)
 #pragma unroll
@@ -221,15 +226,19 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                     if (g < p.group) v = __halves2half2(qrow[kdim(j, c, 2 * hf)], qrow[kdim(j, c, 2 * hf + 1)]);
                     qf[j][hf] = *reinterpret_cast<const uint32_t*>(&v);
                     const float2 f = __half22float2(v);
-                    if (j == 0) s8 += f.x + f.y; else s4 += f.x + f.y;
+                    if (j == 0) s8 += f.x + f.y;
+                    else { s4 += f.x + f.y; o4 += (hf == 0 ? kOffLo : kOffHi) * (f.x + f.y); }  // entries 0-1 lo, 2-3 hi
                 }
             s8 += __shfl_xor_sync(0xffffffffu, s8, 1); s8 += __shfl_xor_sync(0xffffffffu, s8, 2);
             s4 += __shfl_xor_sync(0xffffffffu, s4, 1); s4 += __shfl_xor_sync(0xffffffffu, s4, 2);
+            o4 += __shfl_xor_sync(0xffffffffu, o4, 1); o4 += __shfl_xor_sync(0xffffffffu, o4, 2);
 #pragma unroll
             for (int e = 0; e < 2; ++e) {  // the score fragment's columns are heads 2c, 2c + 1
                 kq8[e] = kLog2eOverSqrtD * __shfl_sync(0xffffffffu, s8, 4 * (2 * c + e));
                 kq4[e] = kLog2eOverSqrtD * __shfl_sync(0xffffffffu, s4, 4 * (2 * c + e));
-                m_run[e] = -INFINITY; l[e] = z8[e] = z4[e] = 0.f;
+                ko8[e] = kOffLo * kq8[e];
+                ko4[e] = kLog2eOverSqrtD * __shfl_sync(0xffffffffu, o4, 4 * (2 * c + e));
+                m_run[e] = -INFINITY; l[e] = z8[e] = z4[e] = ones8[e] = ones4[e] = 0.f;
             }
 #pragma unroll
             for (int mt = 0; mt < 8; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
@@ -237,6 +246,10 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
         if (!mbar_wait(&full[stage], phase, &abort_flag)) { ok = false; break; }
         const uint8_t* st = ring + stage * kBlk;
         const int valid = min(RESQ_KV_BLOCK, cons.len - RESQ_KV_BLOCK * cons.blk);
+        if (valid < RESQ_KV_BLOCK) {  // last block of a sequence: the unused slots hold anything -- zero their value scales
+            if (lane >= valid) *reinterpret_cast<float4*>(ring + stage * kBlk + kOffVM + lane * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
+            __syncwarp();
+        }
 
         // ---- scores of the 32 positions (two 16-row products), in log2 units, plus the value-scale exponent
         float sc[2][4];
@@ -265,12 +278,15 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
             const float4 kmA = *reinterpret_cast<const float4*>(st + kOffKM + tokA * 16);
             const float4 kmB = *reinterpret_cast<const float4*>(st + kOffKM + tokB * 16);
             const bool vA = tokA < valid, vB = tokB < valid;
-            vs[m][0] = value_scale(st + kOffVM, tokA, vA);
-            vs[m][1] = value_scale(st + kOffVM, tokB, vB);
+            vs[m][0] = value_scale(st + kOffVM, tokA);
+            vs[m][1] = value_scale(st + kOffVM, tokB);
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-                const float sA = kLog2eOverSqrtD * (kmA.x * d8[e] + kmA.z * d4[e]) + kmA.y * kq8[e] + kmA.w * kq4[e] + vs[m][0].e;
-                const float sB = kLog2eOverSqrtD * (kmB.x * d8[2 + e] + kmB.z * d4[2 + e]) + kmB.y * kq8[e] + kmB.w * kq4[e] + vs[m][1].e;
+                // d8, d4 carry the code offsets: remove offset * sum(q) (ko8, ko4) before the key scales apply
+                const float sA = kmA.x * fmaf(kLog2eOverSqrtD, d8[e], -ko8[e]) + kmA.z * fmaf(kLog2eOverSqrtD, d4[e], -ko4[e]) +
+                                 kmA.y * kq8[e] + kmA.w * kq4[e] + vs[m][0].e;
+                const float sB = kmB.x * fmaf(kLog2eOverSqrtD, d8[2 + e], -ko8[e]) + kmB.z * fmaf(kLog2eOverSqrtD, d4[2 + e], -ko4[e]) +
+                                 kmB.y * kq8[e] + kmB.w * kq4[e] + vs[m][1].e;
                 sc[m][e] = vA ? sA : -INFINITY;
                 sc[m][2 + e] = vB ? sB : -INFINITY;
             }
@@ -289,7 +305,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const float a = ex2(m_run[e] - mn[e]);
-                l[e] *= a; z8[e] *= a; z4[e] *= a;
+                l[e] *= a; z8[e] *= a; z4[e] *= a; ones8[e] *= a; ones4[e] *= a;
 #pragma unroll
                 for (int mt = 0; mt < 8; ++mt) { acc[mt][e] *= a; acc[mt][2 + e] *= a; }
                 m_run[e] = mn[e];
@@ -311,6 +327,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                 }
             const uint32_t b80 = movmatrix_trans(pack_h2(p8[0][0], p8[0][1])), b81 = movmatrix_trans(pack_h2(p8[1][0], p8[1][1]));
             const uint32_t b40 = movmatrix_trans(pack_h2(p4[0][0], p4[0][1])), b41 = movmatrix_trans(pack_h2(p4[1][0], p4[1][1]));
+            {   // sum of the (rounded) weights per head, for the code offsets: a product with an all-ones operand
+                float t8[4] = {ones8[0], ones8[1], 0.f, 0.f}, t4[4] = {ones4[0], ones4[1], 0.f, 0.f};
+                mma_f16(t8, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, b80, b81);
+                mma_f16(t4, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, b40, b41);
+                ones8[0] = t8[0]; ones8[1] = t8[1]; ones4[0] = t4[0]; ones4[1] = t4[1];
+            }
             const int t0 = 16 * m + 4 * c;  // contraction entries 2c, 2c+1, 2c+8, 2c+9 are positions t0, t0+2, t0+1, t0+3
             {
                 const uint8_t* v8 = st + kOffV8 + t0 * 16 + 2 * g;
@@ -353,18 +375,20 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                 float* r = rec + (2 * c + e) * (kD + 2);
                 if (g == 0) { r[0] = m_run[e]; r[1] = l[e]; }
                 r += 2;
-                r[2 * g] = acc[0][e] + z8[e];
-                r[2 * g + 1] = acc[0][2 + e] + z8[e];
+                // rows g of the output products carry offset kOffLo, rows g + 8 kOffLo (8-bit) or kOffHi (4-bit)
+                const float f8 = z8[e] - kOffLo * ones8[e], f4lo = z4[e] - kOffLo * ones4[e], f4hi = z4[e] - kOffHi * ones4[e];
+                r[2 * g] = acc[0][e] + f8;
+                r[2 * g + 1] = acc[0][2 + e] + f8;
 #pragma unroll
                 for (int i3 = 0; i3 < 3; ++i3) {
                     const int d0 = 16 + 4 * (g + 8 * i3);
-                    r[d0] = acc[1 + 2 * i3][e] + z4[e];
-                    r[d0 + 1] = acc[1 + 2 * i3][2 + e] + z4[e];
-                    r[d0 + 2] = acc[2 + 2 * i3][e] + z4[e];
-                    r[d0 + 3] = acc[2 + 2 * i3][2 + e] + z4[e];
+                    r[d0] = acc[1 + 2 * i3][e] + f4lo;
+                    r[d0 + 1] = acc[1 + 2 * i3][2 + e] + f4hi;
+                    r[d0 + 2] = acc[2 + 2 * i3][e] + f4lo;
+                    r[d0 + 3] = acc[2 + 2 * i3][2 + e] + f4hi;
                 }
-                r[112 + 2 * g] = acc[7][e] + z4[e];
-                r[113 + 2 * g] = acc[7][2 + e] + z4[e];
+                r[112 + 2 * g] = acc[7][e] + f4lo;
+                r[113 + 2 * g] = acc[7][2 + e] + f4hi;
             }
             fresh = true;
         }
@@ -380,18 +404,18 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
     }
 }
 
-// Merges the partial records of one (sequence, query head): out = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i.
-// The warps that hold a record of this (sequence, KV head) are those whose runs meet its range of the block list.
+// Merges the partial records: out = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i.  One CTA per (sequence, KV head),
+// thread d = output coefficient d of every query head of the group.  The warps that hold a record of this
+// (sequence, KV head) are those whose runs meet its range of the block list.  Launched so that it may start
+// while the attention kernel drains: everything before griddepcontrol.wait reads only the sequence lengths.
 __global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams p) {
     __shared__ long long red[2][kD / 32];
-    const int n_q_heads = p.n_kv_heads * p.group;
-    const int b = blockIdx.x / n_q_heads, hq = blockIdx.x - b * n_q_heads;
-    const int hk = hq / p.group, hg = hq - hk * p.group, d = threadIdx.x;
+    const int b = blockIdx.x / p.n_kv_heads, hk = blockIdx.x - b * p.n_kv_heads, d = threadIdx.x;
     long long before = 0, total = 0;
     for (int i = d; i < p.n_seqs; i += kD) {
         const int len = p.seq_lens[i];
-        if (hq == 0 && b == 0 && (len < 0 || len > p.capacity)) atomicOr(p.status, RESQ_ERR_INDEX);
-        const int t = (clamped_len(p.seq_lens, i, p.capacity) + 31) >> 5;
+        if (blockIdx.x == 0 && (len < 0 || len > p.capacity)) atomicOr(p.status, RESQ_ERR_INDEX);
+        const int t = ((len < 0 ? 0 : (len > p.capacity ? p.capacity : len)) + 31) >> 5;
         total += t;
         if (i < b) before += t;
     }
@@ -404,38 +428,51 @@ __global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams 
     __syncthreads();
     before = red[0][0] + red[0][1] + red[0][2] + red[0][3];
     total = (red[1][0] + red[1][1] + red[1][2] + red[1][3]) * p.n_kv_heads;
-    float* out = p.out + (static_cast<long long>(b) * n_q_heads + hq) * kD;
+    float* out = p.out + (static_cast<long long>(b) * p.n_kv_heads + hk) * p.group * kD;
     const int nblk = (clamped_len(p.seq_lens, b, p.capacity) + 31) >> 5;
     if (nblk == 0) {  // empty sequence
-        out[d] = 0.f;
+        for (int hg = 0; hg < p.group; ++hg) out[hg * kD + d] = 0.f;
         return;
     }
     const long long lo = before * p.n_kv_heads + static_cast<long long>(hk) * nblk, hi = lo + nblk;  // [lo, hi)
-    const long long nw = p.n_warps_total;
-    const long long w_first = ((lo + 1) * nw - 1) / total, w_last = (hi * nw - 1) / total;
+    constexpr long long nw = kNumWarps;
+    const int w_first = static_cast<int>(((lo + 1) * nw - 1) / total), w_last = static_cast<int>((hi * nw - 1) / total);
     const long long s = static_cast<long long>(b) * p.n_kv_heads + hk;
-    float M = -INFINITY;
-    for (long long w = w_first; w <= w_last; ++w) {
+    auto holds_record = [&](int w) {  // a non-empty run that meets [lo, hi)
         const long long rs = total * w / nw, re = total * (w + 1) / nw;
-        if (re <= rs || re <= lo || rs >= hi) continue;  // empty run, or no block of this range
-        M = fmaxf(M, p.partial[(w + s) * kRecFloats + hg * (kD + 2)]);
+        return re > rs && re > lo && rs < hi;
+    };
+    griddep_wait();
+    float M[8], num[8], den[8];
+#pragma unroll
+    for (int hg = 0; hg < 8; ++hg) { M[hg] = -INFINITY; num[hg] = den[hg] = 0.f; }
+    for (int w = w_first; w <= w_last; ++w) {
+        if (!holds_record(w)) continue;
+        const float* r = p.partial + (w + s) * kRecFloats;
+#pragma unroll
+        for (int hg = 0; hg < 8; ++hg)
+            if (hg < p.group) M[hg] = fmaxf(M[hg], __ldcg(r + hg * (kD + 2)));
     }
-    float num = 0.f, den = 0.f;
-    for (long long w = w_first; w <= w_last; ++w) {
-        const long long rs = total * w / nw, re = total * (w + 1) / nw;
-        if (re <= rs || re <= lo || rs >= hi) continue;
-        const float* r = p.partial + (w + s) * kRecFloats + hg * (kD + 2);
-        const float f = ex2(r[0] - M);
-        den = fmaf(f, r[1], den);
-        num = fmaf(f, r[2 + d], num);
+    for (int w = w_first; w <= w_last; ++w) {
+        if (!holds_record(w)) continue;
+        const float* r = p.partial + (w + s) * kRecFloats;
+#pragma unroll
+        for (int hg = 0; hg < 8; ++hg)
+            if (hg < p.group) {
+                const float f = ex2(__ldcg(r + hg * (kD + 2)) - M[hg]);
+                den[hg] = fmaf(f, __ldcg(r + hg * (kD + 2) + 1), den[hg]);
+                num[hg] = fmaf(f, __ldcg(r + hg * (kD + 2) + 2 + d), num[hg]);
+            }
     }
-    out[d] = num / den;
+#pragma unroll
+    for (int hg = 0; hg < 8; ++hg)
+        if (hg < p.group) out[hg * kD + d] = num[hg] / den[hg];
 }
 
 }  // namespace
 
 size_t attention_scratch_bytes(int n_seqs, int n_kv_heads) {
-    return (static_cast<size_t>(148) * kWarps + static_cast<size_t>(n_seqs) * n_kv_heads) * kRecFloats * sizeof(float);
+    return (static_cast<size_t>(kNumWarps) + static_cast<size_t>(n_seqs) * n_kv_heads) * kRecFloats * sizeof(float);
 }
 
 cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q16, int n_q_heads, const int32_t* seq_lens,
@@ -461,11 +498,18 @@ cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q1
     p.n_kv_heads = cache.n_kv_heads;
     p.group = n_q_heads / cache.n_kv_heads;
     p.capacity = cache.capacity;
-    p.n_warps_total = 148 * kWarps;
     attention_decode_kernel<<<148, kWarps * 32, kSmem, st>>>(p);
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
-    attention_combine_kernel<<<cache.n_seqs * n_q_heads, kD, 0, st>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cache.n_seqs * cache.n_kv_heads, 1, 1);
+    cfg.blockDim = dim3(kD, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, attention_combine_kernel, p);
 }
 
 }  // namespace resq
