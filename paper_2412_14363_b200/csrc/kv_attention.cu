@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
 #pragma unroll
         for (int m = 0; m < 2; ++m) {
             const int tokA = 16 * m + 2 * g, tokB = tokA + 1;  // rows g and g + 8 of the product
-            float d8[4] = {0.f, 0.f, 0.f, 0.f}, d4[4] = {0.f, 0.f, 0.f, 0.f};
+            float d8[4] = {0.f, 0.f, 0.f, 0.f}, d4[4] = {0.f, 0.f, 0.f, 0.f}, d4b[4] = {0.f, 0.f, 0.f, 0.f};  // two chains for the 4-bit steps
             {
                 const uint32_t wa = lds32(st + kOffK8 + tokA * 16 + 4 * c), wb = lds32(st + kOffK8 + tokB * 16 + 4 * c);
                 mma_f16(d8, bytes_h2<0x4140>(wa), bytes_h2<0x4140>(wb), bytes_h2<0x4342>(wa), bytes_h2<0x4342>(wb),
@@ -268,13 +268,15 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                 uint32_t wa = lds32(st + kOffK4 + tokA * 56 + 4 * (c + 4 * i3)), wb = lds32(st + kOffK4 + tokB * 56 + 4 * (c + 4 * i3));
                 mma_f16(d4, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[1 + 2 * i3][0], qf[1 + 2 * i3][1]);
                 wa >>= 8; wb >>= 8;
-                mma_f16(d4, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[2 + 2 * i3][0], qf[2 + 2 * i3][1]);
+                mma_f16(d4b, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[2 + 2 * i3][0], qf[2 + 2 * i3][1]);
             }
             {
                 uint32_t xa = lds16(st + kOffK4 + tokA * 56 + 48 + 2 * c), xb = lds16(st + kOffK4 + tokB * 56 + 48 + 2 * c);
                 xa |= xa << 8; xb |= xb << 8;
-                mma_f16(d4, nib_lo(xa), nib_lo(xb), nib_hi(xa), nib_hi(xb), qf[7][0], qf[7][1]);
+                mma_f16(d4b, nib_lo(xa), nib_lo(xb), nib_hi(xa), nib_hi(xb), qf[7][0], qf[7][1]);
             }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) d4[e] += d4b[e];
             const float4 kmA = *reinterpret_cast<const float4*>(st + kOffKM + tokA * 16);
             const float4 kmB = *reinterpret_cast<const float4*>(st + kOffKM + tokB * 16);
             const bool vA = tokA < valid, vB = tokB < valid;
@@ -404,13 +406,20 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
     }
 }
 
-// Merges the partial records: out = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i.  One CTA per (sequence, KV head),
-// thread d = output coefficient d of every query head of the group.  The warps that hold a record of this
-// (sequence, KV head) are those whose runs meet its range of the block list.  Launched so that it may start
-// while the attention kernel drains: everything before griddepcontrol.wait reads only the sequence lengths.
+// Merges the partial records of one (sequence, query head): out = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i.
+// The warps that hold a record of this (sequence, KV head) are those whose runs meet its range of the block
+// list; they are taken 128 at a time: thread t reads (m, l) of candidate t, the block agrees on the maximum,
+// then every thread (one output coefficient each) adds the weighted records with eight loads in flight.
+// Launched so that it may start while the attention kernel drains: everything before griddepcontrol.wait
+// reads only the sequence lengths.
 __global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams p) {
     __shared__ long long red[2][kD / 32];
-    const int b = blockIdx.x / p.n_kv_heads, hk = blockIdx.x - b * p.n_kv_heads, d = threadIdx.x;
+    __shared__ float redf[2][kD / 32];
+    __shared__ float f_s[kD];
+    __shared__ long long rec_s[kD];
+    const int n_q_heads = p.n_kv_heads * p.group;
+    const int b = blockIdx.x / n_q_heads, hq = blockIdx.x - b * n_q_heads;
+    const int hk = hq / p.group, hg = hq - hk * p.group, d = threadIdx.x, warp = d >> 5;
     long long before = 0, total = 0;
     for (int i = d; i < p.n_seqs; i += kD) {
         const int len = p.seq_lens[i];
@@ -424,49 +433,65 @@ __global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams 
         before += __shfl_xor_sync(0xffffffffu, before, o);
         total += __shfl_xor_sync(0xffffffffu, total, o);
     }
-    if ((d & 31) == 0) { red[0][d >> 5] = before; red[1][d >> 5] = total; }
+    if ((d & 31) == 0) { red[0][warp] = before; red[1][warp] = total; }
     __syncthreads();
     before = red[0][0] + red[0][1] + red[0][2] + red[0][3];
     total = (red[1][0] + red[1][1] + red[1][2] + red[1][3]) * p.n_kv_heads;
-    float* out = p.out + (static_cast<long long>(b) * p.n_kv_heads + hk) * p.group * kD;
+    float* out = p.out + (static_cast<long long>(b) * n_q_heads + hq) * kD;
     const int nblk = (clamped_len(p.seq_lens, b, p.capacity) + 31) >> 5;
     if (nblk == 0) {  // empty sequence
-        for (int hg = 0; hg < p.group; ++hg) out[hg * kD + d] = 0.f;
+        out[d] = 0.f;
         return;
     }
     const long long lo = before * p.n_kv_heads + static_cast<long long>(hk) * nblk, hi = lo + nblk;  // [lo, hi)
     constexpr long long nw = kNumWarps;
     const int w_first = static_cast<int>(((lo + 1) * nw - 1) / total), w_last = static_cast<int>((hi * nw - 1) / total);
     const long long s = static_cast<long long>(b) * p.n_kv_heads + hk;
-    auto holds_record = [&](int w) {  // a non-empty run that meets [lo, hi)
-        const long long rs = total * w / nw, re = total * (w + 1) / nw;
-        return re > rs && re > lo && rs < hi;
-    };
     griddep_wait();
-    float M[8], num[8], den[8];
+    float M = -INFINITY, num = 0.f, den = 0.f;  // den is a per-thread partial until the end
+    for (int w0 = w_first; w0 <= w_last; w0 += kD) {
+        const int w = w0 + d;
+        bool have = false;
+        if (w <= w_last) {  // a non-empty run that meets [lo, hi)
+            const long long rs = total * w / nw, re = total * (w + 1) / nw;
+            have = re > rs && re > lo && rs < hi;
+        }
+        const long long off = (w + s) * kRecFloats + hg * (kD + 2);
+        float m = -INFINITY, lw = 0.f;
+        if (have) { m = __ldcg(p.partial + off); lw = __ldcg(p.partial + off + 1); }
+        float mx = m;
 #pragma unroll
-    for (int hg = 0; hg < 8; ++hg) { M[hg] = -INFINITY; num[hg] = den[hg] = 0.f; }
-    for (int w = w_first; w <= w_last; ++w) {
-        if (!holds_record(w)) continue;
-        const float* r = p.partial + (w + s) * kRecFloats;
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        __syncthreads();  // the previous chunk's f_s / rec_s / redf are no longer read
+        if ((d & 31) == 0) redf[0][warp] = mx;
+        __syncthreads();
+        const float Mn = fmaxf(M, fmaxf(fmaxf(redf[0][0], redf[0][1]), fmaxf(redf[0][2], redf[0][3])));
+        const float resc = ex2(M - Mn);  // 0 on the first chunk
+        M = Mn;
+        const float f = have ? ex2(m - M) : 0.f;
+        f_s[d] = f;
+        rec_s[d] = have ? off + 2 : -1;
+        num *= resc;
+        den = fmaf(f, lw, den * resc);
+        __syncthreads();
+        const int cnt = min(kD, w_last - w0 + 1);
+        for (int i0 = 0; i0 < cnt; i0 += 8) {
+            float v[8];
 #pragma unroll
-        for (int hg = 0; hg < 8; ++hg)
-            if (hg < p.group) M[hg] = fmaxf(M[hg], __ldcg(r + hg * (kD + 2)));
-    }
-    for (int w = w_first; w <= w_last; ++w) {
-        if (!holds_record(w)) continue;
-        const float* r = p.partial + (w + s) * kRecFloats;
-#pragma unroll
-        for (int hg = 0; hg < 8; ++hg)
-            if (hg < p.group) {
-                const float f = ex2(__ldcg(r + hg * (kD + 2)) - M[hg]);
-                den[hg] = fmaf(f, __ldcg(r + hg * (kD + 2) + 1), den[hg]);
-                num[hg] = fmaf(f, __ldcg(r + hg * (kD + 2) + 2 + d), num[hg]);
+            for (int k = 0; k < 8; ++k) {
+                const long long r = i0 + k < cnt ? rec_s[i0 + k] : -1;
+                v[k] = r >= 0 ? __ldcg(p.partial + r + d) : 0.f;
             }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) num = fmaf(i0 + k < cnt ? f_s[i0 + k] : 0.f, v[k], num);
+        }
     }
 #pragma unroll
-    for (int hg = 0; hg < 8; ++hg)
-        if (hg < p.group) out[hg * kD + d] = num[hg] / den[hg];
+    for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    __syncthreads();
+    if ((d & 31) == 0) redf[1][warp] = den;
+    __syncthreads();
+    out[d] = num / (redf[1][0] + redf[1][1] + redf[1][2] + redf[1][3]);
 }
 
 }  // namespace
@@ -501,7 +526,7 @@ cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q1
     attention_decode_kernel<<<148, kWarps * 32, kSmem, st>>>(p);
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cache.n_seqs * cache.n_kv_heads, 1, 1);
+    cfg.gridDim = dim3(cache.n_seqs * n_q_heads, 1, 1);
     cfg.blockDim = dim3(kD, 1, 1);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
