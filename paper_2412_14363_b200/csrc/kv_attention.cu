@@ -104,9 +104,20 @@ __device__ __forceinline__ void advance(Cursor& cu, const AttnParams& p) {
 // subtracted per element: they add offset * sum(other operand) to a product, which is removed once per
 // position (scores) or once per record (outputs, via a product with an all-ones operand).
 constexpr float kOffLo = 1024.f, kOffHi = 64.f;
-// Two codes held in bits 0-3 / 16-19 (lo) or 4-7 / 20-23 (hi) of w.
-__device__ __forceinline__ uint32_t nib_lo(uint32_t w) { return (w & 0x000F000Fu) | 0x64006400u; }
-__device__ __forceinline__ uint32_t nib_hi(uint32_t w) { return (w & 0x00F000F0u) | 0x54005400u; }
+// Two codes held in bits 0-3 / 16-19 (lo) or 4-7 / 20-23 (hi) of w: (w & mask) | exponent as ONE three-input
+// logic op.  That needs mask and exponent in registers (the instruction takes a single immediate, and with two
+// compile-time constants the assembler emits an AND and an OR), so the kernel derives the four words from a
+// run-time value once and passes them around in this struct.
+struct NibbleConsts {
+    uint32_t mask_lo, exp_lo, mask_hi, exp_hi;
+};
+__device__ __forceinline__ uint32_t and_or(uint32_t w, uint32_t mask, uint32_t bits) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(w), "r"(mask), "r"(bits));  // (w & mask) | bits
+    return d;
+}
+#define nib_lo(w) and_or((w), nc.mask_lo, nc.exp_lo)
+#define nib_hi(w) and_or((w), nc.mask_hi, nc.exp_hi)
 // Two bytes of w (picked by SEL), each with 0x64 as the upper byte of its half: 1024 + c.
 template <uint32_t SEL>
 __device__ __forceinline__ uint32_t bytes_h2(uint32_t w) { return __byte_perm(w, 0x64646464u, SEL); }
@@ -145,21 +156,24 @@ __device__ __forceinline__ int kdim(int j, int c, int e) {
     return 16 + 8 * (c + 4 * i) + 2 * sub + ((e & 1) << 2) + (e >> 1);
 }
 
-struct ValueScale {  // per position: scales times 2^-E, zero-points, 2^-E, E (E from the larger value scale)
-    float sn8, sn4, z8, z4, i2e, e;
+struct ValueScale {  // per position: value scales times 2^-E (E: the block's exponent), zero-points
+    float sn8, sn4, z8, z4;
 };
-__device__ __forceinline__ ValueScale value_scale(const uint8_t* vm, int tok) {
+__device__ __forceinline__ ValueScale value_scale(const uint8_t* vm, int tok, float i2e) {
     const float4 m = *reinterpret_cast<const float4*>(vm + tok * 16);
-    uint32_t eb = __float_as_uint(fmaxf(m.x, m.z)) & 0x7F800000u;
-    eb = min(max(eb, 63u << 23), 191u << 23);  // 2^-64 .. 2^64
     ValueScale v;
-    v.i2e = __uint_as_float((254u << 23) - eb);
-    v.e = static_cast<float>(static_cast<int>(eb >> 23) - 127);
-    v.sn8 = m.x * v.i2e;
-    v.sn4 = m.z * v.i2e;
+    v.sn8 = m.x * i2e;
+    v.sn4 = m.z * i2e;
     v.z8 = m.y;
     v.z4 = m.w;
     return v;
+}
+// First product of a chain: C = 0.
+__device__ __forceinline__ void mma_f16_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                              uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 
 __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const AttnParams p) {
@@ -207,13 +221,16 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
     long long issued = 0;
     for (; issued < n && issued < kStages; ++issued) issue(static_cast<int>(issued));
 
+    // capacity is positive; the compiler cannot know, so the four words stay in registers (see NibbleConsts)
+    const uint32_t never = p.capacity < 0 ? 1u : 0u;
+    const NibbleConsts nc{0x000F000Fu ^ never, 0x64006400u ^ never, 0x00F000F0u ^ never, 0x54005400u ^ never};
     uint32_t qf[8][2];
-    float kq8[2], kq4[2], ko8[2], ko4[2], m_run[2], l[2], z8[2], z4[2], acc[8][4], ones8[2], ones4[2];
+    float kq8[2], kq4[2], ko8[2], ko4[2], m_run[2], l[2], z8[2], z4[2], acc[8][4], ones8[4], ones4[4];
     bool fresh = true, ok = true;
     long long i = 0;
+    int stage = 0;
+    uint32_t phase = 0;
     for (; i < n; ++i) {
-        const int stage = static_cast<int>(i % kStages);
-        const uint32_t phase = static_cast<uint32_t>(i / kStages) & 1u;
         if (fresh) {  // a new (sequence, KV head): query fragments of its group, empty running state
             fresh = false;
             const __half* qrow = p.q + (static_cast<long long>(cons.b) * p.n_kv_heads * p.group + cons.h * p.group + g) * kD;
@@ -238,7 +255,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                 kq4[e] = kLog2eOverSqrtD * __shfl_sync(0xffffffffu, s4, 4 * (2 * c + e));
                 ko8[e] = kOffLo * kq8[e];
                 ko4[e] = kLog2eOverSqrtD * __shfl_sync(0xffffffffu, o4, 4 * (2 * c + e));
-                m_run[e] = -INFINITY; l[e] = z8[e] = z4[e] = ones8[e] = ones4[e] = 0.f;
+                m_run[e] = -INFINITY; l[e] = z8[e] = z4[e] = ones8[e] = ones4[e] = ones8[2 + e] = ones4[2 + e] = 0.f;
             }
 #pragma unroll
             for (int mt = 0; mt < 8; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
@@ -250,48 +267,67 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
             if (lane >= valid) *reinterpret_cast<float4*>(ring + stage * kBlk + kOffVM + lane * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
             __syncwarp();
         }
+        // ---- the block's exponent: E from the largest value scale, clamped to 2^-64 .. 2^64 (0 scales included)
+        float e_blk, i2e;
+        {
+            const float4 vm = *reinterpret_cast<const float4*>(st + kOffVM + lane * 16);
+            uint32_t eb = __reduce_max_sync(0xffffffffu, __float_as_uint(fmaxf(fmaxf(vm.x, vm.z), 0.f))) & 0x7F800000u;
+            eb = min(max(eb, 63u << 23), 191u << 23);
+            i2e = __uint_as_float((254u << 23) - eb);
+            e_blk = static_cast<float>(static_cast<int>(eb >> 23) - 127);
+        }
 
-        // ---- scores of the 32 positions (two 16-row products), in log2 units, plus the value-scale exponent
+        // ---- scores of the 32 positions (two 16-row products), in log2 units, plus the block's exponent
         float sc[2][4];
         ValueScale vs[2][2];
 #pragma unroll
         for (int m = 0; m < 2; ++m) {
             const int tokA = 16 * m + 2 * g, tokB = tokA + 1;  // rows g and g + 8 of the product
-            float d8[4] = {0.f, 0.f, 0.f, 0.f}, d4[4] = {0.f, 0.f, 0.f, 0.f}, d4b[4] = {0.f, 0.f, 0.f, 0.f};  // two chains for the 4-bit steps
+            float d8[4], d4[4], d4b[4];  // two chains for the 4-bit steps
             {
                 const uint32_t wa = lds32(st + kOffK8 + tokA * 16 + 4 * c), wb = lds32(st + kOffK8 + tokB * 16 + 4 * c);
-                mma_f16(d8, bytes_h2<0x4140>(wa), bytes_h2<0x4140>(wb), bytes_h2<0x4342>(wa), bytes_h2<0x4342>(wb),
-                        qf[0][0], qf[0][1]);
+                mma_f16_first(d8, bytes_h2<0x4140>(wa), bytes_h2<0x4140>(wb), bytes_h2<0x4342>(wa), bytes_h2<0x4342>(wb),
+                              qf[0][0], qf[0][1]);
             }
 #pragma unroll
             for (int i3 = 0; i3 < 3; ++i3) {
                 uint32_t wa = lds32(st + kOffK4 + tokA * 56 + 4 * (c + 4 * i3)), wb = lds32(st + kOffK4 + tokB * 56 + 4 * (c + 4 * i3));
-                mma_f16(d4, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[1 + 2 * i3][0], qf[1 + 2 * i3][1]);
+                if (i3 == 0) mma_f16_first(d4, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[1][0], qf[1][1]);
+                else mma_f16(d4, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[1 + 2 * i3][0], qf[1 + 2 * i3][1]);
                 wa >>= 8; wb >>= 8;
-                mma_f16(d4b, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[2 + 2 * i3][0], qf[2 + 2 * i3][1]);
+                if (i3 == 0) mma_f16_first(d4b, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[2][0], qf[2][1]);
+                else mma_f16(d4b, nib_lo(wa), nib_lo(wb), nib_hi(wa), nib_hi(wb), qf[2 + 2 * i3][0], qf[2 + 2 * i3][1]);
             }
             {
                 uint32_t xa = lds16(st + kOffK4 + tokA * 56 + 48 + 2 * c), xb = lds16(st + kOffK4 + tokB * 56 + 48 + 2 * c);
-                xa |= xa << 8; xb |= xb << 8;
+                xa = __byte_perm(xa, 0u, 0x4110); xb = __byte_perm(xb, 0u, 0x4110);  // nibbles 2, 3 up to bits 16-23
                 mma_f16(d4b, nib_lo(xa), nib_lo(xb), nib_hi(xa), nib_hi(xb), qf[7][0], qf[7][1]);
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e) d4[e] += d4b[e];
             const float4 kmA = *reinterpret_cast<const float4*>(st + kOffKM + tokA * 16);
             const float4 kmB = *reinterpret_cast<const float4*>(st + kOffKM + tokB * 16);
-            const bool vA = tokA < valid, vB = tokB < valid;
-            vs[m][0] = value_scale(st + kOffVM, tokA);
-            vs[m][1] = value_scale(st + kOffVM, tokB);
+            vs[m][0] = value_scale(st + kOffVM, tokA, i2e);
+            vs[m][1] = value_scale(st + kOffVM, tokB, i2e);
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 // d8, d4 carry the code offsets: remove offset * sum(q) (ko8, ko4) before the key scales apply
                 const float sA = kmA.x * fmaf(kLog2eOverSqrtD, d8[e], -ko8[e]) + kmA.z * fmaf(kLog2eOverSqrtD, d4[e], -ko4[e]) +
-                                 kmA.y * kq8[e] + kmA.w * kq4[e] + vs[m][0].e;
+                                 kmA.y * kq8[e] + kmA.w * kq4[e] + e_blk;
                 const float sB = kmB.x * fmaf(kLog2eOverSqrtD, d8[2 + e], -ko8[e]) + kmB.z * fmaf(kLog2eOverSqrtD, d4[2 + e], -ko4[e]) +
-                                 kmB.y * kq8[e] + kmB.w * kq4[e] + vs[m][1].e;
-                sc[m][e] = vA ? sA : -INFINITY;
-                sc[m][2 + e] = vB ? sB : -INFINITY;
+                                 kmB.y * kq8[e] + kmB.w * kq4[e] + e_blk;
+                sc[m][e] = sA;
+                sc[m][2 + e] = sB;
             }
+        }
+        if (valid < RESQ_KV_BLOCK) {  // unused slots of a sequence's last block take no weight
+#pragma unroll
+            for (int m = 0; m < 2; ++m)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    if (16 * m + 2 * g >= valid) sc[m][e] = -INFINITY;
+                    if (16 * m + 2 * g + 1 >= valid) sc[m][2 + e] = -INFINITY;
+                }
         }
         // ---- running maximum per head (columns 2c, 2c + 1), shared by the 8 lanes with this c
         float mn[2];
@@ -307,7 +343,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const float a = ex2(m_run[e] - mn[e]);
-                l[e] *= a; z8[e] *= a; z4[e] *= a; ones8[e] *= a; ones4[e] *= a;
+                l[e] *= a; z8[e] *= a; z4[e] *= a; ones8[e] *= a; ones4[e] *= a; ones8[2 + e] *= a; ones4[2 + e] *= a;
 #pragma unroll
                 for (int mt = 0; mt < 8; ++mt) { acc[mt][e] *= a; acc[mt][2 + e] *= a; }
                 m_run[e] = mn[e];
@@ -323,35 +359,33 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                 for (int e = 0; e < 2; ++e) {
                     const ValueScale& v = vs[m][t];
                     const float pw = ex2(sc[m][2 * t + e] - m_run[e]);
-                    const float w = pw * v.i2e;
+                    const float w = pw * i2e;
                     l[e] += w; z8[e] = fmaf(w, v.z8, z8[e]); z4[e] = fmaf(w, v.z4, z4[e]);
                     p8[t][e] = pw * v.sn8; p4[t][e] = pw * v.sn4;
                 }
             const uint32_t b80 = movmatrix_trans(pack_h2(p8[0][0], p8[0][1])), b81 = movmatrix_trans(pack_h2(p8[1][0], p8[1][1]));
             const uint32_t b40 = movmatrix_trans(pack_h2(p4[0][0], p4[0][1])), b41 = movmatrix_trans(pack_h2(p4[1][0], p4[1][1]));
             {   // sum of the (rounded) weights per head, for the code offsets: a product with an all-ones operand
-                float t8[4] = {ones8[0], ones8[1], 0.f, 0.f}, t4[4] = {ones4[0], ones4[1], 0.f, 0.f};
-                mma_f16(t8, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, b80, b81);
-                mma_f16(t4, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, b40, b41);
-                ones8[0] = t8[0]; ones8[1] = t8[1]; ones4[0] = t4[0]; ones4[1] = t4[1];
+                mma_f16(ones8, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, b80, b81);  // all 16 rows alike
+                mma_f16(ones4, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, 0x3C003C00u, b40, b41);
             }
             const int t0 = 16 * m + 4 * c;  // contraction entries 2c, 2c+1, 2c+8, 2c+9 are positions t0, t0+2, t0+1, t0+3
             {
                 const uint8_t* v8 = st + kOffV8 + t0 * 16 + 2 * g;
-                const uint32_t w02 = lds16(v8) | (lds16(v8 + 32) << 16), w13 = lds16(v8 + 16) | (lds16(v8 + 48) << 16);
+                const uint32_t w02 = __byte_perm(lds16(v8), lds16(v8 + 32), 0x5410), w13 = __byte_perm(lds16(v8 + 16), lds16(v8 + 48), 0x5410);
                 mma_f16(acc[0], bytes_h2<0x4240>(w02), bytes_h2<0x4341>(w02), bytes_h2<0x4240>(w13), bytes_h2<0x4341>(w13), b80, b81);
             }
 #pragma unroll
             for (int i3 = 0; i3 < 3; ++i3) {
                 const uint8_t* v4 = st + kOffV4 + t0 * 56 + 2 * (g + 8 * i3);
-                uint32_t w02 = lds16(v4) | (lds16(v4 + 112) << 16), w13 = lds16(v4 + 56) | (lds16(v4 + 168) << 16);
+                uint32_t w02 = __byte_perm(lds16(v4), lds16(v4 + 112), 0x5410), w13 = __byte_perm(lds16(v4 + 56), lds16(v4 + 168), 0x5410);
                 mma_f16(acc[1 + 2 * i3], nib_lo(w02), nib_hi(w02), nib_lo(w13), nib_hi(w13), b40, b41);
                 w02 >>= 8; w13 >>= 8;
                 mma_f16(acc[2 + 2 * i3], nib_lo(w02), nib_hi(w02), nib_lo(w13), nib_hi(w13), b40, b41);
             }
             {
                 const uint8_t* v4 = st + kOffV4 + t0 * 56 + 48 + g;
-                const uint32_t w02 = v4[0] | (static_cast<uint32_t>(v4[112]) << 16), w13 = v4[56] | (static_cast<uint32_t>(v4[168]) << 16);
+                const uint32_t w02 = __byte_perm(v4[0], v4[112], 0x5410), w13 = __byte_perm(v4[56], v4[168], 0x5410);
                 mma_f16(acc[7], nib_lo(w02), nib_hi(w02), nib_lo(w13), nib_hi(w13), b40, b41);
             }
         }
@@ -360,6 +394,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
             issue(stage);
             ++issued;
         }
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
         // ---- leaving this (sequence, head), or the run: one partial record
         if (cons.blk == cons.nblk - 1 || i == n - 1) {
 #pragma unroll
