@@ -104,6 +104,7 @@ __device__ __forceinline__ void advance(Cursor& cu, const AttnParams& p) {
 // subtracted per element: they add offset * sum(other operand) to a product, which is removed once per
 // position (scores) or once per record (outputs, via a product with an all-ones operand).
 constexpr float kOffLo = 1024.f, kOffHi = 64.f;
+constexpr float kSlack = 8.f;  // log2 of the largest softmax weight before the reference is raised
 // Two codes held in bits 0-3 / 16-19 (lo) or 4-7 / 20-23 (hi) of w: (w & mask) | exponent as ONE three-input
 // logic op.  That needs mask and exponent in registers (the instruction takes a single immediate, and with two
 // compile-time constants the assembler emits an AND and an OR), so the kernel derives the four words from a
@@ -329,24 +330,27 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                     if (16 * m + 2 * g + 1 >= valid) sc[m][2 + e] = -INFINITY;
                 }
         }
-        // ---- running maximum per head (columns 2c, 2c + 1), shared by the 8 lanes with this c
-        float mn[2];
+        // ---- reference exponent per head (columns 2c, 2c + 1), shared by the 8 lanes with this c.  It is raised to
+        // the running maximum only when some score exceeds it by more than kSlack (and at a record's first block,
+        // where it is -inf), so the usual block needs one vote instead of a shuffle reduction; meanwhile weights reach
+        // at most 2^kSlack, far inside half's range.
+        {
+            const float mx0 = fmaxf(fmaxf(sc[0][0], sc[0][2]), fmaxf(sc[1][0], sc[1][2]));
+            const float mx1 = fmaxf(fmaxf(sc[0][1], sc[0][3]), fmaxf(sc[1][1], sc[1][3]));
+            if (__any_sync(0xffffffffu, mx0 > m_run[0] + kSlack || mx1 > m_run[1] + kSlack)) {
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            float mx = fmaxf(fmaxf(sc[0][e], sc[0][2 + e]), fmaxf(sc[1][e], sc[1][2 + e]));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-            mn[e] = fmaxf(m_run[e], mx);
-        }
-        if (__any_sync(0xffffffffu, mn[0] != m_run[0] || mn[1] != m_run[1])) {
+                for (int e = 0; e < 2; ++e) {
+                    float mx = e == 0 ? mx0 : mx1;
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                    const float mn = fmaxf(m_run[e], mx);
+                    const float a = ex2(m_run[e] - mn);
+                    l[e] *= a; z8[e] *= a; z4[e] *= a; ones8[e] *= a; ones4[e] *= a; ones8[2 + e] *= a; ones4[2 + e] *= a;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const float a = ex2(m_run[e] - mn[e]);
-                l[e] *= a; z8[e] *= a; z4[e] *= a; ones8[e] *= a; ones4[e] *= a; ones8[2 + e] *= a; ones4[2 + e] *= a;
-#pragma unroll
-                for (int mt = 0; mt < 8; ++mt) { acc[mt][e] *= a; acc[mt][2 + e] *= a; }
-                m_run[e] = mn[e];
+                    for (int mt = 0; mt < 8; ++mt) { acc[mt][e] *= a; acc[mt][2 + e] *= a; }
+                    m_run[e] = mn;
+                }
             }
         }
         // ---- weights, their transposes as B fragments, and the output products
