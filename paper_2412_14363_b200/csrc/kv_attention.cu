@@ -104,6 +104,7 @@ __device__ __forceinline__ void advance(Cursor& cu, const AttnParams& p) {
 // subtracted per element: they add offset * sum(other operand) to a product, which is removed once per
 // position (scores) or once per record (outputs, via a product with an all-ones operand).
 constexpr float kOffLo = 1024.f, kOffHi = 64.f;
+constexpr float kMid8 = 128.f, kMid4 = 8.f;  // centres of the code ranges
 constexpr float kSlack = 8.f;  // log2 of the largest softmax weight before the reference is raised
 // Two codes held in bits 0-3 / 16-19 (lo) or 4-7 / 20-23 (hi) of w: (w & mask) | exponent as ONE three-input
 // logic op.  That needs mask and exponent in registers (the instruction takes a single immediate, and with two
@@ -226,7 +227,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
     const uint32_t never = p.capacity < 0 ? 1u : 0u;
     const NibbleConsts nc{0x000F000Fu ^ never, 0x64006400u ^ never, 0x00F000F0u ^ never, 0x54005400u ^ never};
     uint32_t qf[8][2];
-    float kq8[2], kq4[2], ko8[2], ko4[2], m_run[2], l[2], z8[2], z4[2], acc[8][4], ones8[4], ones4[4];
+    float kq8[2], kq4[2], ko8[2], ko4[2], m_run[2], l[2], z8[2], z4[2], acc[8][4], ones8[4], ones4[4], wx8[2], wx4[2];
     bool fresh = true, ok = true;
     long long i = 0;
     int stage = 0;
@@ -256,7 +257,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                 kq4[e] = kLog2eOverSqrtD * __shfl_sync(0xffffffffu, s4, 4 * (2 * c + e));
                 ko8[e] = kOffLo * kq8[e];
                 ko4[e] = kLog2eOverSqrtD * __shfl_sync(0xffffffffu, o4, 4 * (2 * c + e));
-                m_run[e] = -INFINITY; l[e] = z8[e] = z4[e] = ones8[e] = ones4[e] = ones8[2 + e] = ones4[2 + e] = 0.f;
+                m_run[e] = -INFINITY; l[e] = z8[e] = z4[e] = ones8[e] = ones4[e] = ones8[2 + e] = ones4[2 + e] = wx8[e] = wx4[e] = 0.f;
             }
 #pragma unroll
             for (int mt = 0; mt < 8; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
@@ -347,6 +348,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                     const float mn = fmaxf(m_run[e], mx);
                     const float a = ex2(m_run[e] - mn);
                     l[e] *= a; z8[e] *= a; z4[e] *= a; ones8[e] *= a; ones4[e] *= a; ones8[2 + e] *= a; ones4[2 + e] *= a;
+                    wx8[e] *= a; wx4[e] *= a;
 #pragma unroll
                     for (int mt = 0; mt < 8; ++mt) { acc[mt][e] *= a; acc[mt][2 + e] *= a; }
                     m_run[e] = mn;
@@ -366,6 +368,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                     const float w = pw * i2e;
                     l[e] += w; z8[e] = fmaf(w, v.z8, z8[e]); z4[e] = fmaf(w, v.z4, z4[e]);
                     p8[t][e] = pw * v.sn8; p4[t][e] = pw * v.sn4;
+                    wx8[e] += p8[t][e]; wx4[e] += p4[t][e];  // the unrounded weights, for the centring below
                 }
             const uint32_t b80 = movmatrix_trans(pack_h2(p8[0][0], p8[0][1])), b81 = movmatrix_trans(pack_h2(p8[1][0], p8[1][1]));
             const uint32_t b40 = movmatrix_trans(pack_h2(p4[0][0], p4[0][1])), b41 = movmatrix_trans(pack_h2(p4[1][0], p4[1][1]));
@@ -408,6 +411,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                     l[e] += __shfl_xor_sync(0xffffffffu, l[e], o);
                     z8[e] += __shfl_xor_sync(0xffffffffu, z8[e], o);
                     z4[e] += __shfl_xor_sync(0xffffffffu, z4[e], o);
+                    wx8[e] += __shfl_xor_sync(0xffffffffu, wx8[e], o);
+                    wx4[e] += __shfl_xor_sync(0xffffffffu, wx4[e], o);
                 }
             float* rec = p.partial + (wg + static_cast<long long>(cons.b) * p.n_kv_heads + cons.h) * kRecFloats;
 #pragma unroll
@@ -416,8 +421,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                 float* r = rec + (2 * c + e) * (kD + 2);
                 if (g == 0) { r[0] = m_run[e]; r[1] = l[e]; }
                 r += 2;
-                // rows g of the output products carry offset kOffLo, rows g + 8 kOffLo (8-bit) or kOffHi (4-bit)
-                const float f8 = z8[e] - kOffLo * ones8[e], f4lo = z4[e] - kOffLo * ones4[e], f4hi = z4[e] - kOffHi * ones4[e];
+                // Rows g of the output products carry offset kOffLo, rows g + 8 kOffLo (8-bit) or kOffHi (4-bit).  The
+                // codes are also centred: sum w^ (c - mid) + mid * sum w with w^ the half-rounded and w the exact
+                // weights (ones: sum w^, wx: sum w), which halves the effect of the rounding (|c - mid| <= range / 2).
+                const float f8 = z8[e] - (kOffLo + kMid8) * ones8[e] + kMid8 * wx8[e];
+                const float f4lo = z4[e] - (kOffLo + kMid4) * ones4[e] + kMid4 * wx4[e];
+                const float f4hi = z4[e] - (kOffHi + kMid4) * ones4[e] + kMid4 * wx4[e];
                 r[2 * g] = acc[0][e] + f8;
                 r[2 * g + 1] = acc[0][2 + e] + f8;
 #pragma unroll
