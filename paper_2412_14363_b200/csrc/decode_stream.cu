@@ -162,6 +162,16 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
     // Every weight byte is read once: mark the lines evict-first so that the activations, the scales
     // and whatever the neighbouring kernels keep in L2 stay there.
     const uint64_t stream_policy = l2_policy_evict_first();
+    // (w ^ kFlip) & kLo as ONE three-input logic op: the instruction takes a single immediate, so with two
+    // compile-time constants the assembler emits an XOR and an AND.  T is positive, which the compiler cannot know:
+    // the two words stay in registers.
+    const uint32_t never = p.T < 0 ? 1u : 0u;
+    const uint32_t rflip = kFlip ^ never, rlo = kLo ^ never;
+    auto even_codes = [&](uint32_t w) {
+        uint32_t d;
+        asm("lop3.b32 %0, %1, %2, %3, 0x28;" : "=r"(d) : "r"(w), "r"(rflip), "r"(rlo));  // (w ^ rflip) & rlo
+        return d;
+    };
     // Issue cursor of this warp (only lane 0 uses it): next (item, chunk) to copy.
     int is_idx = cb, is_item = cb / nchunks, is_chunk = cb - (cb / nchunks) * nchunks;
     auto issue = [&](int stage) {
@@ -387,9 +397,9 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
 #pragma unroll
                     for (int j = 0; j < 4; j += 2) {
                         mma_s8<ASYM>(accO[0], xo[j], yo[j], xo[j + 1], yo[j + 1], was[j] & kHi, was[j + 1] & kHi);
-                        mma_s8<ASYM>(accE[0], xe[j], ye[j], xe[j + 1], ye[j + 1], (was[j] ^ kFlip) & kLo, (was[j + 1] ^ kFlip) & kLo);
+                        mma_s8<ASYM>(accE[0], xe[j], ye[j], xe[j + 1], ye[j + 1], even_codes(was[j]), even_codes(was[j + 1]));
                         mma_s8<ASYM>(accO[1], xo[j], yo[j], xo[j + 1], yo[j + 1], wbs[j] & kHi, wbs[j + 1] & kHi);
-                        mma_s8<ASYM>(accE[1], xe[j], ye[j], xe[j + 1], ye[j + 1], (wbs[j] ^ kFlip) & kLo, (wbs[j + 1] ^ kFlip) & kLo);
+                        mma_s8<ASYM>(accE[1], xe[j], ye[j], xe[j + 1], ye[j + 1], even_codes(wbs[j]), even_codes(wbs[j + 1]));
                     }
                 }
             }
