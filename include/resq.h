@@ -101,6 +101,20 @@ int resq_pack_weights(const resq_layer_desc_t* desc, const float* W_proj, int8_t
                       void* s_w8, void* s_w4, int8_t* w4_i8, void* stream);
 
 /*
+ * Eq. 3 with the projection done here (Section 4.3: the bases are multiplied into the weights offline): W_raw is
+ * the unprojected weight as bf16 [n_out][K] (row n = the K input weights of output channel n), U the basis as
+ * bf16 [K][K] (row i = input feature, column j = coefficient, as P of resq_project_quantize).  Forms
+ * W_proj = W_raw·U = (U^T W)^T in fp32 on the tensor cores (bf16 products, fp32 accumulation), in panels of
+ * rows staged in the workspace, and quantizes it like resq_pack_weights (round to nearest; GPTQ is not built).
+ * Codes can differ by one step from those of an fp64 projection on a small fraction of elements, like the
+ * online activation path.  Workspace: resq_pack_projected_workspace_bytes(desc) bytes.
+ */
+size_t resq_pack_projected_workspace_bytes(const resq_layer_desc_t* desc);
+int resq_pack_weights_projected(const resq_layer_desc_t* desc, const void* W_raw, const void* U, int8_t* w8,
+                                uint8_t* w4, void* s_w8, void* s_w4, int8_t* w4_i8, void* workspace,
+                                size_t workspace_bytes, void* stream);
+
+/*
  * Eq. 2: per-token split quantization of the coefficients.
  *   P == NULL: the rows of X (bf16 [T][K]) already are the coefficients -- the projection was
  *              folded into the preceding layer's weights (Section 4.3, U_A/U_B).

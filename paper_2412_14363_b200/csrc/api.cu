@@ -126,6 +126,39 @@ int resq_pack_weights(const resq_layer_desc_t* d, const float* W_proj, int8_t* w
                                              static_cast<size_t>(d->K) * 4, static_cast<cudaStream_t>(stream)));
 }
 
+size_t resq_pack_projected_workspace_bytes(const resq_layer_desc_t* d) {
+    if (check_desc(d)) return 0;
+    return align_up(static_cast<size_t>(d->n_out < kPanelRows ? d->n_out : kPanelRows) * d->K * 4);
+}
+
+int resq_pack_weights_projected(const resq_layer_desc_t* d, const void* W_raw, const void* U, int8_t* w8, uint8_t* w4,
+                                void* s_w8, void* s_w4, int8_t* w4_i8, void* workspace, size_t workspace_bytes,
+                                void* stream) {
+    if (int e = check_desc(d)) return e;
+    if (!W_raw || !U || (!w8 && d->r > 0) || !w4 || !s_w8 || !s_w4) return RESQ_ERR_NULL;
+    if (!aligned16(W_raw) || !aligned16(U) || !aligned16(w8) || !aligned16(w4) || !aligned16(s_w8) ||
+        !aligned16(s_w4) || !aligned16(w4_i8) || !aligned16(workspace))
+        return RESQ_ERR_ALIGN;
+    if (!workspace || workspace_bytes < resq_pack_projected_workspace_bytes(d)) return RESQ_ERR_WORKSPACE;
+    if (int e = check_arch()) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* panel = static_cast<float*>(workspace);
+    const size_t K = static_cast<size_t>(d->K), K4 = static_cast<size_t>(d->K - d->r);
+    const size_t sb = d->w_scale_dtype == RESQ_SCALE_FP16 ? 2 : 4;
+    for (int n0 = 0; n0 < d->n_out; n0 += kPanelRows) {
+        const int rows = d->n_out - n0 < kPanelRows ? d->n_out - n0 : kPanelRows;
+        const char* Wp = static_cast<const char*>(W_raw) + static_cast<size_t>(n0) * K * 2;
+        if (cudaError_t e = launch_project_gemm(Wp, U, rows, d->K, panel, st); e != cudaSuccess) return cuda_status(e);
+        if (cudaError_t e = launch_split_quantize(
+                panel, true, rows, d->K, d->r, w8 ? w8 + static_cast<size_t>(n0) * d->r : nullptr, w4 + n0 * K4 / 2,
+                static_cast<char*>(s_w8) + n0 * sb, static_cast<char*>(s_w4) + n0 * sb, sb == 2,
+                w4_i8 ? w4_i8 + n0 * K4 : nullptr, K * 4, st);
+            e != cudaSuccess)
+            return cuda_status(e);
+    }
+    return RESQ_OK;
+}
+
 int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int8_t* x8, uint8_t* x4, float* s_x8,
                           float* s_x4, int8_t* x4_i8, void* workspace, size_t workspace_bytes, void* stream) {
     if (T < 1) return RESQ_ERR_SHAPE;

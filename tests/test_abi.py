@@ -31,6 +31,19 @@ def test_library_exports_every_declared_symbol(resq):
     assert sorted(resq.EXPORTS) == names
 
 
+def test_pack_projected_host_validation(resq):
+    L = resq.lib
+    import ctypes
+    d = resq.layer_desc(512, 64, 64)
+    fake = 1 << 20
+    need = L.resq_pack_projected_workspace_bytes(ctypes.byref(d))
+    assert need == 64 * 512 * 4
+    assert L.resq_pack_projected_workspace_bytes(ctypes.byref(resq.layer_desc(500, 64, 64))) == 0
+    assert L.resq_pack_weights_projected(ctypes.byref(d), fake, None, fake, fake, fake, fake, None, fake, need, None) == resq.ERR_NULL
+    assert L.resq_pack_weights_projected(ctypes.byref(d), fake, fake, fake, fake, fake, fake, None, fake, need - 1, None) == resq.ERR_WORKSPACE
+    assert L.resq_pack_weights_projected(ctypes.byref(d), fake + 2, fake, fake, fake, fake, fake, None, fake, need, None) == resq.ERR_ALIGN
+
+
 def test_every_header_is_covered():
     assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["resq.h", "resq_kv.h"]
 

@@ -101,3 +101,28 @@ def test_projection_alone_against_fp64_sums(resq, T, K):
     Pf = np.abs(synth.bf16_bits_to_f32(P_bits).astype(np.float64))
     bound = (K // 16 + 4) * 2.0 ** -24 * (Xf @ Pf) + 1e-30
     assert (np.abs(host(C).astype(np.float64) - C_ref.astype(np.float64)) <= bound).all()
+
+
+@pytest.mark.parametrize("N,K,r,fp16", [(64, 512, 64, False), (4104, 1024, 128, False), (264, 2048, 256, True)])
+def test_pack_weights_projected(resq, N, K, r, fp16):
+    """Weight projection at pack time (Section 4.3): W_raw·U on the tensor cores, then Eq. 3.  Against the oracle's
+    fp64-summed projection: codes within +-1 on at most 0.1 %, scales within the same ulp bound as the online
+    activation path; the one-code-per-byte copy and the packed nibbles agree with each other bit for bit."""
+    W_bits = synth.f32_to_bf16_bits(synth.weights(K, N, seed=77).T.copy())          # [N][K]: rows = output channels
+    U_bits = synth.f32_to_bf16_bits(synth.kron_orthogonal_bf16(K, inner=128))
+    pw = oracle.pack_weights(oracle.project(W_bits, U_bits), r, scale_fp16=fp16)
+    desc = resq.layer_desc(K, N, r, resq.SCALE_FP16 if fp16 else resq.SCALE_FP32)
+    W = resq.resq_pack_weights_projected(desc, bf16_to_dev(W_bits), bf16_to_dev(U_bits))
+    assert resq.resq_device_status() == resq.OK
+    g8, g4 = host(W.w8).astype(np.int32), host(W.w4_i8).astype(np.int32)
+    assert (host(W.w4) == oracle.pack_nibbles(host(W.w4_i8))).all()
+    assert np.abs(g8 - pw.q8).max() <= 1 and np.abs(g4 - pw.q4).max() <= 1
+    frac = ((g8 != pw.q8).sum() + (g4 != pw.q4).sum()) / float(N * K)
+    assert frac <= 1e-3, frac
+    if fp16:
+        d8 = np.abs(host(W.s_w8).view(np.int16).astype(np.int32) - pw.s8.astype(np.float16).view(np.int16).astype(np.int32))
+        d4 = np.abs(host(W.s_w4).view(np.int16).astype(np.int32) - pw.s4.astype(np.float16).view(np.int16).astype(np.int32))
+        assert d8.max() <= 1 and d4.max() <= 1
+    else:
+        tol = K // 16 + 4
+        assert _ulp_diff(host(W.s_w8), pw.s8).max() <= tol and _ulp_diff(host(W.s_w4), pw.s4).max() <= tol
