@@ -433,6 +433,7 @@ def kv_leg(resq, torch, dev, peaks, steps, n_seqs=16, seq_len=8192, prefill_T=40
     pos1 = torch.full((n_seqs,), seq_len - 1, dtype=torch.int32, device=dev)
     app1_ms = timed(lambda i: kv.resq_kv_append(caches[i % 2], k1, v1, ids1, pos1, wq, s_u), steps)
     qp1_ms = timed(lambda i: kv.resq_query_project(q, wq, s_u, q16), steps)
+    fused1_ms = timed(lambda i: kv.resq_qkv_project_append(caches[i % 2], q, q16, k1, v1, ids1, pos1, wq, s_u), steps)
     # prefill-sized update: prefill_T tokens of one sequence
     T = min(prefill_T, seq_len)
     kp = synth.t_head_vectors(T, KV_HKV, KV_D, dev, stream=3003, lead=1.0)
@@ -453,6 +454,7 @@ def kv_leg(resq, torch, dev, peaks, steps, n_seqs=16, seq_len=8192, prefill_T=40
             "attention_decode_us": round(attn_ms * 1e3, 2), "attention_cache_stream_gbs": round(gbs, 1),
             "attention_frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
             "decode_step_kv_append_us": round(app1_ms * 1e3, 2), "decode_step_query_project_us": round(qp1_ms * 1e3, 2),
+            "decode_step_fused_project_append_us": round(fused1_ms * 1e3, 2),
             "prefill_tokens": T, "prefill_kv_append_us": round(appp_ms * 1e3, 2),
             "prefill_kv_append_gbs": round(app_bytes / (appp_ms * 1e-3) / 1e9, 1),
             "prefill_query_project_us": round(qpp_ms * 1e3, 2),

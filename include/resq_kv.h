@@ -88,6 +88,13 @@ int resq_query_project(const void* q, int64_t rows, int d_head, const int8_t* wq
 int resq_kv_append(const resq_kv_cache_t* cache, const void* k, const void* v, int64_t T, const int32_t* seq_ids,
                    const int32_t* positions, const int8_t* wq, const float* s_u, void* stream);
 
+/* resq_query_project and resq_kv_append of the same T tokens in one launch (q bf16 [T][n_q_heads][d_head]): the
+ * query, key and value head vectors are independent pieces of work, so a generation step's few of them run side
+ * by side instead of as two short kernels one after the other. */
+int resq_qkv_project_append(const resq_kv_cache_t* cache, const void* q, int n_q_heads, void* q_out, const void* k,
+                            const void* v, int64_t T, const int32_t* seq_ids, const int32_t* positions,
+                            const int8_t* wq, const float* s_u, void* stream);
+
 /* Scratch bytes of resq_attention_decode (0 for an invalid geometry). */
 size_t resq_attention_workspace_bytes(int n_seqs, int n_q_heads, int n_kv_heads, int d_head);
 

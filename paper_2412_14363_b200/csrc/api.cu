@@ -491,7 +491,8 @@ int resq_query_project(const void* q, int64_t rows, int d_head, const int8_t* wq
     if (!q || !wq || !s_u || !q_out) return RESQ_ERR_NULL;
     if (!aligned16(q) || !aligned16(wq) || !aligned16(s_u) || !aligned16(q_out)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
-    return cuda_status(launch_query_project(q, rows, wq, s_u, q_out, static_cast<cudaStream_t>(stream)));
+    return cuda_status(launch_qkv_project_append(nullptr, q, rows, q_out, nullptr, nullptr, 0, nullptr, nullptr, wq, s_u,
+                                                 static_cast<cudaStream_t>(stream)));
 }
 
 int resq_kv_append(const resq_kv_cache_t* cache, const void* k, const void* v, int64_t T, const int32_t* seq_ids,
@@ -501,7 +502,21 @@ int resq_kv_append(const resq_kv_cache_t* cache, const void* k, const void* v, i
     if (!k || !v || !seq_ids || !positions || !wq || !s_u) return RESQ_ERR_NULL;
     if (!aligned16(k) || !aligned16(v) || !aligned16(wq) || !aligned16(s_u)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
-    return cuda_status(launch_kv_append(*cache, k, v, T, seq_ids, positions, wq, s_u, static_cast<cudaStream_t>(stream)));
+    return cuda_status(launch_qkv_project_append(cache, nullptr, 0, nullptr, k, v, T, seq_ids, positions, wq, s_u,
+                                                 static_cast<cudaStream_t>(stream)));
+}
+
+int resq_qkv_project_append(const resq_kv_cache_t* cache, const void* q, int n_q_heads, void* q_out, const void* k,
+                            const void* v, int64_t T, const int32_t* seq_ids, const int32_t* positions,
+                            const int8_t* wq, const float* s_u, void* stream) {
+    if (int e = check_cache(cache)) return e;
+    if (T < 0 || n_q_heads < 1) return RESQ_ERR_SHAPE;
+    if (!q || !q_out || !k || !v || !seq_ids || !positions || !wq || !s_u) return RESQ_ERR_NULL;
+    if (!aligned16(q) || !aligned16(q_out) || !aligned16(k) || !aligned16(v) || !aligned16(wq) || !aligned16(s_u))
+        return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_qkv_project_append(cache, q, T * n_q_heads, q_out, k, v, T, seq_ids, positions, wq, s_u,
+                                                 static_cast<cudaStream_t>(stream)));
 }
 
 size_t resq_attention_workspace_bytes(int n_seqs, int n_q_heads, int n_kv_heads, int d_head) {

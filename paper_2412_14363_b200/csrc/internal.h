@@ -76,11 +76,10 @@ int pick_tile_width(int m_tiles, int N, int sms);
 
 // ---- attention-block path (declared in resq_kv.h) ----
 cudaError_t launch_uc_quantize(const float* W_C, int8_t* wq, float* s_u, cudaStream_t st);
-cudaError_t launch_query_project(const void* q, long long rows, const int8_t* wq, const float* s_u, void* q_out,
-                                 cudaStream_t st);
-cudaError_t launch_kv_append(const resq_kv_cache_t& cache, const void* k, const void* v, long long T,
-                             const int32_t* seq_ids, const int32_t* positions, const int8_t* wq, const float* s_u,
-                             cudaStream_t st);
+// Query projection and / or cache update in one launch (either part may be absent: q == NULL, or k == NULL).
+cudaError_t launch_qkv_project_append(const resq_kv_cache_t* cache, const void* q, long long q_rows, void* q_out,
+                                      const void* k, const void* v, long long T, const int32_t* seq_ids,
+                                      const int32_t* positions, const int8_t* wq, const float* s_u, cudaStream_t st);
 size_t attention_scratch_bytes(int n_seqs, int n_kv_heads);
 cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q16, int n_q_heads, const int32_t* seq_lens,
                                     float* out, void* scratch, cudaStream_t st);

@@ -139,38 +139,98 @@ __device__ __forceinline__ void sym8_fragments(const float (&xv)[2][32], uint32_
     }
 }
 
-// KEY = false: q_out[row] = half(x U_C).  KEY = true: the key rows are projected, quantized and appended, then the
-// value rows of the same tokens are quantized and appended.
-template <bool KEY>
-__global__ void __launch_bounds__(kWarps * 32)
-kv_project_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ v, long long rows,
-                  const int8_t* __restrict__ wq, const float* __restrict__ s_u, __half* __restrict__ q_out,
-                  uint8_t* __restrict__ cache, int n_seqs, int n_kv_heads, int capacity,
-                  const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ positions, int* status) {
+struct ProjectParams {
+    const __nv_bfloat16* q;  // [q_rows][128] or null
+    const __nv_bfloat16* k;  // [kv_rows][128] or null
+    const __nv_bfloat16* v;
+    long long q_rows, kv_rows;
+    const int8_t* wq;
+    const float* s_u;
+    __half* q_out;
+    uint8_t* cache;
+    int n_seqs, n_kv_heads, capacity;
+    const int32_t* seq_ids;
+    const int32_t* positions;
+    int* status;
+};
+
+// Asymmetric 8/4-bit codes of one row held by a quad: the lane's n8 values of the 8-bit segment and n4 of the
+// 4-bit one.  Returns the two quantizers (min / max reduced over the quad).
+template <int N8, int N4>
+__device__ __forceinline__ void quad_ranges(const float* v8, const float* v4, float (&lohi)[4]) {
+    float lo8 = 3.402823466e38f, hi8 = -3.402823466e38f, lo4 = lo8, hi4 = hi8;
+#pragma unroll
+    for (int i = 0; i < N8; ++i) { lo8 = fminf(lo8, v8[i]); hi8 = fmaxf(hi8, v8[i]); }
+#pragma unroll
+    for (int i = 0; i < N4; ++i) { lo4 = fminf(lo4, v4[i]); hi4 = fmaxf(hi4, v4[i]); }
+    lohi[0] = quad_min(lo8); lohi[1] = quad_max(hi8); lohi[2] = quad_min(lo4); lohi[3] = quad_max(hi4);
+}
+
+// One warp per tile of 16 head vectors; the tiles of a call are the query tiles (projected, written as half),
+// then the key tiles (projected, quantized, appended), then the value tiles (quantized, appended) -- three
+// independent kinds, so a generation step's few tiles spread over as many warps and run side by side.
+__global__ void __launch_bounds__(kWarps * 32) kv_project_kernel(const ProjectParams p) {
     __shared__ __align__(16) uint8_t w_s[kD * kWStride];
     __shared__ float su_s[kD];
-    __shared__ __align__(16) uint8_t rec_s[KEY ? kWarps : 1][16 * kRec];
-    __shared__ long long slot_s[KEY ? kWarps : 1][16];
+    __shared__ __align__(16) uint8_t rec_s[kWarps][16 * kRec];
+    __shared__ long long slot_s[kWarps][16];
     for (int i = threadIdx.x; i < kD * 8; i += blockDim.x) {  // 16-byte pieces of W_C's codes
-        const int n = i >> 3, p = i & 7;
-        *reinterpret_cast<uint4*>(w_s + n * kWStride + p * 16) = __ldg(reinterpret_cast<const uint4*>(wq + n * kD) + p);
+        const int n = i >> 3, pc = i & 7;
+        *reinterpret_cast<uint4*>(w_s + n * kWStride + pc * 16) = __ldg(reinterpret_cast<const uint4*>(p.wq + n * kD) + pc);
     }
-    for (int i = threadIdx.x; i < kD; i += blockDim.x) su_s[i] = s_u[i];
+    for (int i = threadIdx.x; i < kD; i += blockDim.x) su_s[i] = p.s_u[i];
     __syncthreads();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
-    const long long tiles = (rows + 15) / 16;
+    const long long q_tiles = (p.q_rows + 15) / 16, kv_tiles = (p.kv_rows + 15) / 16, tiles = q_tiles + 2 * kv_tiles;
+    uint8_t* rec = rec_s[warp];
     for (long long tile = static_cast<long long>(blockIdx.x) * kWarps + warp; tile < tiles;
          tile += static_cast<long long>(gridDim.x) * kWarps) {
-        const long long r0 = tile * 16 + g, r1 = r0 + 8;
+        const int kind = tile < q_tiles ? 0 : (tile < q_tiles + kv_tiles ? 1 : 2);  // query, key, value
+        const long long t0 = kind == 0 ? tile : (kind == 1 ? tile - q_tiles : tile - q_tiles - kv_tiles);
+        const long long rows = kind == 0 ? p.q_rows : p.kv_rows;
+        const __nv_bfloat16* x = kind == 0 ? p.q : (kind == 1 ? p.k : p.v);
+        const long long r0 = t0 * 16 + g, r1 = r0 + 8;
         const bool live0 = r0 < rows, live1 = r1 < rows;
         float xv[2][32];
         load_row(x + r0 * kD, c, live0, xv[0]);
         load_row(x + r1 * kD, c, live1, xv[1]);
-        if (KEY && lane < 16) {
-            const long long r = tile * 16 + lane;
-            slot_s[KEY ? warp : 0][lane] =
-                r < rows ? cache_slot(r, n_kv_heads, n_seqs, capacity, seq_ids, positions, status) : -1;
+        if (kind != 0 && lane < 16) {
+            const long long r = t0 * 16 + lane;
+            slot_s[warp][lane] = r < rows ? cache_slot(r, p.n_kv_heads, p.n_seqs, p.capacity, p.seq_ids, p.positions, p.status) : -1;
+        }
+        if (kind == 2) {
+            // ---- value: the bf16 head vectors quantized directly; elements 0-3 of the lane are columns
+            // [4c, 4c + 4), the 8-bit segment
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                float lohi[4];
+                quad_ranges<4, 28>(xv[rr], xv[rr] + 4, lohi);
+                const Asym q8(lohi[0], lohi[1], 255.f), q4(lohi[2], lohi[3], 15.f);
+                uint8_t* rrow = rec + (g + 8 * rr) * kRec;
+                uint32_t w8 = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) w8 |= q8.code(xv[rr][i], 255.f) << (8 * i);
+                *reinterpret_cast<uint32_t*>(rrow + 4 * c) = w8;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf) {
+                        if (ks == 0 && hf == 0) continue;
+                        const float* e = xv[rr] + 8 * ks + 4 * hf;
+                        const int col = 32 * ks + 16 * hf + 4 * c;  // >= 16
+                        *reinterpret_cast<uint16_t*>(rrow + 16 + (col - 16) / 2) = static_cast<uint16_t>(
+                            q4.code(e[0], 15.f) | (q4.code(e[1], 15.f) << 4) | (q4.code(e[2], 15.f) << 8) | (q4.code(e[3], 15.f) << 12));
+                    }
+                if (c == 0) {
+                    float* m = reinterpret_cast<float*>(rrow + 72);
+                    m[0] = q8.s; m[1] = q8.z; m[2] = q4.s; m[3] = q4.z;
+                }
+            }
+            __syncwarp();
+            flush_records(rec, slot_s[warp], p.cache, 1, lane);
+            __syncwarp();
+            continue;
         }
         float sx[2];
         uint32_t a[4][4];
@@ -187,88 +247,48 @@ kv_project_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __re
                        *reinterpret_cast<const uint32_t*>(wrow + 32 * ks + 16));
         }
         // y[row g][8 nt + 2c + e] = acc[nt][e], y[row g + 8][...] = acc[nt][2 + e]
-        if (!KEY) {
+        if (kind == 0) {
 #pragma unroll
             for (int nt = 0; nt < 16; ++nt) {
                 const float u0 = su_s[8 * nt + 2 * c], u1 = su_s[8 * nt + 2 * c + 1];
                 if (live0)
-                    *reinterpret_cast<__half2*>(q_out + r0 * kD + 8 * nt + 2 * c) = __floats2half2_rn(
+                    *reinterpret_cast<__half2*>(p.q_out + r0 * kD + 8 * nt + 2 * c) = __floats2half2_rn(
                         __fmul_rn(static_cast<float>(acc[nt][0]), __fmul_rn(sx[0], u0)),
                         __fmul_rn(static_cast<float>(acc[nt][1]), __fmul_rn(sx[0], u1)));
                 if (live1)
-                    *reinterpret_cast<__half2*>(q_out + r1 * kD + 8 * nt + 2 * c) = __floats2half2_rn(
+                    *reinterpret_cast<__half2*>(p.q_out + r1 * kD + 8 * nt + 2 * c) = __floats2half2_rn(
                         __fmul_rn(static_cast<float>(acc[nt][2]), __fmul_rn(sx[1], u0)),
                         __fmul_rn(static_cast<float>(acc[nt][3]), __fmul_rn(sx[1], u1)));
             }
             continue;
         }
-        uint8_t* rec = rec_s[KEY ? warp : 0];
         // ---- key: asymmetric 8/4-bit codes of the fp32 coefficients (column tiles 0-1 are the 8-bit segment)
 #pragma unroll
         for (int rr = 0; rr < 2; ++rr) {
-            float y[16][2];
-            float lo8 = 3.402823466e38f, hi8 = -3.402823466e38f, lo4 = lo8, hi4 = hi8;
+            float y[32];  // y[2 nt + e]
 #pragma unroll
             for (int nt = 0; nt < 16; ++nt)
 #pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const float val = __fmul_rn(static_cast<float>(acc[nt][2 * rr + e]),
-                                                __fmul_rn(sx[rr], su_s[8 * nt + 2 * c + e]));
-                    y[nt][e] = val;
-                    if (nt < 2) { lo8 = fminf(lo8, val); hi8 = fmaxf(hi8, val); }
-                    else { lo4 = fminf(lo4, val); hi4 = fmaxf(hi4, val); }
-                }
-            const Asym q8(quad_min(lo8), quad_max(hi8), 255.f), q4(quad_min(lo4), quad_max(hi4), 15.f);
+                for (int e = 0; e < 2; ++e)
+                    y[2 * nt + e] = __fmul_rn(static_cast<float>(acc[nt][2 * rr + e]), __fmul_rn(sx[rr], su_s[8 * nt + 2 * c + e]));
+            float lohi[4];
+            quad_ranges<4, 28>(y, y + 4, lohi);
+            const Asym q8(lohi[0], lohi[1], 255.f), q4(lohi[2], lohi[3], 15.f);
             uint8_t* rrow = rec + (g + 8 * rr) * kRec;
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt)
                 *reinterpret_cast<uint16_t*>(rrow + 8 * nt + 2 * c) =
-                    static_cast<uint16_t>(q8.code(y[nt][0], 255.f) | (q8.code(y[nt][1], 255.f) << 8));
+                    static_cast<uint16_t>(q8.code(y[2 * nt], 255.f) | (q8.code(y[2 * nt + 1], 255.f) << 8));
 #pragma unroll
             for (int nt = 2; nt < 16; ++nt)
-                rrow[16 + 4 * (nt - 2) + c] = static_cast<uint8_t>(q4.code(y[nt][0], 15.f) | (q4.code(y[nt][1], 15.f) << 4));
+                rrow[16 + 4 * (nt - 2) + c] = static_cast<uint8_t>(q4.code(y[2 * nt], 15.f) | (q4.code(y[2 * nt + 1], 15.f) << 4));
             if (c == 0) {
                 float* m = reinterpret_cast<float*>(rrow + 72);
                 m[0] = q8.s; m[1] = q8.z; m[2] = q4.s; m[3] = q4.z;
             }
         }
         __syncwarp();
-        flush_records(rec, slot_s[KEY ? warp : 0], cache, 0, lane);
-        __syncwarp();
-        // ---- value: the bf16 head vectors of the same rows, quantized directly
-        load_row(v + r0 * kD, c, live0, xv[0]);
-        load_row(v + r1 * kD, c, live1, xv[1]);
-#pragma unroll
-        for (int rr = 0; rr < 2; ++rr) {
-            float lo8 = 3.402823466e38f, hi8 = -3.402823466e38f, lo4 = lo8, hi4 = hi8;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {  // elements 0-3 of the lane are columns [4c, 4c + 4): the 8-bit segment
-                if (i < 4) { lo8 = fminf(lo8, xv[rr][i]); hi8 = fmaxf(hi8, xv[rr][i]); }
-                else { lo4 = fminf(lo4, xv[rr][i]); hi4 = fmaxf(hi4, xv[rr][i]); }
-            }
-            const Asym q8(quad_min(lo8), quad_max(hi8), 255.f), q4(quad_min(lo4), quad_max(hi4), 15.f);
-            uint8_t* rrow = rec + (g + 8 * rr) * kRec;
-            uint32_t w8 = 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) w8 |= q8.code(xv[rr][i], 255.f) << (8 * i);
-            *reinterpret_cast<uint32_t*>(rrow + 4 * c) = w8;
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    if (ks == 0 && hf == 0) continue;
-                    const float* e = xv[rr] + 8 * ks + 4 * hf;
-                    const int col = 32 * ks + 16 * hf + 4 * c;  // >= 16
-                    *reinterpret_cast<uint16_t*>(rrow + 16 + (col - 16) / 2) = static_cast<uint16_t>(
-                        q4.code(e[0], 15.f) | (q4.code(e[1], 15.f) << 4) | (q4.code(e[2], 15.f) << 8) | (q4.code(e[3], 15.f) << 12));
-                }
-            if (c == 0) {
-                float* m = reinterpret_cast<float*>(rrow + 72);
-                m[0] = q8.s; m[1] = q8.z; m[2] = q4.s; m[3] = q4.z;
-            }
-        }
-        __syncwarp();
-        flush_records(rec, slot_s[KEY ? warp : 0], cache, 1, lane);
+        flush_records(rec, slot_s[warp], p.cache, 0, lane);
         __syncwarp();
     }
 }
@@ -293,9 +313,16 @@ __global__ void __launch_bounds__(32) uc_quantize_kernel(const float* __restrict
     if (lane == 0) s_u[row] = s;
 }
 
-int grid_for(long long rows) {
-    const long long tiles = (rows + 15) / 16, ctas = (tiles + kWarps - 1) / kWarps;
+int grid_for(long long tiles) {
+    const long long ctas = (tiles + kWarps - 1) / kWarps;
     return static_cast<int>(ctas < 148 * 8 ? (ctas > 0 ? ctas : 1) : 148 * 8);
+}
+
+cudaError_t launch_project(const ProjectParams& p, cudaStream_t st) {
+    const long long tiles = (p.q_rows + 15) / 16 + 2 * ((p.kv_rows + 15) / 16);
+    if (tiles == 0) return cudaSuccess;
+    kv_project_kernel<<<grid_for(tiles), kWarps * 32, 0, st>>>(p);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -305,25 +332,29 @@ cudaError_t launch_uc_quantize(const float* W_C, int8_t* wq, float* s_u, cudaStr
     return cudaGetLastError();
 }
 
-cudaError_t launch_query_project(const void* q, long long rows, const int8_t* wq, const float* s_u, void* q_out,
-                                 cudaStream_t st) {
-    if (rows == 0) return cudaSuccess;
-    kv_project_kernel<false><<<grid_for(rows), kWarps * 32, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(q), nullptr, rows, wq, s_u, static_cast<__half*>(q_out), nullptr, 0, 1, 0,
-        nullptr, nullptr, device_status_ptr());
-    return cudaGetLastError();
-}
-
-cudaError_t launch_kv_append(const resq_kv_cache_t& cache, const void* k, const void* v, long long T,
-                             const int32_t* seq_ids, const int32_t* positions, const int8_t* wq, const float* s_u,
-                             cudaStream_t st) {
-    if (T == 0) return cudaSuccess;
-    const long long rows = T * cache.n_kv_heads;
-    kv_project_kernel<true><<<grid_for(rows), kWarps * 32, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), rows, wq, s_u, nullptr,
-        static_cast<uint8_t*>(cache.data), cache.n_seqs, cache.n_kv_heads, cache.capacity, seq_ids, positions,
-        device_status_ptr());
-    return cudaGetLastError();
+// q (q_rows head vectors) and / or k, v (T tokens) in one launch; either part may be absent (null / 0).
+cudaError_t launch_qkv_project_append(const resq_kv_cache_t* cache, const void* q, long long q_rows, void* q_out,
+                                      const void* k, const void* v, long long T, const int32_t* seq_ids,
+                                      const int32_t* positions, const int8_t* wq, const float* s_u, cudaStream_t st) {
+    ProjectParams p{};
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.q_rows = q ? q_rows : 0;
+    p.q_out = static_cast<__half*>(q_out);
+    p.wq = wq;
+    p.s_u = s_u;
+    p.status = device_status_ptr();
+    if (cache && k) {
+        p.k = static_cast<const __nv_bfloat16*>(k);
+        p.v = static_cast<const __nv_bfloat16*>(v);
+        p.kv_rows = T * cache->n_kv_heads;
+        p.cache = static_cast<uint8_t*>(cache->data);
+        p.n_seqs = cache->n_seqs;
+        p.n_kv_heads = cache->n_kv_heads;
+        p.capacity = cache->capacity;
+        p.seq_ids = seq_ids;
+        p.positions = positions;
+    }
+    return launch_project(p, st);
 }
 
 }  // namespace resq

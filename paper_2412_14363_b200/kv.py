@@ -7,7 +7,7 @@ from . import ERR_CUDA, OK, ResqError, _check, _ptr, _stream, lib  # noqa: F401
 
 KV_BLOCK, KV_BLOCK_BYTES = 32, 5632
 ERR_INDEX = 8
-KV_EXPORTS = ["resq_kv_cache_bytes", "resq_uc_quantize", "resq_query_project", "resq_kv_append",
+KV_EXPORTS = ["resq_kv_cache_bytes", "resq_uc_quantize", "resq_query_project", "resq_kv_append", "resq_qkv_project_append",
               "resq_attention_workspace_bytes", "resq_attention_decode"]
 
 
@@ -23,6 +23,7 @@ lib.resq_kv_cache_bytes.argtypes = [_i, _i, _i, _i]
 lib.resq_uc_quantize.argtypes = [_vp, _i, _vp, _vp, _vp]
 lib.resq_query_project.argtypes = [_vp, _i64, _i, _vp, _vp, _vp, _vp]
 lib.resq_kv_append.argtypes = [_cp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
+lib.resq_qkv_project_append.argtypes = [_cp, _vp, _i, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
 lib.resq_attention_workspace_bytes.restype = _sz
 lib.resq_attention_workspace_bytes.argtypes = [_i, _i, _i, _i]
 lib.resq_attention_decode.argtypes = [_cp, _vp, _i, _vp, _vp, _vp, _sz, _vp]
@@ -66,6 +67,13 @@ def resq_kv_append(cache: KvCache, k, v, seq_ids, positions, wq, s_u):
     """k, v bf16 [T][n_kv_heads][128]; seq_ids, positions int32 [T]."""
     _check(lib.resq_kv_append(ctypes.byref(cache.c), _ptr(k), _ptr(v), k.shape[0], _ptr(seq_ids), _ptr(positions),
                               _ptr(wq), _ptr(s_u), _stream()), "resq_kv_append")
+
+
+def resq_qkv_project_append(cache: KvCache, q, q_out, k, v, seq_ids, positions, wq, s_u):
+    """q bf16 [T][n_q_heads][128] -> q_out half; k, v bf16 [T][n_kv_heads][128] appended; one launch."""
+    _check(lib.resq_qkv_project_append(ctypes.byref(cache.c), _ptr(q), q.shape[1], _ptr(q_out), _ptr(k), _ptr(v),
+                                       k.shape[0], _ptr(seq_ids), _ptr(positions), _ptr(wq), _ptr(s_u), _stream()),
+           "resq_qkv_project_append")
 
 
 def attention_workspace(cache: KvCache, n_q_heads: int):

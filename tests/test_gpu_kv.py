@@ -116,6 +116,29 @@ def test_kv_append_decode_step_and_bad_index(resq, kv, uc):
     assert (image[seq_ids[4]] == 0).all()
 
 
+def test_fused_project_append_matches_the_two_calls(resq, kv, uc):
+    """resq_qkv_project_append writes the same bytes as resq_query_project + resq_kv_append (a generation step:
+    one token for each of 5 sequences, and a ragged prefill of 37 tokens)."""
+    W_C, wq, s_u = uc
+    for T, Hq, Hkv, seq, pos in ((5, 8, 2, np.arange(5), np.array([9, 0, 31, 32, 63])), (37, 4, 4, np.zeros(37), np.arange(20, 57))):
+        q = bf16_to_dev(synth.f32_to_bf16_bits(synth.head_vectors(T, Hq, D, stream=700 + T, lead=1.0)))
+        k = bf16_to_dev(synth.f32_to_bf16_bits(synth.head_vectors(T, Hkv, D, stream=710 + T, lead=1.0)))
+        v = bf16_to_dev(synth.f32_to_bf16_bits(synth.head_vectors(T, Hkv, D, stream=720 + T)))
+        seq_ids, positions = dev(seq.astype(np.int32)), dev(pos.astype(np.int32))
+        ca, cb = kv.KvCache(5, Hkv, 64), kv.KvCache(5, Hkv, 64)
+        ca.data.fill_(7)
+        cb.data.fill_(7)
+        qa = torch.empty((T, Hq, D), dtype=torch.float16, device="cuda")
+        qb = torch.empty_like(qa)
+        kv.resq_query_project(q, wq, s_u, qa)
+        kv.resq_kv_append(ca, k, v, seq_ids, positions, wq, s_u)
+        kv.resq_qkv_project_append(cb, q, qb, k, v, seq_ids, positions, wq, s_u)
+        assert resq.resq_device_status() == resq.OK
+        assert (host(qa).view(np.uint16) == host(qb).view(np.uint16)).all()
+        assert (host(ca.data) == host(cb.data)).all()
+        assert (host(ca.data) != 7).any()
+
+
 def _attention_case(kv, seq_lens, Hq, Hkv, capacity, seed, v_scale=1.0, v_shift=0.3, fill=0xFF):
     """Cache image built on the CPU from the oracle's codes (no GPU kernel upstream), attention on both sides."""
     B = len(seq_lens)
