@@ -89,3 +89,63 @@ def test_down_proj_full_size_sampled_rows(resq, T, K, N):
     y32, ybf = oracle.epilogue(acc8, acc4, gs8, gs4, pw.s8, pw.s4)
     res = oracle.LayerResult(None, g8, g4, oracle.pack_nibbles(g4), gs8, gs4, acc8, acc4, y32, ybf)
     check_output(res, pw, host(Y[idx]))
+
+
+def test_attention_full_size_sampled_heads():
+    """The attention-block path at the benchmark's size (Llama-3-8B geometry: 32 query / 8 KV heads, 16 sequences x
+    8192 cached positions, 184.5 MB of cache), cache filled through resq_kv_append as the benchmark does.  For two
+    sampled sequences the oracle recomputes every cache byte (bit for bit) and single-query attention of sampled
+    query heads (within 1e-3 of the value magnitude, as in the small tests)."""
+    import paper_2412_14363_b200 as resq
+    from oracle import kv as okv
+    from paper_2412_14363_b200 import kv
+    from tests import kv_util
+    from tests.gpu_util import dev as to_dev
+
+    B, S, Hq, Hkv, D = 16, 8192, 32, 8, 128
+    device = torch.device("cuda")
+    W_C = np.ascontiguousarray(synth.haar_orthogonal(D).T.astype(np.float32))
+    wq, s_u = kv.resq_uc_quantize(to_dev(W_C))
+    cache = kv.KvCache(B, Hkv, S)
+    cache.data.fill_(0xFF)
+    pos = torch.arange(S, dtype=torch.int32, device=device)
+    sampled = (3, 15)
+    kept = {}
+    for b in range(B):
+        k = synth.t_head_vectors(S, Hkv, D, device, stream=1000 + b, lead=1.0, scale=1.5)
+        v = synth.t_head_vectors(S, Hkv, D, device, stream=2000 + b, lead=4.0, shift=0.2)
+        kv.resq_kv_append(cache, k, v, torch.full((S,), b, dtype=torch.int32, device=device), pos, wq, s_u)
+        if b in sampled:
+            kept[b] = (synth.bf16_bits_to_f32(_bits(k)), synth.bf16_bits_to_f32(_bits(v)))
+    lens = np.full(B, S, np.int32)
+    lens[3] = S - 45                                    # a ragged last block for one of the sampled sequences
+    q = synth.t_head_vectors(B, Hq, D, device, stream=3000, lead=1.0, scale=1.5)
+    q16 = torch.empty((B, Hq, D), dtype=torch.float16, device=device)
+    kv.resq_query_project(q, wq, s_u, q16)
+    out = torch.empty((B, Hq, D), dtype=torch.float32, device=device)
+    kv.resq_attention_decode(cache, q16, to_dev(lens), out, kv.attention_workspace(cache, Hq))
+    assert resq.resq_device_status() == resq.OK
+    image = host(cache.data).reshape(B, Hkv, S // 32, kv_util.BLOCK_BYTES)
+    out_h, q16_h = host(out), host(q16)
+    # the projected queries of the sampled sequences, bit for bit
+    Yq, _, _ = okv.project_int8(synth.bf16_bits_to_f32(_bits(q)).reshape(-1, D), *okv.quantize_uc(W_C))
+    assert (q16_h.view(np.uint16) == okv.query_fp16(Yq).reshape(B, Hq, D).view(np.uint16)).all()
+    for b in sampled:
+        kf, vf = kept[b]
+        Yk, _, _ = okv.project_int8(kf.reshape(-1, D), *okv.quantize_uc(W_C))
+        hk, hv = okv.kv_quantize(Yk), okv.kv_quantize(vf.reshape(-1, D))
+        for h in (0, 5):                                # every cache byte of two KV heads
+            blocks = image[b, h]
+            for which, rec, (o8, o4, om) in (("k", hk, kv_util.OFF["k"]), ("v", hv, kv_util.OFF["v"])):
+                rows = np.arange(S) * Hkv + h
+                assert (blocks[:, o8:o8 + 512].reshape(S, 16) == rec.c8[rows]).all(), (which, b, h)
+                assert (blocks[:, o4:o4 + 1792].reshape(S, 56) == rec.c4[rows]).all(), (which, b, h)
+                assert (np.ascontiguousarray(blocks[:, om:om + 512]).view(np.uint32).reshape(S, 4)
+                        == rec.meta[rows].view(np.uint32)).all(), (which, b, h)
+        dk, dv = okv.kv_dequantize(hk).reshape(S, Hkv, D), okv.kv_dequantize(hv).reshape(S, Hkv, D)
+        n = int(lens[b])
+        for hq in (0, 7, 22, 31):                       # sampled query heads: KV heads 0, 1, 5, 7
+            hk_i = hq // (Hq // Hkv)
+            ref = okv.attention_decode(q16_h[b:b + 1, hq:hq + 1], [[dk[:, hk_i]]], [[dv[:, hk_i]]], [n], 1, 1)[0, 0]
+            vmax = np.abs(dv[:n, hk_i]).max()
+            assert np.abs(out_h[b, hq] - ref).max() <= 1e-3 * vmax, (b, hq)
