@@ -148,8 +148,14 @@ int resq_hadamard_quantize(const void* X, int T, int K, int r, int8_t* x8, uint8
  * input feature, column j = coefficient), C fp32 [T][K], bf16 products accumulated in fp32 on the
  * tensor cores.  This is the first half of resq_project_quantize with P != NULL, exposed so that the
  * coefficients can be inspected and the GEMM timed on its own.  K % 8 == 0.
+ * workspace (optional, may be NULL): resq_project_workspace_bytes() bytes of scratch.  With it, when the
+ * last round of 256 x 256 output tiles would occupy less than half of the GPU, those tiles are cut along K
+ * into partial tiles that a second kernel adds up in a fixed order (deterministic; the fp32 sums are then
+ * formed in that order instead of one run over K).  resq_workspace_bytes() with has_P includes this scratch.
  */
-int resq_project(const void* X, const void* P, int T, int K, float* C, void* stream);
+size_t resq_project_workspace_bytes(void);
+int resq_project(const void* X, const void* P, int T, int K, float* C, void* workspace, size_t workspace_bytes,
+                 void* stream);
 
 /*
  * Eq. 4 with the dequantizing epilogue: Y = diag(s_x8)(x8·w8^T)diag(s_w8) + diag(s_x4)(x4·w4^T)diag(s_w4).

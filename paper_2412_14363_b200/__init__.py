@@ -22,7 +22,7 @@ Y_BF16, Y_FP32 = 0, 1
 
 EXPORTS = [
     "resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_bytes", "resq_workspace_bytes",
-    "resq_pack_weights", "resq_pack_weights_projected", "resq_pack_projected_workspace_bytes", "resq_project", "resq_hadamard_quantize", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
+    "resq_pack_weights", "resq_pack_weights_projected", "resq_pack_projected_workspace_bytes", "resq_project", "resq_project_workspace_bytes", "resq_hadamard_quantize", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
     "resq_unpack_int4", "resq_set_option",
     "resq_weight_row_sums", "resq_project_quantize_asym", "resq_mixed_gemm_asym", "resq_linear_asym",
     "resq_workspace_bytes_asym",
@@ -63,7 +63,9 @@ lib.resq_pack_weights.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_pack_projected_workspace_bytes.restype = _sz
 lib.resq_pack_projected_workspace_bytes.argtypes = [_dp]
 lib.resq_pack_weights_projected.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
-lib.resq_project.argtypes = [_vp, _vp, _i, _i, _vp, _vp]
+lib.resq_project.argtypes = [_vp, _vp, _i, _i, _vp, _vp, _sz, _vp]
+lib.resq_project_workspace_bytes.restype = _sz
+lib.resq_project_workspace_bytes.argtypes = []
 lib.resq_hadamard_quantize.argtypes = [_vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_project_quantize.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 lib.resq_project_quantize_static.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -175,10 +177,15 @@ def resq_project_quantize(X, P, r: int, x8, x4, s_x8, s_x4, x4_i8=None, workspac
                                      _stream()), "resq_project_quantize")
 
 
-def resq_project(X, P, C):
-    """C (fp32 [T][K]) = X (bf16 [T][K]) · P (bf16 [K][K]): the online projection alone."""
+def resq_project(X, P, C, workspace=None):
+    """C (fp32 [T][K]) = X (bf16 [T][K]) · P (bf16 [K][K]): the online projection alone.  workspace: optional
+    uint8 tensor of resq_project_workspace_bytes() bytes (lets a thin last round of tiles be cut along K)."""
     T, K = X.shape
-    _check(lib.resq_project(_ptr(X), _ptr(P), T, K, _ptr(C), _stream()), "resq_project")
+    _check(lib.resq_project(_ptr(X), _ptr(P), T, K, _ptr(C), _ptr(workspace), _nbytes(workspace), _stream()), "resq_project")
+
+
+def resq_project_workspace_bytes() -> int:
+    return int(lib.resq_project_workspace_bytes())
 
 
 def resq_hadamard_quantize(X, r: int, x8, x4, s_x8, s_x4, x4_i8=None):

@@ -60,7 +60,7 @@ int check_arch() {
 
 // Carving of the caller's workspace.  Every entry point uses the same map (and its own subset).
 struct Workspace {
-    size_t x8, x4, sx8, sx4, zx8, zx4, x4e, w4e, panel, decode, total;
+    size_t x8, x4, sx8, sx4, zx8, zx4, x4e, w4e, panel, decode, total;  // panel: fp32 coefficients + the GEMM's split scratch
 };
 Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     Workspace w{};
@@ -75,7 +75,7 @@ Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     const bool tiles = T > kDecodeMaxT;
     w.x4e = o;    o += tiles ? align_up(Tz * K4) : 0;
     w.w4e = o;    o += (tiles && !has_w4_i8) ? align_up(N * K4) : 0;
-    w.panel = o;  o += has_P ? align_up(static_cast<size_t>(T < kPanelRows ? T : kPanelRows) * K * 4) : 0;
+    w.panel = o;  o += has_P ? align_up(static_cast<size_t>(T < kPanelRows ? T : kPanelRows) * K * 4) + align_up(project_split_scratch_bytes()) : 0;
     w.decode = o; o += tiles ? 0 : align_up(decode_scratch_bytes(T, n_out));
     w.total = o;
     return w;
@@ -177,11 +177,16 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
     const size_t need = align_up(static_cast<size_t>(rows_max) * K * 4);
     if (!workspace || workspace_bytes < need) return RESQ_ERR_WORKSPACE;
     float* panel = static_cast<float*>(workspace);
+    // what the workspace holds beyond the panel serves the GEMM's last-round split (resq_workspace_bytes includes it)
+    const bool has_scratch = workspace_bytes >= need + project_split_scratch_bytes();
+    void* scratch = has_scratch ? static_cast<char*>(workspace) + need : nullptr;
     const size_t K4 = static_cast<size_t>(K - r);
     for (int t0 = 0; t0 < T; t0 += kPanelRows) {
         const int rows = T - t0 < kPanelRows ? T - t0 : kPanelRows;
         const char* Xp = static_cast<const char*>(X) + static_cast<size_t>(t0) * K * 2;
-        if (cudaError_t e = launch_project_gemm(Xp, P, rows, K, panel, st); e != cudaSuccess) return cuda_status(e);
+        if (cudaError_t e = launch_project_gemm(Xp, P, rows, K, panel, st, scratch, project_split_scratch_bytes());
+            e != cudaSuccess)
+            return cuda_status(e);
         if (cudaError_t e = launch_split_quantize(panel, true, rows, K, r, x8 + static_cast<size_t>(t0) * r,
                                                   x4 ? x4 + static_cast<size_t>(t0) * K4 / 2 : nullptr, s_x8 + t0,
                                                   s_x4 + t0, false,
@@ -205,12 +210,17 @@ int resq_hadamard_quantize(const void* X, int T, int K, int r, int8_t* x8, uint8
     return e == cudaErrorNotSupported ? RESQ_ERR_SHAPE : cuda_status(e);
 }
 
-int resq_project(const void* X, const void* P, int T, int K, float* C, void* stream) {
+size_t resq_project_workspace_bytes(void) { return project_split_scratch_bytes(); }
+
+int resq_project(const void* X, const void* P, int T, int K, float* C, void* workspace, size_t workspace_bytes,
+                 void* stream) {
     if (T < 1 || K <= 0 || K % 8 != 0) return RESQ_ERR_SHAPE;
     if (!X || !P || !C) return RESQ_ERR_NULL;
-    if (!aligned16(X) || !aligned16(P) || !aligned16(C)) return RESQ_ERR_ALIGN;
+    if (!aligned16(X) || !aligned16(P) || !aligned16(C) || !aligned16(workspace)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
-    return cuda_status(launch_project_gemm(X, P, T, K, C, static_cast<cudaStream_t>(stream)));
+    const bool has_scratch = workspace && workspace_bytes >= project_split_scratch_bytes();
+    return cuda_status(launch_project_gemm(X, P, T, K, C, static_cast<cudaStream_t>(stream),
+                                           has_scratch ? workspace : nullptr, has_scratch ? workspace_bytes : 0));
 }
 
 static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, const uint8_t* x4,
@@ -328,11 +338,15 @@ int resq_project_quantize_asym(const void* X, const void* P, int T, int K, int r
     const size_t need = align_up(static_cast<size_t>(rows_max) * K * 4);
     if (!workspace || workspace_bytes < need) return RESQ_ERR_WORKSPACE;
     float* panel = static_cast<float*>(workspace);
+    const bool has_scratch = workspace_bytes >= need + project_split_scratch_bytes();
+    void* scratch = has_scratch ? static_cast<char*>(workspace) + need : nullptr;
     const size_t K4 = static_cast<size_t>(K - r);
     for (int t0 = 0; t0 < T; t0 += kPanelRows) {
         const int rows = T - t0 < kPanelRows ? T - t0 : kPanelRows;
         const char* Xp = static_cast<const char*>(X) + static_cast<size_t>(t0) * K * 2;
-        if (cudaError_t e = launch_project_gemm(Xp, P, rows, K, panel, st); e != cudaSuccess) return cuda_status(e);
+        if (cudaError_t e = launch_project_gemm(Xp, P, rows, K, panel, st, scratch, project_split_scratch_bytes());
+            e != cudaSuccess)
+            return cuda_status(e);
         if (cudaError_t e = launch_split_quantize_asym(panel, true, rows, K, r, u8 + static_cast<size_t>(t0) * r,
                                                        u4 ? u4 + static_cast<size_t>(t0) * K4 / 2 : nullptr, s_x8 + t0,
                                                        s_x4 + t0, z_x8 + t0, z_x4 + t0,

@@ -69,7 +69,10 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
 void set_decode_early_weights(int on);
 
 // Online projection C = X·P (bf16 x bf16 -> fp32) on tcgen05 kind::f16, CTA pairs; writes fp32 C [T][K].
-cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, float* C, cudaStream_t st);
+// scratch (optional, project_split_scratch_bytes() bytes): lets a thinly filled last round of tiles be cut along K.
+size_t project_split_scratch_bytes();
+cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, float* C, cudaStream_t st,
+                                void* scratch = nullptr, size_t scratch_bytes = 0);
 
 // Output-tile width of the two tile GEMMs (see the definition for what was measured).
 int pick_tile_width(int m_tiles, int N, int sms);

@@ -42,6 +42,18 @@ struct Params {
     int panel_tiles;                 // pair tiles per row panel of the tile order
     float* C;
     int* status;
+    // The last, partly filled round of the persistent grid: its `split_tiles` tiles are cut into `splits` slices
+    // of `kb_slice` k-blocks each, one work item per slice, written as partial tiles to `partial`
+    // ([split_tiles][splits][256][256] fp32) and summed in slice order by project_reduce_kernel.  0: no split.
+    int full_items, split_tiles, splits, kb_slice;
+    float* partial;
+};
+
+struct Item {
+    int m0, n0, kb0, nkb;
+    float* dst;     // first element of the 256 x 256 output tile (C or a partial tile)
+    size_t ld;      // its row pitch in floats
+    bool bounded;   // rows >= T and columns >= K must not be written (C); partial tiles are written whole
 };
 
 struct __align__(8) Shared {
@@ -81,6 +93,45 @@ __device__ __forceinline__ void tile_coords(const Params& p, int tile, int& m0, 
     n0 = n * BN;
 }
 
+__device__ __forceinline__ Item item_info(const Params& p, int item) {
+    Item it;
+    if (item < p.full_items) {
+        tile_coords(p, item, it.m0, it.n0);
+        it.kb0 = 0;
+        it.nkb = p.kb_total;
+        it.dst = p.C + static_cast<size_t>(it.m0) * p.K + it.n0;
+        it.ld = static_cast<size_t>(p.K);
+        it.bounded = true;
+    } else {
+        const int j = item - p.full_items, t = j / p.splits, sl = j - t * p.splits;
+        tile_coords(p, p.full_items + t, it.m0, it.n0);
+        it.kb0 = sl * p.kb_slice;
+        it.nkb = min(p.kb_slice, p.kb_total - it.kb0);
+        it.dst = p.partial + static_cast<size_t>(j) * (2 * BM) * BN;
+        it.ld = BN;
+        it.bounded = false;
+    }
+    return it;
+}
+
+// C tile = sum of its partial tiles, slices in index order (deterministic).
+__global__ void __launch_bounds__(256) project_reduce_kernel(const Params p) {
+    const int t = blockIdx.y;
+    int m0, n0;
+    tile_coords(p, p.full_items + t, m0, n0);
+    const float* part = p.partial + static_cast<size_t>(t) * p.splits * (2 * BM) * BN;
+    for (int q = blockIdx.x * blockDim.x + threadIdx.x; q < 2 * BM * BN / 4; q += gridDim.x * blockDim.x) {
+        const int row = q / (BN / 4), c4 = q - row * (BN / 4);
+        float4 a = reinterpret_cast<const float4*>(part)[q];
+        for (int sl = 1; sl < p.splits; ++sl) {
+            const float4 b = reinterpret_cast<const float4*>(part + static_cast<size_t>(sl) * (2 * BM) * BN)[q];
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        if (m0 + row < p.T && n0 + 4 * c4 < p.K)
+            *reinterpret_cast<float4*>(p.C + static_cast<size_t>(m0 + row) * p.K + n0 + 4 * c4) = a;
+    }
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmP,
                          const Params p) {
@@ -94,7 +145,7 @@ project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = static_cast<int>(cluster_ctarank());  // 0: even CTA (issues the MMAs), 1: its peer
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-    const int num_tiles = p.m_tiles * p.n_tiles;
+    const int num_items = p.full_items + p.split_tiles * p.splits;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -126,11 +177,10 @@ project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
-                int m0, n0;
-                tile_coords(p, tile, m0, n0);
-                const int my_m = m0 + rank * BM, my_n = n0 + rank * BN_HALF;
-                for (int kb = 0; kb < p.kb_total; ++kb) {
+            for (int item = pair; item < num_items && ok; item += npairs) {
+                const Item it = item_info(p, item);
+                const int my_m = it.m0 + rank * BM, my_n = it.n0 + rank * BN_HALF;
+                for (int kb = it.kb0; kb < it.kb0 + it.nkb; ++kb) {
                     if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
                     // The even CTA arms its barrier for the bytes of both CTAs; the peer only sends its bytes
                     // there (they may land before the barrier is armed: the pending arrival keeps the phase open).
@@ -158,11 +208,12 @@ project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
             uint32_t acc_phase[2] = {0, 0};
             int buf = 0;
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+            for (int item = pair; item < num_items && ok; item += npairs) {
+                const int nkb = item_info(p, item).nkb;
                 if (!mbar_wait(&sh->acc_empty[buf], acc_phase[buf] ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + static_cast<uint32_t>(buf * BN);
-                for (int kb = 0; kb < p.kb_total; ++kb) {
+                for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(&sh->full[stage], phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t a_desc = make_smem_desc_k128(smem_u32(sA + stage * A_BYTES));
@@ -185,9 +236,8 @@ project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
         const int et = threadIdx.x - 64;
         uint32_t acc_phase[2] = {0, 0};
         int buf = 0;
-        for (int tile = pair; tile < num_tiles; tile += npairs) {
-            int m0, n0;
-            tile_coords(p, tile, m0, n0);
+        for (int item = pair; item < num_items; item += npairs) {
+            const Item it = item_info(p, item);
             epi_barrier();
             if (et == 0) sh->epi_stop = *abort_flag;
             epi_barrier();
@@ -195,19 +245,19 @@ project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
             if (!mbar_wait(&sh->acc_full[buf], acc_phase[buf], abort_flag)) continue;
             acc_phase[buf] ^= 1;
             tc_fence_after();
-            const int row = m0 + rank * BM + quad * 32 + lane;
+            const int lrow = rank * BM + quad * 32 + lane;  // row inside the pair's tile
             const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + buf * BN;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld32(lane_addr + c * 32, v);
                 tmem_ld_wait();
-                const int nb = n0 + c * 32;
-                if (row < p.T) {
-                    float* cp = p.C + static_cast<size_t>(row) * p.K + nb;
+                const int nb = it.n0 + c * 32;
+                if (!it.bounded || it.m0 + lrow < p.T) {
+                    float* cp = it.dst + static_cast<size_t>(lrow) * it.ld + c * 32;
 #pragma unroll
                     for (int g = 0; g < 8; ++g)
-                        if (nb + g * 4 < p.K)
+                        if (!it.bounded || nb + g * 4 < p.K)
                             reinterpret_cast<uint4*>(cp)[g] = make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
                 }
             }
@@ -247,7 +297,10 @@ bool make_map_bf16(CUtensorMap* m, const void* base, uint64_t rows, uint64_t col
 
 }  // namespace
 
-cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, float* C, cudaStream_t st) {
+size_t project_split_scratch_bytes() { return static_cast<size_t>(74) * (2 * BM) * BN * sizeof(float); }
+
+cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, float* C, cudaStream_t st, void* scratch,
+                                size_t scratch_bytes) {
     static bool attr_set[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -278,8 +331,31 @@ cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, floa
     const int tiles = p.m_tiles * p.n_tiles;
     int pairs = sms / 2;
     if (tiles < pairs) pairs = tiles;
+    // A last round that fills less than half of the grid is cut along K so that it takes a fraction of a round:
+    // each of its tiles becomes `splits` work items whose partial tiles a second kernel adds up in slice order.
+    p.full_items = tiles;
+    p.split_tiles = p.splits = p.kb_slice = 0;
+    p.partial = static_cast<float*>(scratch);
+    const int rem = tiles % pairs;
+    if (scratch && tiles > pairs && rem > 0 && pairs / rem >= 2) {
+        int splits = pairs / rem;
+        if (splits > p.kb_total / 4) splits = p.kb_total / 4;  // at least four k-blocks per slice
+        const int kb_slice = splits > 0 ? (p.kb_total + splits - 1) / splits : 0;
+        if (splits >= 2) splits = (p.kb_total + kb_slice - 1) / kb_slice;  // no empty slice
+        if (splits >= 2 && static_cast<size_t>(rem) * splits * (2 * BM) * BN * sizeof(float) <= scratch_bytes) {
+            p.full_items = tiles - rem;
+            p.split_tiles = rem;
+            p.splits = splits;
+            p.kb_slice = kb_slice;
+        }
+    }
     project_gemm_pair_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tX, tP, p);
-    return cudaGetLastError();
+    if (cudaError_t le = cudaGetLastError(); le != cudaSuccess) return le;
+    if (p.split_tiles > 0) {
+        project_reduce_kernel<<<dim3(16, p.split_tiles), 256, 0, st>>>(p);
+        return cudaGetLastError();
+    }
+    return cudaSuccess;
 }
 
 }  // namespace resq

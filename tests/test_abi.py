@@ -44,6 +44,15 @@ def test_pack_projected_host_validation(resq):
     assert L.resq_pack_weights_projected(ctypes.byref(d), fake + 2, fake, fake, fake, fake, fake, None, fake, need, None) == resq.ERR_ALIGN
 
 
+def test_project_host_validation(resq):
+    L = resq.lib
+    fake = 1 << 20
+    assert L.resq_project_workspace_bytes() == 74 * 256 * 256 * 4
+    assert L.resq_project(fake, fake, 4, 1001, fake, None, 0, None) == resq.ERR_SHAPE
+    assert L.resq_project(fake, None, 4, 1024, fake, None, 0, None) == resq.ERR_NULL
+    assert L.resq_project(fake, fake, 4, 1024, fake, fake + 8, 1 << 30, None) == resq.ERR_ALIGN
+
+
 def test_every_header_is_covered():
     assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["resq.h", "resq_kv.h"]
 

@@ -103,6 +103,33 @@ def test_projection_alone_against_fp64_sums(resq, T, K):
     assert (np.abs(host(C).astype(np.float64) - C_ref.astype(np.float64)) <= bound).all()
 
 
+@pytest.mark.parametrize("T,K", [(4096, 1280), (2200, 2304)])
+def test_projection_with_split_last_round(resq, T, K):
+    """More 256 x 256 tiles than CTA pairs with a thin last round (80 and 81 tiles on 74 pairs): with the scratch
+    workspace those tiles are cut along K and summed in slice order.  Same bound as above plus one rounding per
+    slice; two calls give identical bits (fixed summation order); without the workspace the result obeys the same
+    bound."""
+    X_bits = synth.f32_to_bf16_bits(synth.activations(T, K, "t4", seed=900 + K))
+    P_bits = synth.f32_to_bf16_bits(synth.kron_orthogonal_bf16(K, inner=128))
+    C_ref = oracle.project(X_bits, P_bits).astype(np.float64)
+    Xd, Pd = bf16_to_dev(X_bits), bf16_to_dev(P_bits)
+    ws = torch.empty(resq.resq_project_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)
+    outs = []
+    for w in (ws, ws, None):
+        C = torch.full((T, K), float("nan"), dtype=torch.float32, device="cuda")
+        resq.resq_project(Xd, Pd, C, w)
+        assert resq.resq_device_status() == resq.OK
+        outs.append(host(C))
+    Xf = np.abs(synth.bf16_bits_to_f32(X_bits).astype(np.float64))
+    Pf = np.abs(synth.bf16_bits_to_f32(P_bits).astype(np.float64))
+    bound = (K // 16 + 20) * 2.0 ** -24 * (Xf @ Pf) + 1e-30
+    for C in outs:
+        assert (np.abs(C.astype(np.float64) - C_ref) <= bound).all()
+    assert (outs[0].view(np.uint32) == outs[1].view(np.uint32)).all()
+    assert (outs[0] != outs[2]).any()          # the split really changed the summation order somewhere
+
+
 @pytest.mark.parametrize("N,K,r,fp16", [(64, 512, 64, False), (4104, 1024, 128, False), (264, 2048, 256, True)])
 def test_pack_weights_projected(resq, N, K, r, fp16):
     """Weight projection at pack time (Section 4.3): W_raw·U on the tensor cores, then Eq. 3.  Against the oracle's
