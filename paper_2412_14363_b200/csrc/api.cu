@@ -60,7 +60,7 @@ int check_arch() {
 
 // Carving of the caller's workspace.  Every entry point uses the same map (and its own subset).
 struct Workspace {
-    size_t x8, x4, sx8, sx4, zx8, zx4, x4e, w4e, panel, decode, msplit, total;  // panel: fp32 coefficients + the GEMM's split scratch
+    size_t x8, x4, sx8, sx4, zx8, zx4, x4e, w4e, panel, decode, total;  // panel: fp32 coefficients + the GEMM's split scratch
 };
 Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     Workspace w{};
@@ -77,7 +77,6 @@ Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     w.w4e = o;    o += (tiles && !has_w4_i8) ? align_up(N * K4) : 0;
     w.panel = o;  o += has_P ? align_up(static_cast<size_t>(T < kPanelRows ? T : kPanelRows) * K * 4) + align_up(project_split_scratch_bytes()) : 0;
     w.decode = o; o += tiles ? 0 : align_up(decode_scratch_bytes(T, n_out));
-    w.msplit = o; o += tiles ? align_up(mixed_split_scratch_bytes()) : 0;  // partial tiles of the tile GEMM's last round
     w.total = o;
     return w;
 }
@@ -253,8 +252,7 @@ static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, 
         w4e = buf;
     }
     return cuda_status(launch_mixed_gemm_tiles(T, d->n_out, d->K, d->r, x8, x4e, s_x8, s_x4, W->w8, w4e, W->s_w8,
-                                               W->s_w4, fp16, Y, y_dtype, dbg8, dbg4, st, nullptr, nullptr, nullptr, nullptr,
-                                               ws + map.msplit, mixed_split_scratch_bytes()));
+                                               W->s_w4, fp16, Y, y_dtype, dbg8, dbg4, st));
 }
 
 static int check_weights(const resq_weights_t* W, int r) {
@@ -389,7 +387,7 @@ static int mixed_gemm_asym_impl(const resq_layer_desc_t* d, int T, const uint8_t
     return cuda_status(launch_mixed_gemm_tiles(T, d->n_out, d->K, d->r, reinterpret_cast<const int8_t*>(u8), x4e, s_x8,
                                                s_x4, W->w8, w4e, W->s_w8, W->s_w4,
                                                d->w_scale_dtype == RESQ_SCALE_FP16, Y, y_dtype, dbg8, dbg4, st, z_x8,
-                                               z_x4, wsum8, wsum4, ws + map.msplit, mixed_split_scratch_bytes()));
+                                               z_x4, wsum8, wsum4));
 }
 
 // The tile kernel serves every T here, so the workspace is carved as for T > 16.

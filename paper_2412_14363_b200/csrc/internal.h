@@ -37,9 +37,7 @@ cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8
                                     const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
                                     int32_t* dbg8, int32_t* dbg4, cudaStream_t st, const float* z_x8 = nullptr,
                                     const float* z_x4 = nullptr, const int32_t* wsum8 = nullptr,
-                                    const int32_t* wsum4 = nullptr, void* scratch = nullptr, size_t scratch_bytes = 0);
-// scratch (optional, mixed_split_scratch_bytes() bytes): lets a thinly filled last round of tiles be cut along K.
-size_t mixed_split_scratch_bytes();
+                                    const int32_t* wsum4 = nullptr);
 // z_x8 != NULL selects asymmetric activations: x8 / x4e then hold UNSIGNED codes (0..255, 0..15) and the
 // epilogue adds z_x8[t] * s_w8[n] * wsum8[n] + z_x4[t] * s_w4[n] * wsum4[n].
 

@@ -60,34 +60,7 @@ struct Params {
     int32_t* dbg8;
     int32_t* dbg4;
     int* status;
-    // The last, partly filled round of the persistent grid: its `split_tiles` tiles are cut into `splits` slices of
-    // the k-block list (INT4 blocks, then INT8 blocks), `kb_slice` blocks each, the last slice taking the rest and
-    // with it every INT8 block.  A slice is one work item; its raw int32 accumulators go to part4
-    // ([split_tiles][splits][256][256]) and, from the last slice, part8 ([split_tiles][256][256]);
-    // mixed_reduce_kernel adds the INT4 parts (exact) and applies the epilogue.  split_tiles = 0: no split.
-    int full_items, split_tiles, splits, kb_slice;
-    int32_t* part4;
-    int32_t* part8;
 };
-
-struct Item {
-    int tile, kb0, nkb, slot;  // slot >= 0: index of the partial INT4 tile of a split item
-    bool last;                 // the slice that also holds the INT8 blocks
-};
-__device__ __forceinline__ Item item_info(const Params& p, int item) {
-    Item it;
-    if (item < p.full_items) {
-        it.tile = item; it.kb0 = 0; it.nkb = p.kb8 + p.kb4; it.slot = -1; it.last = true;
-    } else {
-        const int j = item - p.full_items, t = j / p.splits, sl = j - t * p.splits;
-        it.tile = p.full_items + t;
-        it.kb0 = sl * p.kb_slice;
-        it.last = sl == p.splits - 1;
-        it.nkb = it.last ? p.kb8 + p.kb4 - it.kb0 : p.kb_slice;
-        it.slot = j;
-    }
-    return it;
-}
 
 struct __align__(8) Shared {
     uint64_t full[STAGES];
@@ -129,7 +102,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = static_cast<int>(cluster_ctarank());  // 0: even CTA (issues the MMAs), 1: its peer
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-    const int num_items = p.full_items + p.split_tiles * p.splits;  // tiles (m_tiles counts 256-row pair tiles) and slices
+    const int num_tiles = p.m_tiles * p.n_tiles;  // m_tiles counts 256-row pair tiles
+    const int kb_total = p.kb8 + p.kb4;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -162,11 +136,10 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int item = pair; item < num_items && ok; item += npairs) {
-                const Item it = item_info(p, item);
-                const int m0 = (it.tile % p.m_tiles) * 2 * BM + rank * BM;        // this CTA's token rows
-                const int n0 = (it.tile / p.m_tiles) * p.bn + rank * BN_HALF;     // this CTA's weight rows
-                for (int kb = it.kb0; kb < it.kb0 + it.nkb; ++kb) {
+            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+                const int m0 = (tile % p.m_tiles) * 2 * BM + rank * BM;        // this CTA's token rows
+                const int n0 = (tile / p.m_tiles) * p.bn + rank * BN_HALF;     // this CTA's weight rows
+                for (int kb = 0; kb < kb_total; ++kb) {
                     if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
                     // The even CTA arms its barrier for the bytes of both CTAs; the peer only sends its
                     // bytes there (if they land first, the pending arrival keeps the phase open).
@@ -195,12 +168,11 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             int stage = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int item = pair; item < num_items && ok; item += npairs) {
-                const Item it = item_info(p, item);
+            for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
                 // INT4 columns are free once the previous tile's epilogue has copied them out.
                 if (!mbar_wait(&sh->acc4_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                for (int kb = it.kb0; kb < it.kb0 + it.nkb; ++kb) {
+                for (int kb = 0; kb < kb_total; ++kb) {
                     const bool seg4 = kb < p.kb4;
                     if (kb == p.kb4) {
                         // ... the INT8 columns once it has finished with the tile.
@@ -212,7 +184,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                     const uint64_t a_desc = make_smem_desc_k128(smem_u32(sA + stage * A_BYTES));
                     const uint64_t b_desc = make_smem_desc_k128(smem_u32(sB + stage * B_BYTES));
                     const uint32_t d = tmem_base + (seg4 ? static_cast<uint32_t>(BN) : 0u);
-                    const bool first = kb == it.kb0 || kb == p.kb4;  // a slice starts inside the INT4 blocks
+                    const bool first = kb == 0 || kb == p.kb4;
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)
                         mma_i8_ss_pair(d, a_desc + 2 * k, b_desc + 2 * k, idesc, (first && k == 0) ? 0u : 1u);
@@ -232,9 +204,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
         uint32_t acc_phase = 0;
         // The epilogue threads meet at named barriers, so they must leave the loop together:
         // one thread samples the abort flag and the others take its reading.
-        for (int item = pair; item < num_items; item += npairs) {
-            const Item it = item_info(p, item);
-            const int tile = it.tile;
+        for (int tile = pair; tile < num_tiles; tile += npairs) {
             const int m0 = (tile % p.m_tiles) * 2 * BM + rank * BM, n0 = (tile / p.m_tiles) * p.bn;
             epi_barrier();  // previous tile's readers of sw8/sw4/epi_stop are done
             if (et == 0) sh->epi_stop = *abort_flag;
@@ -282,19 +252,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                 const int cb = ch * (BN / 2) + c * 16;  // first column of the chunk inside the tile
                 const int nb = n0 + cb;
                 const uint32_t* a4c = &a4[c >> 1][(c & 1) * 16];
-                if (it.slot >= 0) {  // a slice: raw accumulators into the partial tiles, whole (rows past T are zero)
-                    const size_t poff = (static_cast<size_t>(rank * BM + quad * 32 + lane)) * BN + cb;
-                    int32_t* q4 = p.part4 + static_cast<size_t>(it.slot) * (2 * BM) * BN + poff;
-#pragma unroll
-                    for (int g = 0; g < 4; ++g)
-                        reinterpret_cast<uint4*>(q4)[g] = make_uint4(a4c[4 * g], a4c[4 * g + 1], a4c[4 * g + 2], a4c[4 * g + 3]);
-                    if (it.last) {
-                        int32_t* q8 = p.part8 + static_cast<size_t>(it.slot / p.splits) * (2 * BM) * BN + poff;
-#pragma unroll
-                        for (int g = 0; g < 4; ++g)
-                            reinterpret_cast<uint4*>(q8)[g] = make_uint4(a8[4 * g], a8[4 * g + 1], a8[4 * g + 2], a8[4 * g + 3]);
-                    }
-                } else if (row_ok) {
+                if (row_ok) {
                     const size_t off = static_cast<size_t>(row) * p.N + nb;
                     if (p.dbg8) {
 #pragma unroll
@@ -353,52 +311,6 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
     }
 }
 
-// Finishes the split tiles: the INT4 accumulator is the sum of the slices' partial tiles (integers: exact in any
-// order), the INT8 accumulator comes from the last slice; then the same epilogue as in the GEMM kernel.
-template <bool ASYM>
-__global__ void __launch_bounds__(256) mixed_reduce_kernel(const Params p) {
-    const int t = blockIdx.y, tile = p.full_items + t;
-    const int m0 = (tile % p.m_tiles) * 2 * BM, n0 = (tile / p.m_tiles) * p.bn;
-    const int32_t* q4 = p.part4 + static_cast<size_t>(t) * p.splits * (2 * BM) * BN;
-    const int32_t* q8 = p.part8 + static_cast<size_t>(t) * (2 * BM) * BN;
-    for (int q = blockIdx.x * blockDim.x + threadIdx.x; q < 2 * BM * BN / 4; q += gridDim.x * blockDim.x) {
-        const int lrow = q / (BN / 4), cb = 4 * (q - lrow * (BN / 4));
-        const int row = m0 + lrow, nb = n0 + cb;
-        if (row >= p.T || nb >= p.N || cb >= p.bn) continue;
-        int4 a4 = reinterpret_cast<const int4*>(q4)[q];
-        for (int sl = 1; sl < p.splits; ++sl) {
-            const int4 b = reinterpret_cast<const int4*>(q4 + static_cast<size_t>(sl) * (2 * BM) * BN)[q];
-            a4.x += b.x; a4.y += b.y; a4.z += b.z; a4.w += b.w;
-        }
-        int4 a8 = make_int4(0, 0, 0, 0);
-        if (p.kb8 > 0) a8 = reinterpret_cast<const int4*>(q8)[q];
-        const size_t off = static_cast<size_t>(row) * p.N + nb;
-        if (p.dbg8) {
-            *reinterpret_cast<int4*>(p.dbg8 + off) = a8;
-            *reinterpret_cast<int4*>(p.dbg4 + off) = a4;
-        }
-        const float sx8 = __ldg(p.s_x8 + row), sx4 = __ldg(p.s_x4 + row);
-        const float zx8 = ASYM ? __ldg(p.z_x8 + row) : 0.f, zx4 = ASYM ? __ldg(p.z_x4 + row) : 0.f;
-        const int v8[4] = {a8.x, a8.y, a8.z, a8.w}, v4[4] = {a4.x, a4.y, a4.z, a4.w};
-        float y[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float w8s = load_scale(p.s_w8, nb + j, p.w_fp16), w4s = load_scale(p.s_w4, nb + j, p.w_fp16);
-            const float t8 = static_cast<float>(v8[j]) * (sx8 * w8s);
-            const float t4 = static_cast<float>(v4[j]) * (sx4 * w4s);
-            y[j] = t8 + t4;
-            if (ASYM) y[j] += zx8 * (static_cast<float>(p.wsum8[nb + j]) * w8s) + zx4 * (static_cast<float>(p.wsum4[nb + j]) * w4s);
-        }
-        if (p.y_dtype == RESQ_Y_BF16) {
-            __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0], y[1]), h1 = __floats2bfloat162_rn(y[2], y[3]);
-            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.Y) + off) =
-                make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
-        } else {
-            *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.Y) + off) = make_float4(y[0], y[1], y[2], y[3]);
-        }
-    }
-}
-
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -424,14 +336,11 @@ bool make_map_u8(CUtensorMap* m, const void* base, uint64_t rows, uint64_t kbyte
 // than 256-wide ones in both GEMMs, which costs far more than the partly filled round they save.
 int pick_tile_width(int /*m_tiles*/, int /*N*/, int /*sms*/) { return 256; }
 
-size_t mixed_split_scratch_bytes() { return static_cast<size_t>(148) * (2 * BM) * BN * sizeof(int32_t); }
-
 cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8, const int8_t* x4e,
                                     const float* s_x8, const float* s_x4, const int8_t* w8, const int8_t* w4e,
                                     const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
                                     int32_t* dbg8, int32_t* dbg4, cudaStream_t st, const float* z_x8,
-                                    const float* z_x4, const int32_t* wsum8, const int32_t* wsum4, void* scratch,
-                                    size_t scratch_bytes) {
+                                    const float* z_x4, const int32_t* wsum8, const int32_t* wsum4) {
     const bool asym = z_x8 != nullptr;  // then x8 / x4e hold unsigned codes
     static bool attr_set[64] = {};
     int dev = 0;
@@ -471,37 +380,9 @@ cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8
     p.status = device_status_ptr();
     const int tiles = p.m_tiles * p.n_tiles;
     const int pairs = tiles < sms / 2 ? tiles : sms / 2;
-    // A last round that fills less than half of the pairs is cut along the k-block list: up to 7 slices, so that
-    // the INT8 blocks (1/8 of the list) all fall into the last one, at least four blocks per slice.
-    p.full_items = tiles;
-    p.split_tiles = p.splits = p.kb_slice = 0;
-    p.part4 = p.part8 = nullptr;
-    const int rem = tiles % pairs, kb_total = p.kb8 + p.kb4;
-    if (scratch && tiles > pairs && rem > 0 && pairs / rem >= 2) {
-        int splits = pairs / rem;
-        if (splits > 7) splits = 7;
-        if (splits > kb_total / 4) splits = kb_total / 4;
-        const int kb_slice = splits >= 2 ? (kb_total + splits - 1) / splits : 0;
-        const size_t tile_bytes = static_cast<size_t>(2 * BM) * BN * sizeof(int32_t);
-        if (splits >= 2 && (splits - 1) * kb_slice < p.kb4 &&
-            static_cast<size_t>(rem) * (splits + 1) * tile_bytes <= scratch_bytes) {
-            p.full_items = tiles - rem;
-            p.split_tiles = rem;
-            p.splits = splits;
-            p.kb_slice = kb_slice;
-            p.part4 = static_cast<int32_t*>(scratch);
-            p.part8 = p.part4 + static_cast<size_t>(rem) * splits * (2 * BM) * BN;
-        }
-    }
     if (asym) mixed_gemm_kernel<true><<<2 * pairs, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
     else mixed_gemm_kernel<false><<<2 * pairs, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
-    if (cudaError_t le = cudaGetLastError(); le != cudaSuccess) return le;
-    if (p.split_tiles > 0) {
-        if (asym) mixed_reduce_kernel<true><<<dim3(16, p.split_tiles), 256, 0, st>>>(p);
-        else mixed_reduce_kernel<false><<<dim3(16, p.split_tiles), 256, 0, st>>>(p);
-        return cudaGetLastError();
-    }
-    return cudaSuccess;
+    return cudaGetLastError();
 }
 
 }  // namespace resq
