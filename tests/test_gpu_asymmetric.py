@@ -85,6 +85,7 @@ def _check_output(res, pw, y32_gpu, ybf_bits=None):
     (16, 512, 512, 64, False, True),
     (17, 512, 264, 64, False, True),      # ragged rows and columns
     (300, 2048, 520, 256, True, False),   # two pair tiles of rows, partial column tile, kernel expands packed weights
+    (2304, 1024, 2304, 128, False, True),  # 81 tiles on 74 CTA pairs: two rounds of the persistent grid
     (1, 4096, 1024, 512, True, True),     # a single token through the tile kernel
     (257, 1024, 768, 128, False, True),
 ])

@@ -197,6 +197,9 @@ def oracle_case(T, K, N, r, fp16=False, seed_shift=0):
     (128, 4096, 1024, 512, True, True),   # k/v projection shape of the 8B model
     (1, 512, 512, 64, False, True),
     (4, 4096, 256, 512, True, True),
+    (2304, 1024, 2304, 128, False, True),   # 81 tiles on 74 CTA pairs: a second, thin round of the persistent grid
+    (2200, 2048, 2560, 256, True, True),    # 90 tiles, ragged last row tile
+    (2304, 1024, 2304, 0, False, True),     # the same with an empty INT8 segment
 ])
 def test_mixed_gemm_bit_exact(resq, T, K, N, r, fp16, w4i8):
     _, _, pw, res = oracle_case(T, K, N, r, fp16, seed_shift=T)
