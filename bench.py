@@ -25,11 +25,26 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-WORKLOAD = "llama3-8b-decoder-block-linears-prefill-T4096"
-T_PREFILL = 4096
-# (name, K, n_out, online projection)
-LAYERS = [("qkv", 4096, 6144, False), ("o", 4096, 4096, False), ("gate_up", 4096, 28672, False),
-          ("down", 14336, 4096, True)]
+# The headline workload (--model 8b) and the two other block shapes of the benchmark configurations
+# (--model 1b / 70b: same legs, for the per-configuration table; not the headline line).
+# name -> (workload, prefill tokens, [(layer, K, n_out, online projection)])
+MODELS = {
+    "1b": ("llama3.2-1b-decoder-block-linears-prefill-T2048", 2048,
+           [("qkv", 2048, 3072, False), ("o", 2048, 2048, False), ("gate_up", 2048, 16384, False), ("down", 8192, 2048, True)]),
+    "8b": ("llama3-8b-decoder-block-linears-prefill-T4096", 4096,
+           [("qkv", 4096, 6144, False), ("o", 4096, 4096, False), ("gate_up", 4096, 28672, False), ("down", 14336, 4096, True)]),
+    "70b": ("llama3-70b-decoder-block-linears-prefill-T8192", 8192,
+            [("qkv", 8192, 10240, False), ("o", 8192, 8192, False), ("gate_up", 8192, 57344, False), ("down", 28672, 8192, True)]),
+}
+MODEL = "8b"
+WORKLOAD, T_PREFILL, LAYERS = MODELS[MODEL]
+
+
+def select_model(name: str):
+    global MODEL, WORKLOAD, T_PREFILL, LAYERS
+    MODEL = name
+    WORKLOAD, T_PREFILL, LAYERS = MODELS[name]
+
 ORACLE_SAMPLE_ROWS = 1024      # cpu_baseline leg of our arm: one pass, about 10-20 s of CPU work
 REFERENCE_STEP_ROWS = 64       # --impl reference: rows per step, so that K steps end within minutes
 NOMINAL = {"int8_tops": 4500.0, "bf16_tflops": 2250.0, "hbm_gbs": 7700.0}
@@ -109,9 +124,10 @@ class Layer:
     pass
 
 
-def build_layers(device, rows=T_PREFILL, with_weights=True, only=None):
+def build_layers(device, rows=None, with_weights=True, only=None):
     """Seeded synthetic inputs of the workload on `device` (activations, projected weights, P)."""
     import synth
+    rows = T_PREFILL if rows is None else rows
     layers = []
     for li, (name, K, N, online) in enumerate(LAYERS):
         if only and name not in only:
@@ -177,7 +193,7 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
         sets.append((L, desc, copies))
         weight_bytes += L.N * (L.r + (L.K - L.r) // 2) + 2 * 2 * L.N
     p_bytes = sum(2 * L.K * L.K for L in layers if L.online)
-    out = {"workload": "llama3-8b-decoder-block-linears-decode", "weight_bytes_per_step": weight_bytes,
+    out = {"workload": WORKLOAD.split("-prefill")[0] + "-decode", "weight_bytes_per_step": weight_bytes,
            "p_bytes_per_step": p_bytes, "weight_copies_cycled": DECODE_COPIES, "steps": steps}
     for T in DECODE_T:
         bufs = []
@@ -608,7 +624,7 @@ def run_ours(args):
         kernels["project_gemm"] = {"bound": "tensor", "dtype": "bf16",
                                    "achieved": round(2.0 * T * L.K * L.K / (g_ms * 1e-3) / 1e12, 1),
                                    "peak": round(bf16_peak, 1), "unit": "TFLOP/s", "ms_per_step": round(g_ms, 4),
-                                   "traffic": NCU_TRAFFIC_BYTES.get("project_gemm")}
+                                   "traffic": NCU_TRAFFIC_BYTES.get("project_gemm") if MODEL == "8b" else None}
     for k in kernels.values():
         k["frac"] = round(k["achieved"] / k["peak"], 4)
     # Dominant kernel: the single launch with the most time per step (the combined figure of the online
@@ -697,7 +713,7 @@ def run_ours(args):
 
     # ---- the attention-block path: U_C projection, mixed-precision KV cache, single-query attention
     kvp = None
-    if not args.no_kv and not only:
+    if not args.no_kv and not only and MODEL == "8b":
         kvp = kv_leg(resq, torch, dev, peaks, max(5, min(args.steps, 20)), args.kv_seqs, args.kv_len)
         kernels["attention_decode"] = {"bound": "hbm", "dtype": "f16", "achieved": kvp["attention_cache_stream_gbs"],
                                        "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -708,7 +724,7 @@ def run_ours(args):
     cpu_baseline, parity = None, None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        S = min(ORACLE_SAMPLE_ROWS, T)
+        S = min(ORACLE_SAMPLE_ROWS if MODEL != "70b" else 128, T)   # the 28672-wide fp64 projection is 4x the work per row
         hs = host_sample(layers, S)
         t0 = time.perf_counter()
         res = oracle_sample_step(hs)
@@ -796,8 +812,10 @@ def main():
     ap.add_argument("--kv-only", action="store_true", help="run only the attention-block leg (profiling runs)")
     ap.add_argument("--kv-seqs", type=int, default=16, help="sequences in the attention-block leg")
     ap.add_argument("--kv-len", type=int, default=8192, help="cached positions per sequence in the attention-block leg")
+    ap.add_argument("--model", default="8b", choices=sorted(MODELS), help="block shape: 8b is the headline workload")
     ap.add_argument("--layers", default="", help="comma-separated subset of qkv,o,gate_up,down (profiling runs)")
     args = ap.parse_args()
+    select_model(args.model)
     if args.impl == "reference":
         run_reference(args)
     else:
