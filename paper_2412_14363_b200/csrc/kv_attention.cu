@@ -456,20 +456,26 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
 
 // Merges the partial records of one (sequence, query head): out = sum_i 2^(m_i - M) o_i / sum_i 2^(m_i - M) l_i.
 // The warps that hold a record of this (sequence, KV head) are those whose runs meet its range of the block
-// list; they are taken 128 at a time: thread t reads (m, l) of candidate t, the block agrees on the maximum,
-// then every thread (one output coefficient each) adds the weighted records with eight loads in flight.
-// Launched so that it may start while the attention kernel drains: everything before griddepcontrol.wait
-// reads only the sequence lengths.
-__global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams p) {
-    __shared__ long long red[2][kD / 32];
-    __shared__ float redf[2][kD / 32];
-    __shared__ float f_s[kD];
-    __shared__ long long rec_s[kD];
+// list.  The CTA has 128 x G threads: candidates are taken blockDim at a time (thread t reads (m, l) of candidate
+// t, the block agrees on the maximum), then group g adds the weighted records g, g + G, ... eight at a time, one
+// output coefficient per thread, and the G partial sums are added in group order.  G = 4 when few (sequence, head)
+// pairs share the grid's warps (long contexts: hundreds of records each), else 1.  Launched so that it may start
+// while the attention kernel drains: everything before griddepcontrol.wait reads only the sequence lengths.
+constexpr int kMaxGroups = 4;
+__global__ void __launch_bounds__(kD * kMaxGroups) attention_combine_kernel(const AttnParams p) {
+    __shared__ long long red[2][kD * kMaxGroups / 32];
+    __shared__ float redf[2][kD * kMaxGroups / 32];
+    extern __shared__ __align__(16) uint8_t merge_smem[];  // rec_s [nthr] long long, f_s [nthr] float, num_s [groups][128] float
     const int n_q_heads = p.n_kv_heads * p.group;
     const int b = blockIdx.x / n_q_heads, hq = blockIdx.x - b * n_q_heads;
-    const int hk = hq / p.group, hg = hq - hk * p.group, d = threadIdx.x, warp = d >> 5;
+    const int hk = hq / p.group, hg = hq - hk * p.group;
+    const int tid = threadIdx.x, nthr = blockDim.x, nwarp = nthr >> 5, warp = tid >> 5;
+    const int d = tid & (kD - 1), grp = tid >> 7, groups = nthr >> 7;
+    long long* rec_s = reinterpret_cast<long long*>(merge_smem);
+    float* f_s = reinterpret_cast<float*>(rec_s + nthr);
+    float* num_s = f_s + nthr;
     long long before = 0, total = 0;
-    for (int i = d; i < p.n_seqs; i += kD) {
+    for (int i = tid; i < p.n_seqs; i += nthr) {
         const int len = p.seq_lens[i];
         if (blockIdx.x == 0 && (len < 0 || len > p.capacity)) atomicOr(p.status, RESQ_ERR_INDEX);
         const int t = ((len < 0 ? 0 : (len > p.capacity ? p.capacity : len)) + 31) >> 5;
@@ -481,14 +487,15 @@ __global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams 
         before += __shfl_xor_sync(0xffffffffu, before, o);
         total += __shfl_xor_sync(0xffffffffu, total, o);
     }
-    if ((d & 31) == 0) { red[0][warp] = before; red[1][warp] = total; }
+    if ((tid & 31) == 0) { red[0][warp] = before; red[1][warp] = total; }
     __syncthreads();
-    before = red[0][0] + red[0][1] + red[0][2] + red[0][3];
-    total = (red[1][0] + red[1][1] + red[1][2] + red[1][3]) * p.n_kv_heads;
+    before = total = 0;
+    for (int w = 0; w < nwarp; ++w) { before += red[0][w]; total += red[1][w]; }
+    total *= p.n_kv_heads;
     float* out = p.out + (static_cast<long long>(b) * n_q_heads + hq) * kD;
     const int nblk = (clamped_len(p.seq_lens, b, p.capacity) + 31) >> 5;
     if (nblk == 0) {  // empty sequence
-        out[d] = 0.f;
+        if (grp == 0) out[d] = 0.f;
         return;
     }
     const long long lo = before * p.n_kv_heads + static_cast<long long>(hk) * nblk, hi = lo + nblk;  // [lo, hi)
@@ -496,9 +503,9 @@ __global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams 
     const int w_first = static_cast<int>(((lo + 1) * nw - 1) / total), w_last = static_cast<int>((hi * nw - 1) / total);
     const long long s = static_cast<long long>(b) * p.n_kv_heads + hk;
     griddep_wait();
-    float M = -INFINITY, num = 0.f, den = 0.f;  // den is a per-thread partial until the end
-    for (int w0 = w_first; w0 <= w_last; w0 += kD) {
-        const int w = w0 + d;
+    float M = -INFINITY, num = 0.f, den = 0.f;  // num: this group's share; den: a per-thread partial until the end
+    for (int w0 = w_first; w0 <= w_last; w0 += nthr) {
+        const int w = w0 + tid;
         bool have = false;
         if (w <= w_last) {  // a non-empty run that meets [lo, hi)
             const long long rs = total * w / nw, re = total * (w + 1) / nw;
@@ -511,19 +518,20 @@ __global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams 
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         __syncthreads();  // the previous chunk's f_s / rec_s / redf are no longer read
-        if ((d & 31) == 0) redf[0][warp] = mx;
+        if ((tid & 31) == 0) redf[0][warp] = mx;
         __syncthreads();
-        const float Mn = fmaxf(M, fmaxf(fmaxf(redf[0][0], redf[0][1]), fmaxf(redf[0][2], redf[0][3])));
+        float Mn = M;
+        for (int k = 0; k < nwarp; ++k) Mn = fmaxf(Mn, redf[0][k]);
         const float resc = ex2(M - Mn);  // 0 on the first chunk
         M = Mn;
         const float f = have ? ex2(m - M) : 0.f;
-        f_s[d] = f;
-        rec_s[d] = have ? off + 2 : -1;
+        f_s[tid] = f;
+        rec_s[tid] = have ? off + 2 : -1;
         num *= resc;
         den = fmaf(f, lw, den * resc);
         __syncthreads();
-        const int cnt = min(kD, w_last - w0 + 1);
-        for (int i0 = 0; i0 < cnt; i0 += 8) {
+        const int cnt = min(nthr, w_last - w0 + 1);
+        for (int i0 = 8 * grp; i0 < cnt; i0 += 8 * groups) {
             float v[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
@@ -537,9 +545,15 @@ __global__ void __launch_bounds__(kD) attention_combine_kernel(const AttnParams 
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
     __syncthreads();
-    if ((d & 31) == 0) redf[1][warp] = den;
+    if ((tid & 31) == 0) redf[1][warp] = den;
+    num_s[grp * kD + d] = num;
     __syncthreads();
-    out[d] = num / (redf[1][0] + redf[1][1] + redf[1][2] + redf[1][3]);
+    if (grp == 0) {
+        float dsum = 0.f, nsum = 0.f;
+        for (int k = 0; k < nwarp; ++k) dsum += redf[1][k];
+        for (int g = 0; g < groups; ++g) nsum += num_s[g * kD + d];
+        out[d] = nsum / dsum;
+    }
 }
 
 }  // namespace
@@ -575,7 +589,10 @@ cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q1
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cache.n_seqs * n_q_heads, 1, 1);
-    cfg.blockDim = dim3(kD, 1, 1);
+    // few (sequence, head) pairs share the grid's warps: each has many records, so four groups of threads add them
+    const int merge_threads = cache.n_seqs * cache.n_kv_heads <= 64 ? kD * kMaxGroups : kD;
+    cfg.blockDim = dim3(merge_threads, 1, 1);
+    cfg.dynamicSmemBytes = static_cast<size_t>(merge_threads) * (sizeof(long long) + sizeof(float)) + (merge_threads / kD) * kD * sizeof(float);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
