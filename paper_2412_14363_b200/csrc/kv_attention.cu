@@ -229,12 +229,14 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
     uint32_t qf[8][2];
     float kq8[2], kq4[2], ko8[2], ko4[2], m_run[2], l[2], z8[2], z4[2], acc[8][4], ones8[4], ones4[4], wx8[2], wx4[2];
     bool fresh = true, ok = true;
+    int rec_blk0 = 0;  // block of the (sequence, head) at which the current record began
     long long i = 0;
     int stage = 0;
     uint32_t phase = 0;
     for (; i < n; ++i) {
         if (fresh) {  // a new (sequence, KV head): query fragments of its group, empty running state
             fresh = false;
+            rec_blk0 = cons.blk;
             const __half* qrow = p.q + (static_cast<long long>(cons.b) * p.n_kv_heads * p.group + cons.h * p.group + g) * kD;
             float s8 = 0.f, s4 = 0.f, o4 = 0.f;  // sums of q over the segments; offset-weighted sum of the 4-bit part
 #pragma unroll
@@ -414,31 +416,35 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
                     wx8[e] += __shfl_xor_sync(0xffffffffu, wx8[e], o);
                     wx4[e] += __shfl_xor_sync(0xffffffffu, wx4[e], o);
                 }
+            // A warp that saw every block of the (sequence, head) writes the final output itself (the merge kernel
+            // finds a single owner by the same run arithmetic and leaves at once); otherwise a partial record.
+            const bool sole = rec_blk0 == 0 && cons.blk == cons.nblk - 1;
             float* rec = p.partial + (wg + static_cast<long long>(cons.b) * p.n_kv_heads + cons.h) * kRecFloats;
+            float* fin = p.out + (static_cast<long long>(cons.b) * p.n_kv_heads + cons.h) * p.group * kD;
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 if (2 * c + e >= p.group) continue;
-                float* r = rec + (2 * c + e) * (kD + 2);
-                if (g == 0) { r[0] = m_run[e]; r[1] = l[e]; }
-                r += 2;
+                float* r = sole ? fin + (2 * c + e) * kD : rec + (2 * c + e) * (kD + 2) + 2;
+                const float nrm = sole ? 1.f / l[e] : 1.f;
+                if (!sole && g == 0) { r[-2] = m_run[e]; r[-1] = l[e]; }
                 // Rows g of the output products carry offset kOffLo, rows g + 8 kOffLo (8-bit) or kOffHi (4-bit).  The
                 // codes are also centred: sum w^ (c - mid) + mid * sum w with w^ the half-rounded and w the exact
                 // weights (ones: sum w^, wx: sum w), which halves the effect of the rounding (|c - mid| <= range / 2).
                 const float f8 = z8[e] - (kOffLo + kMid8) * ones8[e] + kMid8 * wx8[e];
                 const float f4lo = z4[e] - (kOffLo + kMid4) * ones4[e] + kMid4 * wx4[e];
                 const float f4hi = z4[e] - (kOffHi + kMid4) * ones4[e] + kMid4 * wx4[e];
-                r[2 * g] = acc[0][e] + f8;
-                r[2 * g + 1] = acc[0][2 + e] + f8;
+                r[2 * g] = (acc[0][e] + f8) * nrm;
+                r[2 * g + 1] = (acc[0][2 + e] + f8) * nrm;
 #pragma unroll
                 for (int i3 = 0; i3 < 3; ++i3) {
                     const int d0 = 16 + 4 * (g + 8 * i3);
-                    r[d0] = acc[1 + 2 * i3][e] + f4lo;
-                    r[d0 + 1] = acc[1 + 2 * i3][2 + e] + f4hi;
-                    r[d0 + 2] = acc[2 + 2 * i3][e] + f4lo;
-                    r[d0 + 3] = acc[2 + 2 * i3][2 + e] + f4hi;
+                    r[d0] = (acc[1 + 2 * i3][e] + f4lo) * nrm;
+                    r[d0 + 1] = (acc[1 + 2 * i3][2 + e] + f4hi) * nrm;
+                    r[d0 + 2] = (acc[2 + 2 * i3][e] + f4lo) * nrm;
+                    r[d0 + 3] = (acc[2 + 2 * i3][2 + e] + f4hi) * nrm;
                 }
-                r[112 + 2 * g] = acc[7][e] + f4lo;
-                r[113 + 2 * g] = acc[7][2 + e] + f4hi;
+                r[112 + 2 * g] = (acc[7][e] + f4lo) * nrm;
+                r[113 + 2 * g] = (acc[7][2 + e] + f4hi) * nrm;
             }
             fresh = true;
         }
@@ -501,6 +507,7 @@ __global__ void __launch_bounds__(kD * kMaxGroups) attention_combine_kernel(cons
     const long long lo = before * p.n_kv_heads + static_cast<long long>(hk) * nblk, hi = lo + nblk;  // [lo, hi)
     constexpr long long nw = kNumWarps;
     const int w_first = static_cast<int>(((lo + 1) * nw - 1) / total), w_last = static_cast<int>((hi * nw - 1) / total);
+    if (w_first == w_last) return;  // one warp saw the whole (sequence, head) and wrote the output itself
     const long long s = static_cast<long long>(b) * p.n_kv_heads + hk;
     griddep_wait();
     float M = -INFINITY, num = 0.f, den = 0.f;  // num: this group's share; den: a per-thread partial until the end
