@@ -120,7 +120,9 @@ int resq_pack_weights_projected(const resq_layer_desc_t* desc, const void* W_raw
  *              folded into the preceding layer's weights (Section 4.3, U_A/U_B).
  *   P != NULL: bf16 [K][K], row i = input feature, column j = coefficient; C = X·P is formed online
  *              on the tensor cores with fp32 accumulation (Section 4.3, U_D for the down_proj input)
- *              and quantized from fp32 without an intermediate bf16 rounding.  Needs workspace.
+ *              and quantized from fp32 without an intermediate bf16 rounding.  Needs workspace
+ *              (the fp32 panel; what resq_workspace_bytes adds beyond it is the projection GEMM's
+ *              scratch, see resq_project -- a workspace that only holds the panel is accepted too).
  * Outputs: x8 int8 [T][r]; x4 packed uint8 [T][(K-r)/2]; s_x8, s_x4 fp32 [T].
  * x4_i8 (optional, may be NULL): the INT4 codes one per byte, int8 [T][K-r].
  */
