@@ -43,7 +43,8 @@ def _run(resq, X_bits, r):
 
 
 @pytest.mark.parametrize("T,K,r", [(5, 64, 0), (16, 1024, 0), (33, 1024, 128), (7, 384, 0), (9, 896, 0), (20, 3072, 384),
-                                   (300, 8192, 0), (130, 14336, 0), (3, 14336, 1792), (2, 28672, 0)])
+                                   (300, 8192, 0), (130, 14336, 0), (3, 14336, 1792), (2, 28672, 0),
+                                   (11, 1792, 0), (6, 3584, 448), (4, 7168, 0)])  # 28 * 2^6..8: register path with 1, 2, 4 warps
 def test_hadamard_quantize_codes(resq, T, K, r):
     X = synth.activations(T, K, "t4", seed=600 + T)
     X_bits = synth.f32_to_bf16_bits(X)
