@@ -191,7 +191,7 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
                                                   x4 ? x4 + static_cast<size_t>(t0) * K4 / 2 : nullptr, s_x8 + t0,
                                                   s_x4 + t0, false,
                                                   x4_i8 ? x4_i8 + static_cast<size_t>(t0) * K4 : nullptr,
-                                                  static_cast<size_t>(K) * 4, st);
+                                                  static_cast<size_t>(K) * 4, st, true);
             e != cudaSuccess)
             return cuda_status(e);
     }

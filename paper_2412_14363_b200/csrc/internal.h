@@ -16,11 +16,11 @@ int* device_status_ptr();  // device address of the status word of the current d
 // Split quantization of the rows of a [rows][K] matrix (Eq. 2 for activations, Eq. 3 for weights).
 //   in_is_f32: rows are fp32 (weights, projected coefficients) instead of bf16.
 //   scale_fp16: scales are rounded to and stored as fp16 (weights only).
-//   absmax_bits: optional [rows][2] uint32 bit patterns of the precomputed per-segment absmax
-//                (written by the projection GEMM's epilogue); NULL = compute here.
+//   programmatic: enqueue with programmatic stream serialization (the kernel waits for the preceding grid itself,
+//                 so its CTAs can be scheduled while that grid drains); only the whole-row kernel honours it.
 cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, int K, int r, int8_t* q8,
                                   uint8_t* q4, void* s8, void* s4, bool scale_fp16, int8_t* q4_i8,
-                                  size_t in_row_stride, cudaStream_t st);
+                                  size_t in_row_stride, cudaStream_t st, bool programmatic = false);
 
 // Hadamard transform of the bf16 rows (H_K / sqrt(K), K = 2^k * {1, 12, 28}) fused with the split quantizer
 // (r may be 0).  Returns cudaErrorNotSupported for other K or rows wider than 200 KB of fp32.

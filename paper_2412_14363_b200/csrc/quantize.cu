@@ -227,6 +227,9 @@ split_quantize_fast_kernel(const void* __restrict__ in, size_t in_row_bytes, siz
     // A kernel enqueued behind this one with programmatic stream serialization may start its own
     // input-independent prologue now; it still waits for this grid to finish before reading the codes.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Enqueued with programmatic stream serialization itself (behind the projection GEMM), this grid may have been
+    // scheduled before its input was complete: wait for the preceding grid (returns at once otherwise).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t row_bytes = static_cast<uint32_t>(K) * (F32 ? 4u : 2u);
     const size_t row0 = static_cast<size_t>(blockIdx.x) * rows_per_cta;
     const int nrows = static_cast<int>(rows - row0 < static_cast<size_t>(rows_per_cta) ? rows - row0 : rows_per_cta);
@@ -538,7 +541,7 @@ void paley2(int q, float* H /* [2(q+1)]^2 */) {
 
 cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, int K, int r, int8_t* q8,
                                   uint8_t* q4, void* s8, void* s4, bool scale_fp16, int8_t* q4_i8,
-                                  size_t in_row_stride_bytes, cudaStream_t st) {
+                                  size_t in_row_stride_bytes, cudaStream_t st, bool programmatic) {
     if (rows == 0) return cudaSuccess;
     const size_t row_bytes = static_cast<size_t>(K) * (in_is_f32 ? 4 : 2);
     if (!scale_fp16 && row_bytes <= static_cast<size_t>(kFastMaxRowBytes) && in_row_stride_bytes % 16 == 0) {
@@ -557,10 +560,18 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
         }
         const size_t groups = (rows + rpc - 1) / rpc;
         if (groups <= 0x7fffffffu) {
-            kern<<<static_cast<unsigned>(groups), kThreads, smem, st>>>(in, in_row_stride_bytes, rows, K, r, rpc, q8, q4,
-                                                                    static_cast<float*>(s8), static_cast<float*>(s4),
-                                                                    q4_i8, device_status_ptr());
-            return cudaGetLastError();
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(static_cast<unsigned>(groups), 1, 1);
+            cfg.blockDim = dim3(kThreads, 1, 1);
+            cfg.dynamicSmemBytes = smem;
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = programmatic ? 1 : 0;
+            return cudaLaunchKernelEx(&cfg, kern, in, in_row_stride_bytes, rows, K, r, rpc, q8, q4,
+                                      static_cast<float*>(s8), static_cast<float*>(s4), q4_i8, device_status_ptr());
         }
     }
     const unsigned grid = static_cast<unsigned>(rows < 148u * 64u ? rows : 148u * 64u);

@@ -130,6 +130,33 @@ def test_projection_with_split_last_round(resq, T, K):
     assert (outs[0] != outs[2]).any()          # the split really changed the summation order somewhere
 
 
+@pytest.mark.parametrize("T,K", [(1, 512), (5, 1056), (16, 2048), (17, 4096), (33, 2304), (48, 1280), (64, 4096),
+                                 (3, 14336), (16, 14336)])
+def test_projection_few_token_rows(resq, T, K):
+    """Up to 64 token rows take the kernel with the operand roles exchanged (columns of P on the MMA's rows, tokens on
+    its columns, rounded up to 16), every tile cut along K when the scratch workspace is there.  Same bound as the
+    tile kernel's; rows the call does not own stay untouched; repeated calls give identical bits."""
+    X_bits = synth.f32_to_bf16_bits(synth.activations(T, K, "t4", seed=1100 + T))
+    P_bits = synth.f32_to_bf16_bits(synth.kron_orthogonal_bf16(K, inner=32 if K % 128 else 128))
+    C_ref = oracle.project(X_bits, P_bits).astype(np.float64)
+    Xd, Pd = bf16_to_dev(X_bits), bf16_to_dev(P_bits)
+    ws = torch.empty(resq.resq_project_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)
+    Xf = np.abs(synth.bf16_bits_to_f32(X_bits).astype(np.float64))
+    Pf = np.abs(synth.bf16_bits_to_f32(P_bits).astype(np.float64))
+    bound = (K // 16 + 20) * 2.0 ** -24 * (Xf @ Pf) + 1e-30
+    outs = []
+    for w in (ws, ws, None):
+        buf = torch.full((T + 2, K), float("nan"), dtype=torch.float32, device="cuda")
+        resq.resq_project(Xd, Pd, buf[1:T + 1], w)
+        assert resq.resq_device_status() == resq.OK
+        got = host(buf)
+        assert np.isnan(got[0]).all() and np.isnan(got[T + 1]).all()
+        assert (np.abs(got[1:T + 1].astype(np.float64) - C_ref) <= bound).all()
+        outs.append(got[1:T + 1])
+    assert (outs[0].view(np.uint32) == outs[1].view(np.uint32)).all()
+
+
 @pytest.mark.parametrize("N,K,r,fp16", [(64, 512, 64, False), (4104, 1024, 128, False), (264, 2048, 256, True)])
 def test_pack_weights_projected(resq, N, K, r, fp16):
     """Weight projection at pack time (Section 4.3): W_raw·U on the tensor cores, then Eq. 3.  Against the oracle's
