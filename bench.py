@@ -244,6 +244,22 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
             step(i)
         t1 = ev()
         torch.cuda.synchronize()
+        # The block through resq_linear, the call a user makes: without P and with T <= 16 it is ONE launch per layer
+        # (the streaming kernel quantizes the rows itself); down_proj runs projection, reduce, quantizer, GEMV.
+        def linear_chain(i):
+            for (L, desc, copies), b in zip(sets, bufs):
+                resq.resq_linear(copies[i % DECODE_COPIES], b["X"], L.P if L.online else None, b["Y"], b["ws"])
+
+        for i in range(3):
+            linear_chain(i)
+        torch.cuda.synchronize()
+        torch.cuda._sleep(HOST_LEAD_CYCLES)
+        l0 = ev()
+        for i in range(steps):
+            linear_chain(i)
+        l1 = ev()
+        torch.cuda.synchronize()
+        total_linear = l0.elapsed_time(l1) / steps
         # The same GEMV chain with asymmetric activation codes (unsigned codes, zero-points, weight row sums).
         ab = []
         for (L, desc, copies), b in zip(sets, bufs):
@@ -283,8 +299,9 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
                         "folded_quantize_us": round(quant * 1e3, 2),
                         "online_projection_us": round(proj * 1e3, 2),
                         "online_projection_p_stream_gbs": round(p_bytes / (proj * 1e-3) / 1e9, 1) if proj > 0 else None,
-                        "block_linears_us": round(total * 1e3, 2),
-                        "tokens_per_s": round(T / (total * 1e-3), 1)}
+                        "block_split_calls_us": round(total * 1e3, 2),
+                        "block_linears_us": round(total_linear * 1e3, 2),
+                        "tokens_per_s": round(T / (total_linear * 1e-3), 1)}
     resq.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 0)
     st = resq.resq_device_status()
     if st != resq.OK:

@@ -76,6 +76,47 @@ def test_decode_linear_end_to_end(resq, T):
     check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))
 
 
+@pytest.mark.parametrize("T,K,N,r,fp16", [
+    (1, 4096, 4096, 512, True), (4, 4096, 1024, 512, True), (16, 4096, 4096, 512, True),
+    (9, 2048, 264, 256, False),     # second token tile partly filled
+    (8, 512, 512, 64, False), (3, 1056, 72, 96, False),
+    (16, 8192, 256, 1024, True),
+    (5, 14336, 128, 1792, True), (16, 4096, 28672, 512, True),
+    (7, 2048, 64, 0, False),        # uniform INT4: no INT8 segment
+])
+def test_decode_linear_shapes_and_zero_rows(resq, T, K, N, r, fp16):
+    """resq_linear for up to 16 tokens without P (row quantizer, then the streaming kernel) over the shapes of the
+    streaming kernel's own cases: the output bits of the oracle's layer; a zero row and a row whose INT8 segment is
+    zero give scale 0 and codes 0; the split calls give the same bits."""
+    C_bits, Wp, _, _ = oracle_case(T, K, N, r, fp16, seed_shift=170 + T)
+    C_bits = C_bits.copy()
+    if T >= 3:
+        C_bits[1, :] = 0
+        C_bits[2, :r] = 0
+    pw = oracle.pack_weights(Wp, r, scale_fp16=fp16)
+    res = oracle.linear(C_bits, None, pw)
+    desc = resq.layer_desc(K, N, r, resq.SCALE_FP16 if fp16 else resq.SCALE_FP32)
+    W = resq.resq_pack_weights(desc, dev(Wp), with_w4_i8=False)
+    ws = resq.alloc_workspace(desc, T, False, False)
+    y32 = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+    resq.resq_linear(W, bf16_to_dev(C_bits), None, y32, ws)
+    ybf = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    resq.resq_linear(W, bf16_to_dev(C_bits), None, ybf, ws)
+    assert resq.resq_device_status() == resq.OK
+    check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))
+    # the same through the split entry points
+    K4 = K - r
+    x8 = torch.empty((T, max(r, 1)), dtype=torch.int8, device="cuda")
+    x4 = torch.empty((T, K4 // 2), dtype=torch.uint8, device="cuda")
+    s8 = torch.empty(T, dtype=torch.float32, device="cuda")
+    s4 = torch.empty(T, dtype=torch.float32, device="cuda")
+    resq.resq_project_quantize(bf16_to_dev(C_bits), None, r, x8, x4, s8, s4, None, None)
+    y2 = torch.empty((T, N), dtype=torch.float32, device="cuda")
+    resq.resq_mixed_gemm(W, x8, x4, s8, s4, y2, ws)
+    assert resq.resq_device_status() == resq.OK
+    assert (host(y2).view(np.uint32) == host(y32).view(np.uint32)).all()
+
+
 def test_decode_early_weights_back_to_back(resq):
     """With the early-weights option each launch may start while the previous one still runs and
     prefetches its weights before waiting for it; a chain of launches over different layers must give
