@@ -107,11 +107,16 @@ __device__ __forceinline__ Item item_info(const Params& p, int item) {
         it.ld = static_cast<size_t>(p.K);
         it.bounded = true;
     } else {
-        const int j = item - p.full_items, t = j / p.splits, sl = j - t * p.splits;
+        const int j = item - p.full_items;
+        int t = j / p.splits, sl = j - t * p.splits;
+        if (p.full_items == 0) {  // every tile is cut: slice-major, so that the pairs of a round read the same rows of P
+            sl = j / p.split_tiles;
+            t = j - sl * p.split_tiles;
+        }
         tile_coords(p, p.full_items + t, it.m0, it.n0);
         it.kb0 = sl * p.kb_slice;
         it.nkb = min(p.kb_slice, p.kb_total - it.kb0);
-        it.dst = p.partial + static_cast<size_t>(j) * p.prows * BN;
+        it.dst = p.partial + static_cast<size_t>(t * p.splits + sl) * p.prows * BN;
         it.ld = BN;
         it.bounded = false;
     }
