@@ -404,8 +404,48 @@ def hadamard_leg(resq, torch, dev, L, T, steps, peaks):
     st = resq.resq_device_status()
     if st != resq.OK:
         raise SystemExit(f"device status {st}: {resq.status_string(st)}")
+    # The same layer for a generation step (T = 1, 4, 16): transform + quantize, then the streaming kernel on packed
+    # INT4 weights; five weight copies (> L2 together) are cycled so that every weight byte comes from DRAM.
+    copies = [resq.resq_pack_weights(desc, L.W_proj, with_w4_i8=False) for _ in range(5)]
+    few = {}
+    for Tf in DECODE_T:
+        Xf = L.X[:Tf].contiguous()
+        x4 = torch.empty((Tf, L.K // 2), dtype=torch.uint8, device=dev)
+        f8 = torch.empty(Tf, dtype=torch.float32, device=dev)
+        f4 = torch.empty(Tf, dtype=torch.float32, device=dev)
+        Yf = torch.empty((Tf, L.N), dtype=torch.bfloat16, device=dev)
+        wsf = resq.alloc_workspace(desc, Tf, False, False, device=dev)
+
+        def few_step(i, events=None):
+            e0 = ev() if events is not None else None
+            resq.resq_hadamard_quantize(Xf, 0, None, x4, f8, f4, None)
+            e1 = ev() if events is not None else None
+            resq.resq_mixed_gemm(copies[i % len(copies)], None, x4, f8, f4, Yf, wsf)
+            if events is not None:
+                events.append((e0, e1, ev()))
+
+        for i in range(3):
+            few_step(i)
+        torch.cuda.synchronize()
+        fev = []
+        for i in range(steps):
+            few_step(i, fev)
+        torch.cuda.synchronize()
+        torch.cuda._sleep(HOST_LEAD_CYCLES)
+        c0 = ev()
+        for i in range(steps):
+            few_step(i)
+        c1 = ev()
+        torch.cuda.synchronize()
+        few[f"T{Tf}"] = {"hadamard_quantize_us": round(statistics.mean(a.elapsed_time(b) for a, b, _ in fev) * 1e3, 2),
+                         "int4_gemv_us": round(statistics.mean(b.elapsed_time(c) for _, b, c in fev) * 1e3, 2),
+                         "layer_us": round(c0.elapsed_time(c1) / steps * 1e3, 2)}
+    st = resq.resq_device_status()
+    if st != resq.OK:
+        raise SystemExit(f"device status {st}: {resq.status_string(st)}")
     bytes_q = T * (2.0 * L.K + L.K + 8)   # read bf16, write one code per byte + scales
     return {"workload": f"down_proj {L.K}->{L.N}, T={T}: Hadamard U_D + uniform INT4 (r = 0)", "steps": steps,
+            "few_tokens": few,
             "hadamard_quantize_ms": round(q, 4), "hadamard_quantize_gbs": round(bytes_q / (q * 1e-3) / 1e9, 1),
             "hadamard_quantize_frac_of_hbm_peak": round(bytes_q / (q * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
             "int4_gemm_ms": round(g, 4), "int4_gemm_tops": round(2.0 * T * L.K * L.N / (g * 1e-3) / 1e12, 1),

@@ -359,29 +359,43 @@ __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* _
 // Sylvester butterflies three index bits per pass (eight values in registers, conflict-free strides),
 // scaled, and then quantized exactly as in the fast path above (absmax per segment, reciprocal-product
 // rounding with the exact fallback).  r = 0 gives the paper's uniform INT4 down_proj input.
+constexpr int kWideThreads = 1024;  // threads per row when there are at most kWideMaxRows rows (one CTA per SM)
+constexpr int kWideMaxRows = 148;
 __constant__ float c_paley12[12 * 12];
 __constant__ float c_paley28[28 * 28];
+// The same factors in global memory: the few-row variant copies its factor to shared memory with one batch of
+// loads, since a single CTA would wait for the constant cache to fill line by line (no other CTA shares the cost).
+__device__ float g_paley12[12 * 12];
+__device__ float g_paley28[28 * 28];
 
 template <int M>
 __device__ __forceinline__ const float* small_factor() {
     return M == 12 ? c_paley12 : c_paley28;
 }
 
-template <int M>
-__global__ void __launch_bounds__(kThreads)
+// NT threads per row: 256 when rows outnumber the SMs (throughput: several CTAs per SM), 1024 for the few rows of a
+// generation step, where one row's chain of passes is all there is to wait for.
+template <int M, int NT>
+__global__ void __launch_bounds__(NT)
 hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K, int kbits, int r, float inv_sqrt_k,
                          int8_t* __restrict__ q8, uint8_t* __restrict__ q4, float* __restrict__ s8_out,
                          float* __restrict__ s4_out, int8_t* __restrict__ q4e) {
     extern __shared__ __align__(16) float hrow[];  // [K]
-    __shared__ float red[2][kThreads / 32];
+    __shared__ float red[2][NT / 32];
+    constexpr bool kStagedFactor = NT == kWideThreads && M > 1;
+    __shared__ __align__(16) float hfac[kStagedFactor ? M * M : 4];
     const int tid = threadIdx.x;
+    if constexpr (kStagedFactor) {
+        const float* g = M == 12 ? g_paley12 : g_paley28;
+        for (int i = tid; i < M * M; i += NT) hfac[i] = g[i];  // visible after the barrier that follows step 1
+    }
     const int nchunks = K >> 3, rchunks = r >> 3;
     const int K4 = K - r;
     const uint8_t* srow = reinterpret_cast<const uint8_t*>(hrow);
     for (size_t row = blockIdx.x; row < rows; row += gridDim.x) {
         // 1. widen the bf16 row
         const uint4* xp = reinterpret_cast<const uint4*>(X + row * static_cast<size_t>(K));
-        for (int c = tid; c < nchunks; c += kThreads) {
+        for (int c = tid; c < nchunks; c += NT) {
             const uint4 u = __ldg(xp + c);
             const uint32_t w[4] = {u.x, u.y, u.z, u.w};
             float4 a, b;
@@ -395,8 +409,8 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
         __syncthreads();
         // 2. the small factor, one group of M consecutive coefficients per thread, in place
         if constexpr (M > 1) {
-            const float* H = small_factor<M>();
-            for (int a = tid; a < (K / M); a += kThreads) {
+            const float* H = kStagedFactor ? hfac : small_factor<M>();
+            for (int a = tid; a < (K / M); a += NT) {
                 // M * 4 bytes is a multiple of 16: the group moves as float4s (conflict-free at this stride)
                 float4* gp = reinterpret_cast<float4*>(hrow + a * M);
                 float x[M], y[M];
@@ -424,7 +438,7 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
             const int nb = kbits - s < 3 ? kbits - s : 3;
             const int count = K >> nb;
             const int stride = M << s;
-            for (int i = tid; i < count; i += kThreads) {
+            for (int i = tid; i < count; i += NT) {
                 const int arest = i / M, b = i - arest * M;
                 const int a0 = ((arest >> s) << (s + nb)) | (arest & ((1 << s) - 1));
                 float* base = hrow + a0 * M + b;
@@ -452,7 +466,7 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
         }
         // 4. scale by 1 / sqrt(K) and take the two absmax values
         float a8 = 0.f, a4 = 0.f;
-        for (int c = tid; c < nchunks; c += kThreads) {
+        for (int c = tid; c < nchunks; c += NT) {
             float4* p = reinterpret_cast<float4*>(hrow) + 2 * c;
             float4 a = p[0], b = p[1];
             a.x *= inv_sqrt_k; a.y *= inv_sqrt_k; a.z *= inv_sqrt_k; a.w *= inv_sqrt_k;
@@ -474,7 +488,7 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
         }
         __syncthreads();  // also: every thread's scaled values are in place
 #pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) {
+        for (int w = 0; w < NT / 32; ++w) {
             a8 = fmaxf(a8, red[0][w]);
             a4 = fmaxf(a4, red[1][w]);
         }
@@ -490,7 +504,7 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
         int8_t* q8row = q8 + row * static_cast<size_t>(r);
         uint8_t* q4row = q4 ? q4 + row * static_cast<size_t>(K4 >> 1) : nullptr;
         int8_t* q4e_row = q4e ? q4e + row * static_cast<size_t>(K4) : nullptr;
-        for (int c = tid; c < nchunks; c += kThreads) {
+        for (int c = tid; c < nchunks; c += NT) {
             uint32_t t[8];
             const bool seg8 = c < rchunks;
             const float s = seg8 ? s8 : s4;
@@ -629,7 +643,11 @@ cudaError_t launch_hadamard_quantize(const void* X, size_t rows, int K, int r, i
         paley2(13, h28);
         if ((e = cudaMemcpyToSymbol(c_paley12, h12, sizeof(h12))) != cudaSuccess) return e;
         if ((e = cudaMemcpyToSymbol(c_paley28, h28, sizeof(h28))) != cudaSuccess) return e;
-        for (auto k : {hadamard_quantize_kernel<1>, hadamard_quantize_kernel<12>, hadamard_quantize_kernel<28>})
+        if ((e = cudaMemcpyToSymbol(g_paley12, h12, sizeof(h12))) != cudaSuccess) return e;
+        if ((e = cudaMemcpyToSymbol(g_paley28, h28, sizeof(h28))) != cudaSuccess) return e;
+        for (auto k : {hadamard_quantize_kernel<1, kThreads>, hadamard_quantize_kernel<12, kThreads>,
+                       hadamard_quantize_kernel<28, kThreads>, hadamard_quantize_kernel<1, kWideThreads>,
+                       hadamard_quantize_kernel<12, kWideThreads>, hadamard_quantize_kernel<28, kWideThreads>})
             if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess)
                 return e;
         ready[dev] = true;
@@ -637,9 +655,15 @@ cudaError_t launch_hadamard_quantize(const void* X, size_t rows, int K, int r, i
     const float inv_sqrt_k = static_cast<float>(1.0 / sqrt(static_cast<double>(K)));
     const unsigned grid = static_cast<unsigned>(rows < 148u * 16u ? rows : 148u * 16u);
     const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(X);
-    if (m == 1) hadamard_quantize_kernel<1><<<grid, kThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
-    else if (m == 12) hadamard_quantize_kernel<12><<<grid, kThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
-    else hadamard_quantize_kernel<28><<<grid, kThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
+    if (rows <= kWideMaxRows) {
+        if (m == 1) hadamard_quantize_kernel<1, kWideThreads><<<grid, kWideThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
+        else if (m == 12) hadamard_quantize_kernel<12, kWideThreads><<<grid, kWideThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
+        else hadamard_quantize_kernel<28, kWideThreads><<<grid, kWideThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
+        return cudaGetLastError();
+    }
+    if (m == 1) hadamard_quantize_kernel<1, kThreads><<<grid, kThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
+    else if (m == 12) hadamard_quantize_kernel<12, kThreads><<<grid, kThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
+    else hadamard_quantize_kernel<28, kThreads><<<grid, kThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
     return cudaGetLastError();
 }
 
