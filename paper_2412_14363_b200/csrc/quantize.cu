@@ -359,20 +359,30 @@ __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* _
 // Sylvester butterflies three index bits per pass (eight values in registers, conflict-free strides),
 // scaled, and then quantized exactly as in the fast path above (absmax per segment, reciprocal-product
 // rounding with the exact fallback).  r = 0 gives the paper's uniform INT4 down_proj input.
+// Paley's second construction for a prime q = 1 (mod 4): H = S (x) [[1,1],[1,-1]] + I (x) [[1,-1],[-1,-1]] of order
+// 2 (q + 1), with S = [[0, 1^T], [1, chi(i - j)]] and chi the quadratic character of GF(q).  S is evaluated at compile
+// time, so the product with H is additions and subtractions only: with p_i = x_2i + x_2i+1 and m_i = x_2i - x_2i+1,
+//   y_2j = m_j + sum_i S_ij p_i,   y_2j+1 = -p_j + sum_i S_ij m_i      (M / 2 * (M - 2) + 2 M operations, not M * M).
+constexpr int quad_char(int q, int a) {
+    a = ((a % q) + q) % q;
+    if (a == 0) return 0;
+    for (int x = 1; x < q; ++x)
+        if ((x * x) % q == a) return 1;
+    return -1;
+}
+template <int M>
+struct Conference {
+    int s[M / 2][M / 2];
+    constexpr Conference() : s() {
+        constexpr int q = M / 2 - 1;
+        for (int i = 0; i < M / 2; ++i)
+            for (int j = 0; j < M / 2; ++j)
+                s[i][j] = i == 0 ? (j == 0 ? 0 : 1) : (j == 0 ? 1 : quad_char(q, (i - 1) - (j - 1)));
+    }
+};
+
 constexpr int kWideThreads = 1024;  // threads per row when there are at most kWideMaxRows rows (one CTA per SM)
 constexpr int kWideMaxRows = 148;
-__constant__ float c_paley12[12 * 12];
-__constant__ float c_paley28[28 * 28];
-// The same factors in global memory: the few-row variant copies its factor to shared memory with one batch of
-// loads, since a single CTA would wait for the constant cache to fill line by line (no other CTA shares the cost).
-__device__ float g_paley12[12 * 12];
-__device__ float g_paley28[28 * 28];
-
-template <int M>
-__device__ __forceinline__ const float* small_factor() {
-    return M == 12 ? c_paley12 : c_paley28;
-}
-
 // NT threads per row: 256 when rows outnumber the SMs (throughput: several CTAs per SM), 1024 for the few rows of a
 // generation step, where one row's chain of passes is all there is to wait for.
 template <int M, int NT>
@@ -382,13 +392,7 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
                          float* __restrict__ s4_out, int8_t* __restrict__ q4e) {
     extern __shared__ __align__(16) float hrow[];  // [K]
     __shared__ float red[2][NT / 32];
-    constexpr bool kStagedFactor = NT == kWideThreads && M > 1;
-    __shared__ __align__(16) float hfac[kStagedFactor ? M * M : 4];
     const int tid = threadIdx.x;
-    if constexpr (kStagedFactor) {
-        const float* g = M == 12 ? g_paley12 : g_paley28;
-        for (int i = tid; i < M * M; i += NT) hfac[i] = g[i];  // visible after the barrier that follows step 1
-    }
     const int nchunks = K >> 3, rchunks = r >> 3;
     const int K4 = K - r;
     const uint8_t* srow = reinterpret_cast<const uint8_t*>(hrow);
@@ -409,24 +413,32 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
         __syncthreads();
         // 2. the small factor, one group of M consecutive coefficients per thread, in place
         if constexpr (M > 1) {
-            const float* H = kStagedFactor ? hfac : small_factor<M>();
+            constexpr Conference<M> conf{};
+            constexpr int H2 = M / 2;
             for (int a = tid; a < (K / M); a += NT) {
                 // M * 4 bytes is a multiple of 16: the group moves as float4s (conflict-free at this stride)
                 float4* gp = reinterpret_cast<float4*>(hrow + a * M);
-                float x[M], y[M];
+                float x[M], y[M], ps[H2], ms[H2];
 #pragma unroll
                 for (int i = 0; i < M / 4; ++i) {
                     const float4 v = gp[i];
                     x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
                 }
 #pragma unroll
-                for (int i = 0; i < M; ++i) asm volatile("" : "+f"(x[i]));  // keep the group in registers
+                for (int i = 0; i < H2; ++i) {
+                    ps[i] = x[2 * i] + x[2 * i + 1];
+                    ms[i] = x[2 * i] - x[2 * i + 1];
+                }
 #pragma unroll
-                for (int j = 0; j < M; ++j) y[j] = 0.f;
+                for (int j = 0; j < H2; ++j) {
+                    float e = ms[j], o = -ps[j];
 #pragma unroll
-                for (int i = 0; i < M; ++i) {
-#pragma unroll
-                    for (int j = 0; j < M; ++j) y[j] = fmaf(x[i], H[i * M + j], y[j]);
+                    for (int i = 0; i < H2; ++i) {
+                        if (conf.s[i][j] > 0) { e += ps[i]; o += ms[i]; }
+                        else if (conf.s[i][j] < 0) { e -= ps[i]; o -= ms[i]; }
+                    }
+                    y[2 * j] = e;
+                    y[2 * j + 1] = o;
                 }
 #pragma unroll
                 for (int i = 0; i < M / 4; ++i) gp[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
@@ -531,26 +543,6 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
     }
 }
 
-// Paley's second construction for a prime q = 1 (mod 4): a Hadamard matrix of order 2 (q + 1) from the
-// quadratic character chi of GF(q): S = [[0, 1^T], [1, chi(i - j)]], H = S (x) [[1,1],[1,-1]] + I (x) [[1,-1],[-1,-1]].
-void paley2(int q, float* H /* [2(q+1)]^2 */) {
-    const int n = q + 1, N = 2 * n;
-    auto chi = [q](int a) {
-        a = ((a % q) + q) % q;
-        if (a == 0) return 0;
-        for (int x = 1; x < q; ++x)
-            if ((x * x) % q == a) return 1;
-        return -1;
-    };
-    auto S = [&](int i, int j) { return i == 0 ? (j == 0 ? 0 : 1) : (j == 0 ? 1 : chi((i - 1) - (j - 1))); };
-    const int A[2][2] = {{1, 1}, {1, -1}}, B[2][2] = {{1, -1}, {-1, -1}};
-    for (int i = 0; i < n; ++i)
-        for (int j = 0; j < n; ++j)
-            for (int u = 0; u < 2; ++u)
-                for (int v = 0; v < 2; ++v)
-                    H[(2 * i + u) * N + 2 * j + v] = static_cast<float>(S(i, j) * A[u][v] + (i == j ? B[u][v] : 0));
-}
-
 }  // namespace
 
 cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, int K, int r, int8_t* q8,
@@ -637,14 +629,7 @@ cudaError_t launch_hadamard_quantize(const void* X, size_t rows, int K, int r, i
     if (e != cudaSuccess) return e;
     static bool ready[64] = {};
     if (dev < 64 && !ready[dev]) {
-        // Once per device: the two small factors into constant memory, the shared-memory limit of the kernels.
-        static float h12[12 * 12], h28[28 * 28];
-        paley2(5, h12);
-        paley2(13, h28);
-        if ((e = cudaMemcpyToSymbol(c_paley12, h12, sizeof(h12))) != cudaSuccess) return e;
-        if ((e = cudaMemcpyToSymbol(c_paley28, h28, sizeof(h28))) != cudaSuccess) return e;
-        if ((e = cudaMemcpyToSymbol(g_paley12, h12, sizeof(h12))) != cudaSuccess) return e;
-        if ((e = cudaMemcpyToSymbol(g_paley28, h28, sizeof(h28))) != cudaSuccess) return e;
+        // Once per device: the shared-memory limit of the kernels.
         for (auto k : {hadamard_quantize_kernel<1, kThreads>, hadamard_quantize_kernel<12, kThreads>,
                        hadamard_quantize_kernel<28, kThreads>, hadamard_quantize_kernel<1, kWideThreads>,
                        hadamard_quantize_kernel<12, kWideThreads>, hadamard_quantize_kernel<28, kWideThreads>})
