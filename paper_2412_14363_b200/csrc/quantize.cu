@@ -397,9 +397,9 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
     const int K4 = K - r;
     const uint8_t* srow = reinterpret_cast<const uint8_t*>(hrow);
     for (size_t row = blockIdx.x; row < rows; row += gridDim.x) {
-        // 1. widen the bf16 row
+        // 1. widen the bf16 row (M = 1; otherwise the small factor below reads its groups straight from global memory)
         const uint4* xp = reinterpret_cast<const uint4*>(X + row * static_cast<size_t>(K));
-        for (int c = tid; c < nchunks; c += NT) {
+        for (int c = tid; M == 1 && c < nchunks; c += NT) {
             const uint4 u = __ldg(xp + c);
             const uint32_t w[4] = {u.x, u.y, u.z, u.w};
             float4 a, b;
@@ -410,19 +410,22 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
             reinterpret_cast<float4*>(hrow)[2 * c] = a;
             reinterpret_cast<float4*>(hrow)[2 * c + 1] = b;
         }
-        __syncthreads();
-        // 2. the small factor, one group of M consecutive coefficients per thread, in place
+        if constexpr (M == 1) __syncthreads();
+        // 2. the small factor, one group of M consecutive coefficients per thread: bf16 from global memory (M * 2 bytes
+        //    per group, a multiple of 8), fp32 result to the row buffer
         if constexpr (M > 1) {
             constexpr Conference<M> conf{};
             constexpr int H2 = M / 2;
             for (int a = tid; a < (K / M); a += NT) {
                 // M * 4 bytes is a multiple of 16: the group moves as float4s (conflict-free at this stride)
                 float4* gp = reinterpret_cast<float4*>(hrow + a * M);
+                const uint2* xg = reinterpret_cast<const uint2*>(X + row * static_cast<size_t>(K) + static_cast<size_t>(a) * M);
                 float x[M], y[M], ps[H2], ms[H2];
 #pragma unroll
                 for (int i = 0; i < M / 4; ++i) {
-                    const float4 v = gp[i];
-                    x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
+                    const uint2 u = __ldg(xg + i);
+                    x[4 * i] = __uint_as_float(u.x << 16); x[4 * i + 1] = __uint_as_float(u.x & 0xFFFF0000u);
+                    x[4 * i + 2] = __uint_as_float(u.y << 16); x[4 * i + 3] = __uint_as_float(u.y & 0xFFFF0000u);
                 }
 #pragma unroll
                 for (int i = 0; i < H2; ++i) {
@@ -446,6 +449,7 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
             __syncthreads();
         }
         // 3. Sylvester butterflies over the index bits of a, three bits per pass
+        float a8 = 0.f, a4 = 0.f;
         for (int s = 0; s < kbits; s += 3) {
             const int nb = kbits - s < 3 ? kbits - s : 3;
             const int count = K >> nb;
@@ -470,15 +474,25 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
                         }
                     }
                 }
+                if (s + nb >= kbits) {  // last pass: 4. scale by 1 / sqrt(K) and take the two absmax values on the way out
+                    const int e0 = a0 * M + b;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (j < (1 << nb)) {
+                            v[j] *= inv_sqrt_k;
+                            if (e0 + j * stride < r) a8 = fmaxf(a8, fabsf(v[j]));
+                            else a4 = fmaxf(a4, fabsf(v[j]));
+                        }
+                    }
+                }
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (j < (1 << nb)) base[j * stride] = v[j];
             }
             __syncthreads();
         }
-        // 4. scale by 1 / sqrt(K) and take the two absmax values
-        float a8 = 0.f, a4 = 0.f;
-        for (int c = tid; c < nchunks; c += NT) {
+        // 4. (no butterfly pass: K = M) scale and absmax in a pass of their own
+        for (int c = tid; kbits == 0 && c < nchunks; c += NT) {
             float4* p = reinterpret_cast<float4*>(hrow) + 2 * c;
             float4 a = p[0], b = p[1];
             a.x *= inv_sqrt_k; a.y *= inv_sqrt_k; a.z *= inv_sqrt_k; a.w *= inv_sqrt_k;
