@@ -356,7 +356,7 @@ __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* _
 // quantizer: C = X * H_K / sqrt(K), H_K = Sylvester(2^k) (x) H_m with coefficient index a * m + b, m = 1, or
 // m = 12 / 28 with Paley's second construction (q = 5 / 13).  One CTA per row: the row is widened to fp32
 // in shared memory, multiplied group-wise by the small factor (constant memory), run through the
-// Sylvester butterflies three index bits per pass (eight values in registers, conflict-free strides),
+// Sylvester butterflies up to five index bits per pass (32 values in registers),
 // scaled, and then quantized exactly as in the fast path above (absmax per segment, reciprocal-product
 // rounding with the exact fallback).  r = 0 gives the paper's uniform INT4 down_proj input.
 // Paley's second construction for a prime q = 1 (mod 4): H = S (x) [[1,1],[1,-1]] + I (x) [[1,-1],[-1,-1]] of order
@@ -383,6 +383,46 @@ struct Conference {
 
 constexpr int kWideThreads = 1024;  // threads per row when there are at most kWideMaxRows rows (one CTA per SM)
 constexpr int kWideMaxRows = 148;
+// One pass of the Sylvester butterflies: index bits [s, s + NB) of a, 2^NB values per thread in registers.  The last
+// pass also scales by 1 / sqrt(K) and collects the two absmax values (elements below r belong to the INT8 segment).
+template <int M, int NT, int NB>
+__device__ __forceinline__ void butterfly_pass(float* hrow, int K, int s, int tid, bool last, float inv_sqrt_k, int r,
+                                               float& a8, float& a4) {
+    constexpr int N = 1 << NB;
+    const int count = K >> NB;
+    const int stride = M << s;
+    for (int i = tid; i < count; i += NT) {
+        const int arest = i / M, b = i - arest * M;
+        const int a0 = ((arest >> s) << (s + NB)) | (arest & ((1 << s) - 1));
+        float* base = hrow + a0 * M + b;
+        float v[N];
+#pragma unroll
+        for (int j = 0; j < N; ++j) v[j] = base[j * stride];
+#pragma unroll
+        for (int bit = 0; bit < NB; ++bit) {
+#pragma unroll
+            for (int j = 0; j < N; ++j) {
+                if (!(j & (1 << bit))) {
+                    const float lo = v[j], hi = v[j | (1 << bit)];
+                    v[j] = lo + hi;
+                    v[j | (1 << bit)] = lo - hi;
+                }
+            }
+        }
+        if (last) {
+            const int e0 = a0 * M + b;
+#pragma unroll
+            for (int j = 0; j < N; ++j) {
+                v[j] *= inv_sqrt_k;
+                if (e0 + j * stride < r) a8 = fmaxf(a8, fabsf(v[j]));
+                else a4 = fmaxf(a4, fabsf(v[j]));
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < N; ++j) base[j * stride] = v[j];
+    }
+}
+
 // NT threads per row: 256 when rows outnumber the SMs (throughput: several CTAs per SM), 1024 for the few rows of a
 // generation step, where one row's chain of passes is all there is to wait for.
 template <int M, int NT>
@@ -448,47 +488,20 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
             }
             __syncthreads();
         }
-        // 3. Sylvester butterflies over the index bits of a, three bits per pass
+        // 3. Sylvester butterflies over the index bits of a, up to five bits (32 values in registers) per pass
         float a8 = 0.f, a4 = 0.f;
-        for (int s = 0; s < kbits; s += 3) {
-            const int nb = kbits - s < 3 ? kbits - s : 3;
-            const int count = K >> nb;
-            const int stride = M << s;
-            for (int i = tid; i < count; i += NT) {
-                const int arest = i / M, b = i - arest * M;
-                const int a0 = ((arest >> s) << (s + nb)) | (arest & ((1 << s) - 1));
-                float* base = hrow + a0 * M + b;
-                float v[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = j < (1 << nb) ? base[j * stride] : 0.f;
-#pragma unroll
-                for (int bit = 0; bit < 3; ++bit) {
-                    if (bit < nb) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            if (!(j & (1 << bit))) {
-                                const float lo = v[j], hi = v[j | (1 << bit)];
-                                v[j] = lo + hi;
-                                v[j | (1 << bit)] = lo - hi;
-                            }
-                        }
-                    }
-                }
-                if (s + nb >= kbits) {  // last pass: 4. scale by 1 / sqrt(K) and take the two absmax values on the way out
-                    const int e0 = a0 * M + b;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (j < (1 << nb)) {
-                            v[j] *= inv_sqrt_k;
-                            if (e0 + j * stride < r) a8 = fmaxf(a8, fabsf(v[j]));
-                            else a4 = fmaxf(a4, fabsf(v[j]));
-                        }
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (j < (1 << nb)) base[j * stride] = v[j];
+        for (int s = 0; s < kbits;) {
+            const int left = kbits - s;
+            const int nb = left <= 5 ? left : (left <= 10 ? (left + 1) / 2 : 5);
+            const bool last = s + nb >= kbits;
+            switch (nb) {
+                case 1: butterfly_pass<M, NT, 1>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
+                case 2: butterfly_pass<M, NT, 2>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
+                case 3: butterfly_pass<M, NT, 3>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
+                case 4: butterfly_pass<M, NT, 4>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
+                default: butterfly_pass<M, NT, 5>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
             }
+            s += nb;
             __syncthreads();
         }
         // 4. (no butterfly pass: K = M) scale and absmax in a pass of their own
