@@ -362,7 +362,9 @@ __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* _
 // Paley's second construction for a prime q = 1 (mod 4): H = S (x) [[1,1],[1,-1]] + I (x) [[1,-1],[-1,-1]] of order
 // 2 (q + 1), with S = [[0, 1^T], [1, chi(i - j)]] and chi the quadratic character of GF(q).  S is evaluated at compile
 // time, so the product with H is additions and subtractions only: with p_i = x_2i + x_2i+1 and m_i = x_2i - x_2i+1,
-//   y_2j = m_j + sum_i S_ij p_i,   y_2j+1 = -p_j + sum_i S_ij m_i      (M / 2 * (M - 2) + 2 M operations, not M * M).
+//   y_2j = m_j + sum_i S_ij p_i,   y_2j+1 = -p_j + sum_i S_ij m_i,
+// and the circulant block of S needs only its quadratic-residue half (see the kernel): about 290 operations for
+// M = 28, not M * M = 784.
 constexpr int quad_char(int q, int a) {
     a = ((a % q) + q) % q;
     if (a == 0) return 0;
@@ -472,16 +474,28 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
                     ps[i] = x[2 * i] + x[2 * i + 1];
                     ms[i] = x[2 * i] - x[2 * i + 1];
                 }
+                // S = [[0, 1^T], [1, Q]] with Q_ij = chi(i - j) circulant of order q = M / 2 - 1.  With t = sum of the
+                // q inner entries and R_j = sum over the quadratic residues k of entry (j + k) mod q, the non-residues
+                // sum to t - entry_j - R_j, so (Q v)_j = 2 R_j - t + v_j: (q - 1) / 2 + 2 operations instead of q - 1.
+                constexpr int Q = H2 - 1;
+                float tp = ps[1], tm = ms[1];
 #pragma unroll
-                for (int j = 0; j < H2; ++j) {
-                    float e = ms[j], o = -ps[j];
+                for (int i = 2; i < H2; ++i) { tp += ps[i]; tm += ms[i]; }
+                y[0] = ms[0] + tp;
+                y[1] = tm - ps[0];
 #pragma unroll
-                    for (int i = 0; i < H2; ++i) {
-                        if (conf.s[i][j] > 0) { e += ps[i]; o += ms[i]; }
-                        else if (conf.s[i][j] < 0) { e -= ps[i]; o -= ms[i]; }
+                for (int jp = 0; jp < Q; ++jp) {
+                    float rp = 0.f, rm = 0.f;
+#pragma unroll
+                    for (int k = 1; k < Q; ++k) {
+                        if (conf.s[1 + k][1] > 0) {  // chi(k) = +1
+                            rp += ps[1 + (jp + k) % Q];
+                            rm += ms[1 + (jp + k) % Q];
+                        }
                     }
-                    y[2 * j] = e;
-                    y[2 * j + 1] = o;
+                    const float qp = fmaf(2.f, rp, ps[jp + 1] - tp), qm = fmaf(2.f, rm, ms[jp + 1] - tm);
+                    y[2 * (jp + 1)] = (ms[jp + 1] + ps[0]) + qp;
+                    y[2 * (jp + 1) + 1] = (ms[0] - ps[jp + 1]) + qm;
                 }
 #pragma unroll
                 for (int i = 0; i < M / 4; ++i) gp[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
