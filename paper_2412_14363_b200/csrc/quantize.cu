@@ -502,18 +502,21 @@ hadamard_quantize_kernel(const __nv_bfloat16* __restrict__ X, size_t rows, int K
             }
             __syncthreads();
         }
-        // 3. Sylvester butterflies over the index bits of a, up to five bits (32 values in registers) per pass
+        // 3. Sylvester butterflies over the index bits of a, up to five bits (32 values in registers) per pass.  With
+        //    M = 1 a thread's values of the first pass are 2^nb consecutive words, i.e. the lanes of a warp sit 2^nb
+        //    banks apart: three bits per pass there (an 8-way conflict on one pass instead of a 32-way one).
+        constexpr int kMaxBits = M == 1 ? 3 : 5;
         float a8 = 0.f, a4 = 0.f;
         for (int s = 0; s < kbits;) {
             const int left = kbits - s;
-            const int nb = left <= 5 ? left : (left <= 10 ? (left + 1) / 2 : 5);
+            const int nb = left <= kMaxBits ? left : (left <= 2 * kMaxBits ? (left + 1) / 2 : kMaxBits);
             const bool last = s + nb >= kbits;
-            switch (nb) {
-                case 1: butterfly_pass<M, NT, 1>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
-                case 2: butterfly_pass<M, NT, 2>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
-                case 3: butterfly_pass<M, NT, 3>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
-                case 4: butterfly_pass<M, NT, 4>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
-                default: butterfly_pass<M, NT, 5>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4); break;
+            if (nb == 1) butterfly_pass<M, NT, 1>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4);
+            else if (nb == 2) butterfly_pass<M, NT, 2>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4);
+            else if (nb == 3) butterfly_pass<M, NT, 3>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4);
+            else if constexpr (kMaxBits > 3) {
+                if (nb == 4) butterfly_pass<M, NT, 4>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4);
+                else butterfly_pass<M, NT, 5>(hrow, K, s, tid, last, inv_sqrt_k, r, a8, a4);
             }
             s += nb;
             __syncthreads();
