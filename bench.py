@@ -193,6 +193,15 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
         sets.append((L, desc, copies))
         weight_bytes += L.N * (L.r + (L.K - L.r) // 2) + 2 * 2 * L.N
     p_bytes = sum(2 * L.K * L.K for L in layers if L.online)
+    # The paper's own form of the layer that needs an online basis (Section 4.3): Hadamard U_D + uniform INT4 weights.
+    had_sets = {}
+    for L in layers:
+        if L.online:
+            d0 = resq.layer_desc(L.K, L.N, 0, resq.SCALE_FP16)
+            b0 = resq.resq_pack_weights(d0, L.W_proj, with_w4_i8=False)
+            had_sets[L.name] = (d0, [b0] + [resq.Weights(d0, b0.w8.clone() if b0.w8 is not None else None, b0.w4.clone(),
+                                                         b0.s_w8.clone(), b0.s_w4.clone())
+                                            for _ in range(DECODE_COPIES - 1)])
     out = {"workload": WORKLOAD.split("-prefill")[0] + "-decode", "weight_bytes_per_step": weight_bytes,
            "p_bytes_per_step": p_bytes, "weight_copies_cycled": DECODE_COPIES, "steps": steps}
     for T in DECODE_T:
@@ -260,6 +269,39 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
         l1 = ev()
         torch.cuda.synchronize()
         total_linear = l0.elapsed_time(l1) / steps
+        # The same block with the Hadamard form of the online layer(s).
+        hb = {}
+        for (L, desc, _), b in zip(sets, bufs):
+            if L.online:
+                d0 = had_sets[L.name][0]
+                hb[L.name] = dict(x4=torch.empty((T, L.K // 2), dtype=torch.uint8, device=dev),
+                                  s8=torch.empty(T, dtype=torch.float32, device=dev),
+                                  s4=torch.empty(T, dtype=torch.float32, device=dev),
+                                  ws=resq.alloc_workspace(d0, T, False, False, device=dev))
+
+        def hadamard_chain(i):
+            for (L, desc, copies), b in zip(sets, bufs):
+                if L.online:
+                    h = hb[L.name]
+                    resq.resq_hadamard_quantize(b["X"], 0, None, h["x4"], h["s8"], h["s4"], None)
+                    resq.resq_mixed_gemm(had_sets[L.name][1][i % DECODE_COPIES], None, h["x4"], h["s8"], h["s4"], b["Y"], h["ws"])
+                else:
+                    resq.resq_linear(copies[i % DECODE_COPIES], b["X"], None, b["Y"], b["ws"])
+
+        total_hadamard = None
+        try:
+            for i in range(3):
+                hadamard_chain(i)
+            torch.cuda.synchronize()
+            torch.cuda._sleep(HOST_LEAD_CYCLES)
+            h0 = ev()
+            for i in range(steps):
+                hadamard_chain(i)
+            h1 = ev()
+            torch.cuda.synchronize()
+            total_hadamard = h0.elapsed_time(h1) / steps
+        except resq.ResqError:   # a width the Hadamard kernel or the streaming kernel's staging does not take
+            torch.cuda.synchronize()
         # The same GEMV chain with asymmetric activation codes (unsigned codes, zero-points, weight row sums).
         ab = []
         for (L, desc, copies), b in zip(sets, bufs):
@@ -301,7 +343,9 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
                         "online_projection_p_stream_gbs": round(p_bytes / (proj * 1e-3) / 1e9, 1) if proj > 0 else None,
                         "block_split_calls_us": round(total * 1e3, 2),
                         "block_linears_us": round(total_linear * 1e3, 2),
-                        "tokens_per_s": round(T / (total_linear * 1e-3), 1)}
+                        "tokens_per_s": round(T / (total_linear * 1e-3), 1),
+                        "block_linears_hadamard_down_us": round(total_hadamard * 1e3, 2) if total_hadamard else None,
+                        "tokens_per_s_hadamard_down": round(T / (total_hadamard * 1e-3), 1) if total_hadamard else None}
     resq.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 0)
     st = resq.resq_device_status()
     if st != resq.OK:

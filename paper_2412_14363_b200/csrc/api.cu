@@ -233,7 +233,23 @@ static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, 
         const cudaError_t e = launch_mixed_gemm_stream(T, d->n_out, d->K, d->r, x8, x4, s_x8, s_x4, W->w8, W->w4,
                                                        W->s_w8, W->s_w4, fp16, Y, y_dtype, dbg8, dbg4, st);
         if (e != cudaErrorNotSupported) return cuda_status(e);
-        if (d->r == 0) return RESQ_ERR_SHAPE;  // the cluster split-K fallback needs an INT8 segment
+        if (d->r == 0) {
+            // The cluster split-K fallback needs an INT8 segment.  Rows too wide to stage 9-16 tokens of uniform INT4
+            // codes run as two launches of at most 8 tokens (the weights are streamed twice).
+            if (T <= 8) return RESQ_ERR_SHAPE;
+            const size_t ysz = y_dtype == RESQ_Y_BF16 ? 2 : 4;
+            for (int t0 = 0; t0 < T; t0 += 8) {
+                const int rows = T - t0 < 8 ? T - t0 : 8;
+                const cudaError_t e2 = launch_mixed_gemm_stream(
+                    rows, d->n_out, d->K, 0, x8, x4 + static_cast<size_t>(t0) * (K4 / 2), s_x8 + t0, s_x4 + t0, W->w8, W->w4,
+                    W->s_w8, W->s_w4, fp16, static_cast<char*>(Y) + static_cast<size_t>(t0) * d->n_out * ysz, y_dtype,
+                    dbg8 ? dbg8 + static_cast<size_t>(t0) * d->n_out : nullptr,
+                    dbg4 ? dbg4 + static_cast<size_t>(t0) * d->n_out : nullptr, st);
+                if (e2 == cudaErrorNotSupported) return RESQ_ERR_SHAPE;
+                if (e2 != cudaSuccess) return cuda_status(e2);
+            }
+            return RESQ_OK;
+        }
     }
     if (T <= kDecodeMaxT)
         return cuda_status(launch_mixed_gemm_decode(T, d->n_out, d->K, d->r, x8, x4, s_x8, s_x4, W->w8, W->w4,

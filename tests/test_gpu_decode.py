@@ -29,6 +29,8 @@ def resq():
     (16, 14336, 4096, 1792, True),  # down_proj: INT4 rows of 6272 bytes span four ring stages
     (16, 28672, 64, 3584, False),   # activations too large to stage whole: the cluster split-K kernel runs
     (5, 28672, 64, 3584, False),    # ... while 8 token rows of the same shape still fit
+    (16, 28672, 64, 0, False),      # uniform INT4 at that width: no INT8 segment for the split-K kernel, two launches of 8 tokens
+    (11, 28672, 72, 0, False),      # ... 8 + 3 tokens, ragged channel block
     (2, 4096, 8, 512, False),       # a single unit
 ])
 def test_decode_bit_exact(resq, T, K, N, r, fp16):
