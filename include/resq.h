@@ -28,7 +28,8 @@
  *  - Shape rules: r % 32 == 0, (K - r) % 32 == 0, 0 <= r < K (r = 0: uniform INT4), n_out % 8 == 0, T >= 1.
  *    Data pointers must be 16-byte aligned.
  *  - Every function returns a resq_status_t (0 = success).  Arguments are validated on the host
- *    before anything is launched; on a non-zero return nothing was enqueued.  Waits inside the
+ *    before the first launch: RESQ_ERR_NULL / _SHAPE / _ALIGN / _WORKSPACE / _ARCH mean that nothing was
+ *    enqueued.  RESQ_ERR_CUDA can also come from a later launch of a call that enqueues several kernels.  Waits inside the
  *    kernels are bounded; a wait that runs out sets a device status word (see resq_device_status)
  *    and the kernel drains and returns.
  *  - Inputs must be finite; NaN/Inf are not checked.
@@ -139,8 +140,7 @@ int resq_project_quantize(const void* X, const void* P, int T, int K, int r, int
  * names no construction; K = 8192, 14336 and 28672 are covered.  Other K, or K·4 bytes > 200 KB, give
  * RESQ_ERR_SHAPE.  Outputs as resq_project_quantize (x8 may be NULL when r = 0).  The weights to pair with it are
  * resq_pack_weights of (H_K^T W / sqrt(K))^T.  Every entry point accepts r = 0 (then w8 / x8 may be NULL).
- * The first call on each device uploads the two small factors to constant memory with a blocking copy: make it
- * outside any stream capture.
+ * The first call on each device sets kernel attributes: make it outside any stream capture.
  */
 int resq_hadamard_quantize(const void* X, int T, int K, int r, int8_t* x8, uint8_t* x4, float* s_x8, float* s_x4,
                            int8_t* x4_i8, void* stream);
@@ -222,15 +222,22 @@ int resq_linear_asym(const resq_layer_desc_t* desc, int T, const void* X, const 
 size_t resq_workspace_bytes_asym(const resq_layer_desc_t* desc, int T, int has_P, int has_w4_i8);
 
 /*
- * (No counterpart in the paper: a deployment aid.)  Same result as resq_project_quantize with
- * P != NULL, for callers that cannot allocate device memory at all -- a server whose start-up code
- * gave the whole GPU to its own pool, a plug-in living inside another program's memory plan, a
- * real-time loop that cannot afford cudaMalloc's device-wide synchronisation.  The fp32 staging panel
- * that the regular call takes from the caller's workspace is instead a fixed array of
- * RESQ_STATIC_SCRATCH_BYTES built into the library (each GPU that loads the library holds it until
- * the process exits).  The call allocates nothing, frees nothing and takes no workspace argument;
- * inputs and outputs are still the caller's buffers, with the meanings and layouts of
- * resq_project_quantize.
+ * (No counterpart in the paper: a deployment aid.)  resq_project_quantize with P != NULL for callers that
+ * cannot allocate device memory at all -- a server whose start-up code gave the whole GPU to its own pool, a
+ * plug-in living inside another program's memory plan, a real-time loop that cannot afford cudaMalloc's
+ * device-wide synchronisation.  The fp32 staging panel that the regular call takes from the caller's workspace
+ * is instead a fixed array of RESQ_STATIC_SCRATCH_BYTES built into the library (each GPU that loads the library
+ * holds it until the process exits).  The call allocates nothing, frees nothing and takes no workspace argument;
+ * inputs and outputs are still the caller's buffers, with the meanings and layouts of resq_project_quantize
+ * (r = 0 and a NULL x8 included).
+ *  - Result: the same kernels as the regular call, run without the projection GEMM's split scratch.  The
+ *    output is therefore identical, bit for bit, to resq_project_quantize given a workspace that holds only
+ *    the panel (T * K * 4 bytes, rounded up to 256).  Against the regular call with the full
+ *    resq_workspace_bytes() workspace it is identical wherever that call does not cut tiles along K; where
+ *    it does -- every call with T <= 64, and larger T whose last round of tiles is thin -- the fp32 sums are
+ *    formed in another order, and codes can differ by one step on a small fraction of elements (both stay
+ *    within the online path's tolerance against exact sums).  Without the split a T <= 64 call also keeps
+ *    only K/256 of the 74 SM pairs busy: at K = 14336 it is about a third slower than the regular call.
  *  - Limit: T * K * 4 bytes must not exceed RESQ_STATIC_SCRATCH_BYTES (K = 4096: T <= 512; K = 14336:
  *    T <= 146; K = 28672: T <= 73); beyond it the call returns RESQ_ERR_WORKSPACE and launches nothing.
  *    P must be non-NULL (without a projection no scratch is needed: use resq_project_quantize).
@@ -253,9 +260,12 @@ int resq_project_quantize_static(const void* X, const void* P, int T, int K, int
  *    the ramp of each short kernel behind the tail of the previous one.  The caller promises that the
  *    packed weights and their scales were complete before the preceding kernel was enqueued (true
  *    for weights packed at load time; false if resq_pack_weights is the preceding kernel).
- * Returns RESQ_ERR_SHAPE for an unknown option.
+ *  RESQ_OPT_WAIT_LIMIT_US (default 2 000 000): wall-clock limit, in microseconds, of a single wait inside a
+ *    kernel (for a copy to land, for a pipeline stage to be released).  Stored on the CURRENT device with a
+ *    blocking copy; kernels enqueued afterwards on that device use it.  value >= 1.
+ * Returns RESQ_ERR_SHAPE for an unknown option or value.
  */
-enum { RESQ_OPT_DECODE_EARLY_WEIGHTS = 1 };
+enum { RESQ_OPT_DECODE_EARLY_WEIGHTS = 1, RESQ_OPT_WAIT_LIMIT_US = 2 };
 int resq_set_option(int option, int value);
 
 /* Inverse of the INT4 packing, for inspection: packed [rows][cols/2] -> int8 [rows][cols]. */
@@ -265,6 +275,18 @@ int resq_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, size_t col
  * RESQ_OK, RESQ_ERR_TIMEOUT, RESQ_ERR_INDEX (a timeout wins if both happened), or RESQ_ERR_CUDA if the stream
  * reported an error. */
 int resq_device_status(void* stream);
+
+/* Self-test of the failure path (no counterpart in the paper).  Every wait inside the kernels of this library is
+ * bounded (Conventions above).  This call enqueues one small kernel whose only CTA waits for a barrier phase
+ * that nothing completes: the wait runs out after the limit of RESQ_OPT_WAIT_LIMIT_US, the kernel records the
+ * condition and returns by itself -- nothing traps, the context stays usable -- and the next resq_device_status
+ * returns RESQ_ERR_TIMEOUT (and RESQ_OK again after that).  Set a short limit first (say 1000 us) and restore it
+ * afterwards; with the default limit the kernel runs for two seconds. */
+int resq_selftest_wait_runs_out(void* stream);
+
+/* Number of kernels that the entry points of this library have enqueued in this process so far (host state; the
+ * attention call counts its two kernels).  For accounting: a benchmark reads it before and after a timed region. */
+unsigned long long resq_launch_count(void);
 
 /* The CUDA runtime's description of the error behind the latest RESQ_ERR_CUDA that any entry point of
  * this process returned ("no error" if there was none).  Host state, for diagnostics. */

@@ -15,9 +15,9 @@ from typing import Optional
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libresq.so")
 
-OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(8)
+OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT, ERR_INDEX = range(9)
 SCALE_FP32, SCALE_FP16 = 0, 1
-OPT_DECODE_EARLY_WEIGHTS = 1
+OPT_DECODE_EARLY_WEIGHTS, OPT_WAIT_LIMIT_US = 1, 2
 Y_BF16, Y_FP32 = 0, 1
 
 EXPORTS = [
@@ -26,7 +26,7 @@ EXPORTS = [
     "resq_unpack_int4", "resq_set_option",
     "resq_weight_row_sums", "resq_project_quantize_asym", "resq_mixed_gemm_asym", "resq_linear_asym",
     "resq_workspace_bytes_asym",
-    "resq_device_status", "resq_status_string", "resq_last_cuda_error",
+    "resq_device_status", "resq_launch_count", "resq_selftest_wait_runs_out", "resq_status_string", "resq_last_cuda_error",
 ]
 
 
@@ -82,6 +82,9 @@ lib.resq_workspace_bytes_asym.restype = _sz
 lib.resq_workspace_bytes_asym.argtypes = [_dp, _i, _i, _i]
 lib.resq_set_option.argtypes = [_i, _i]
 lib.resq_device_status.argtypes = [_vp]
+lib.resq_selftest_wait_runs_out.argtypes = [_vp]
+lib.resq_launch_count.restype = ctypes.c_ulonglong
+lib.resq_launch_count.argtypes = []
 lib.resq_status_string.restype = ctypes.c_char_p
 lib.resq_last_cuda_error.restype = ctypes.c_char_p
 lib.resq_last_cuda_error.argtypes = []
@@ -241,6 +244,16 @@ def resq_set_option(option: int, value: int):
 
 def resq_device_status() -> int:
     return int(lib.resq_device_status(_stream()))
+
+
+def resq_launch_count() -> int:
+    """Kernels enqueued by the library in this process so far."""
+    return int(lib.resq_launch_count())
+
+
+def resq_selftest_wait_runs_out():
+    """Enqueues the kernel whose bounded wait runs out (see resq.h); resq_device_status then reads ERR_TIMEOUT."""
+    _check(lib.resq_selftest_wait_runs_out(_stream()), "resq_selftest_wait_runs_out")
 
 
 def alloc_workspace(desc: LayerDesc, T: int, has_P: bool, has_w4_i8: bool, device="cuda"):

@@ -1,13 +1,36 @@
 // C ABI of the library: argument validation, workspace carving and dispatch.  No arithmetic here.
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cuda_runtime.h>
 
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace resq {
 
-__device__ int g_status_word = 0;
+struct __align__(16) DeviceState {
+    int flags;                          // condition bits (kStatusBit*), cleared by resq_device_status
+    int reserved;
+    unsigned long long wait_limit_ns;   // limit of one bounded wait
+};
+__device__ DeviceState g_state = {0, 0, 2000000000ull};
+
+// A CTA that waits for a barrier phase nothing will ever complete: the bounded wait runs out, the kernel records
+// the condition and returns by itself.  Exercises the path every other kernel takes when a copy never lands.
+__global__ void wait_runs_out_kernel(int* status) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_mbar_init();
+        abort_flag = 0;
+    }
+    __syncthreads();
+    const bool done = mbar_wait(&bar, 0, &abort_flag, status);  // every thread polls; the first to time out tells the rest
+    __syncthreads();
+    if (threadIdx.x == 0 && (!done || abort_flag)) atomicOr(status, kStatusBitTimeout);
+}
 
 int* device_status_ptr() {
     static int* cache[64] = {};
@@ -15,11 +38,14 @@ int* device_status_ptr() {
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     if (!cache[dev]) {
         void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        if (cudaGetSymbolAddress(&p, g_state) != cudaSuccess) return nullptr;
         cache[dev] = static_cast<int*>(p);
     }
     return cache[dev];
 }
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(static_cast<unsigned long long>(n), std::memory_order_relaxed); }
 
 void* tensor_map_encode_fn() {
     static void* fn = nullptr;
@@ -60,7 +86,7 @@ int check_arch() {
 
 // Carving of the caller's workspace.  Every entry point uses the same map (and its own subset).
 struct Workspace {
-    size_t x8, x4, sx8, sx4, zx8, zx4, x4e, w4e, panel, decode, total;  // panel: fp32 coefficients + the GEMM's split scratch
+    size_t x8, x4, sx8, sx4, zx8, zx4, x4e, w4e, panel, total;  // panel: fp32 coefficients + the GEMM's split scratch
 };
 Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     Workspace w{};
@@ -76,7 +102,6 @@ Workspace carve(int K, int n_out, int r, int T, bool has_P, bool has_w4_i8) {
     w.x4e = o;    o += tiles ? align_up(Tz * K4) : 0;
     w.w4e = o;    o += (tiles && !has_w4_i8) ? align_up(N * K4) : 0;
     w.panel = o;  o += has_P ? align_up(static_cast<size_t>(T < kPanelRows ? T : kPanelRows) * K * 4) + align_up(project_split_scratch_bytes()) : 0;
-    w.decode = o; o += tiles ? 0 : align_up(decode_scratch_bytes(T, n_out));
     w.total = o;
     return w;
 }
@@ -233,28 +258,23 @@ static int mixed_gemm_impl(const resq_layer_desc_t* d, int T, const int8_t* x8, 
         const cudaError_t e = launch_mixed_gemm_stream(T, d->n_out, d->K, d->r, x8, x4, s_x8, s_x4, W->w8, W->w4,
                                                        W->s_w8, W->s_w4, fp16, Y, y_dtype, dbg8, dbg4, st);
         if (e != cudaErrorNotSupported) return cuda_status(e);
-        if (d->r == 0) {
-            // The cluster split-K fallback needs an INT8 segment.  Rows too wide to stage 9-16 tokens of uniform INT4
-            // codes run as two launches of at most 8 tokens (the weights are streamed twice).
-            if (T <= 8) return RESQ_ERR_SHAPE;
-            const size_t ysz = y_dtype == RESQ_Y_BF16 ? 2 : 4;
-            for (int t0 = 0; t0 < T; t0 += 8) {
-                const int rows = T - t0 < 8 ? T - t0 : 8;
-                const cudaError_t e2 = launch_mixed_gemm_stream(
-                    rows, d->n_out, d->K, 0, x8, x4 + static_cast<size_t>(t0) * (K4 / 2), s_x8 + t0, s_x4 + t0, W->w8, W->w4,
-                    W->s_w8, W->s_w4, fp16, static_cast<char*>(Y) + static_cast<size_t>(t0) * d->n_out * ysz, y_dtype,
-                    dbg8 ? dbg8 + static_cast<size_t>(t0) * d->n_out : nullptr,
-                    dbg4 ? dbg4 + static_cast<size_t>(t0) * d->n_out : nullptr, st);
-                if (e2 == cudaErrorNotSupported) return RESQ_ERR_SHAPE;
-                if (e2 != cudaSuccess) return cuda_status(e2);
-            }
-            return RESQ_OK;
+        // Rows too wide to stage 9-16 tokens of activation codes beside the weight rings run as two launches of at
+        // most 8 tokens (the weights are streamed twice; only reduction lengths beyond ~24k reach this).
+        if (T <= 8) return RESQ_ERR_SHAPE;
+        const size_t ysz = y_dtype == RESQ_Y_BF16 ? 2 : 4;
+        for (int t0 = 0; t0 < T; t0 += 8) {
+            const int rows = T - t0 < 8 ? T - t0 : 8;
+            const cudaError_t e2 = launch_mixed_gemm_stream(
+                rows, d->n_out, d->K, d->r, x8 ? x8 + static_cast<size_t>(t0) * d->r : nullptr,
+                x4 + static_cast<size_t>(t0) * (K4 / 2), s_x8 + t0, s_x4 + t0, W->w8, W->w4, W->s_w8, W->s_w4, fp16,
+                static_cast<char*>(Y) + static_cast<size_t>(t0) * d->n_out * ysz, y_dtype,
+                dbg8 ? dbg8 + static_cast<size_t>(t0) * d->n_out : nullptr,
+                dbg4 ? dbg4 + static_cast<size_t>(t0) * d->n_out : nullptr, st);
+            if (e2 == cudaErrorNotSupported) return RESQ_ERR_SHAPE;
+            if (e2 != cudaSuccess) return cuda_status(e2);
         }
+        return RESQ_OK;
     }
-    if (T <= kDecodeMaxT)
-        return cuda_status(launch_mixed_gemm_decode(T, d->n_out, d->K, d->r, x8, x4, s_x8, s_x4, W->w8, W->w4,
-                                                    W->s_w8, W->s_w4, fp16, Y, y_dtype, dbg8, dbg4,
-                                                    ws + map.decode, st));
     const int8_t* x4e = x4e_ready;
     if (!x4e) {
         int8_t* buf = reinterpret_cast<int8_t*>(ws + map.x4e);
@@ -477,6 +497,13 @@ int resq_set_option(int option, int value) {
         set_decode_early_weights(value);
         return RESQ_OK;
     }
+    if (option == RESQ_OPT_WAIT_LIMIT_US) {
+        if (value < 1) return RESQ_ERR_SHAPE;
+        int* p = device_status_ptr();
+        if (!p) return RESQ_ERR_CUDA;
+        const unsigned long long ns = static_cast<unsigned long long>(value) * 1000ull;
+        return cuda_status(cudaMemcpy(p + 2, &ns, sizeof(ns), cudaMemcpyHostToDevice));
+    }
     return RESQ_ERR_SHAPE;
 }
 
@@ -489,9 +516,18 @@ int resq_device_status(void* stream) {
     if (v != 0) {
         int zero = 0;
         cudaMemcpy(p, &zero, sizeof(int), cudaMemcpyHostToDevice);
-        return (v & RESQ_ERR_TIMEOUT) ? RESQ_ERR_TIMEOUT : RESQ_ERR_INDEX;  // kernels OR 7 or 8 into the word
+        return (v & kStatusBitTimeout) ? RESQ_ERR_TIMEOUT : RESQ_ERR_INDEX;  // one bit per condition
     }
     return RESQ_OK;
+}
+
+int resq_selftest_wait_runs_out(void* stream) {
+    if (int e = check_arch()) return e;
+    int* p = device_status_ptr();
+    if (!p) return RESQ_ERR_CUDA;
+    count_launch();
+    wait_runs_out_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return cuda_status(cudaGetLastError());
 }
 
 // ---- attention-block path (resq_kv.h) ----
@@ -568,6 +604,8 @@ int resq_attention_decode(const resq_kv_cache_t* cache, const void* q16, int n_q
     return cuda_status(launch_attention_decode(*cache, q16, n_q_heads, seq_lens, out, workspace,
                                                static_cast<cudaStream_t>(stream)));
 }
+
+unsigned long long resq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* resq_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 

@@ -340,7 +340,7 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             for (int i = 0; i < 4; ++i) acc8[h][i] = accO[h][i] = accE[h][i] = 0;
 
         for (; c < nchunks && idx < ce; ++c, ++idx) {
-            if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(&full[stage], phase, abort_flag, p.status)) { ok = false; break; }
             const uint8_t* w0 = ring + static_cast<size_t>(stage) * kStageBytes + wofs;
             const uint8_t* w1 = w0 + 8 * kChunkBytes;
             if (c < p.c8) {
@@ -505,7 +505,7 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         }
     }
     __syncthreads();
-    if (threadIdx.x == 0 && ctl->abort_flag) atomicOr(p.status, RESQ_ERR_TIMEOUT);
+    if (threadIdx.x == 0 && ctl->abort_flag) atomicOr(p.status, kStatusBitTimeout);
 }
 
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
@@ -551,6 +551,7 @@ cudaError_t launch_variant(const CUtensorMap& t8, const CUtensorMap& t4, const P
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = p.early_weights ? 1 : 0;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kern, t8, t4, p);
 }
 

@@ -9,8 +9,14 @@
 
 namespace resq {
 
-// Device status word (one per device that loaded the library); kernels OR an error code into it.
-int* device_status_ptr();  // device address of the status word of the current device, or nullptr
+// Device status block (one per device that loaded the library): int word 0 collects the condition bits that
+// kernels OR in (kStatusBitTimeout, kStatusBitIndex below), the 64-bit word at byte offset 8 holds the limit
+// of one bounded wait in nanoseconds.
+int* device_status_ptr();  // device address of the block of the current device, or nullptr
+// Counts kernels enqueued by this process (resq_launch_count); called once per launch by the wrappers below.
+void count_launch(int n = 1);
+constexpr int kStatusBitTimeout = 1;  // a bounded wait ran out
+constexpr int kStatusBitIndex = 2;    // an index read on the device was out of range
 
 // ---- kernels (launch wrappers; return cudaGetLastError()) ----------------------------------
 // Split quantization of the rows of a [rows][K] matrix (Eq. 2 for activations, Eq. 3 for weights).
@@ -50,16 +56,9 @@ cudaError_t launch_split_quantize_asym(const void* in, bool in_is_f32, size_t ro
 cudaError_t launch_weight_row_sums(const int8_t* w8, const uint8_t* w4, int N, int K, int r, int32_t* wsum8,
                                    int32_t* wsum4, cudaStream_t st);
 
-// Few-token (T <= 16) weight-streaming split-K kernel.  scratch: see decode_scratch_bytes().
-size_t decode_scratch_bytes(int T, int N);
-cudaError_t launch_mixed_gemm_decode(int T, int N, int K, int r, const int8_t* x8, const uint8_t* x4,
-                                     const float* s_x8, const float* s_x4, const int8_t* w8, const uint8_t* w4,
-                                     const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
-                                     int32_t* dbg8, int32_t* dbg4, void* scratch, cudaStream_t st);
-
-// Few-token streaming kernel (persistent grid, bulk-copy ring).  Returns cudaErrorNotSupported, with
-// nothing launched, when the staged activations leave no room for the ring; the caller then uses
-// launch_mixed_gemm_decode.
+// Few-token (T <= 16) streaming kernel (persistent grid, bulk-copy ring).  Returns cudaErrorNotSupported, with
+// nothing launched, when the staged activations leave no room for the ring; the caller then splits the tokens
+// over two launches.
 cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x8, const uint8_t* x4,
                                      const float* s_x8, const float* s_x4, const int8_t* w8, const uint8_t* w4,
                                      const void* s_w8, const void* s_w4, bool w_scale_fp16, void* Y, int y_dtype,
@@ -73,9 +72,6 @@ void set_decode_early_weights(int on);
 size_t project_split_scratch_bytes();
 cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, float* C, cudaStream_t st,
                                 void* scratch = nullptr, size_t scratch_bytes = 0);
-
-// Output-tile width of the two tile GEMMs (see the definition for what was measured).
-int pick_tile_width(int m_tiles, int N, int sms);
 
 // ---- attention-block path (declared in resq_kv.h) ----
 cudaError_t launch_uc_quantize(const float* W_C, int8_t* wq, float* s_u, cudaStream_t st);

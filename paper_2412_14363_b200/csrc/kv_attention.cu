@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
 #pragma unroll
             for (int mt = 0; mt < 8; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
         }
-        if (!mbar_wait(&full[stage], phase, &abort_flag)) { ok = false; break; }
+        if (!mbar_wait(&full[stage], phase, &abort_flag, p.status)) { ok = false; break; }
         const uint8_t* st = ring + stage * kBlk;
         const int valid = min(RESQ_KV_BLOCK, cons.len - RESQ_KV_BLOCK * cons.blk);
         if (valid < RESQ_KV_BLOCK) {  // last block of a sequence: the unused slots hold anything -- zero their value scales
@@ -456,7 +456,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
             const uint32_t phase = static_cast<uint32_t>(k / kStages) & 1u;
             for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&full[stage], phase); ++spin) {}
         }
-        if (lane == 0) atomicOr(p.status, RESQ_ERR_TIMEOUT);
+        if (lane == 0) atomicOr(p.status, kStatusBitTimeout);
     }
 }
 
@@ -483,7 +483,7 @@ __global__ void __launch_bounds__(kD * kMaxGroups) attention_combine_kernel(cons
     long long before = 0, total = 0;
     for (int i = tid; i < p.n_seqs; i += nthr) {
         const int len = p.seq_lens[i];
-        if (blockIdx.x == 0 && (len < 0 || len > p.capacity)) atomicOr(p.status, RESQ_ERR_INDEX);
+        if (blockIdx.x == 0 && (len < 0 || len > p.capacity)) atomicOr(p.status, kStatusBitIndex);
         const int t = ((len < 0 ? 0 : (len > p.capacity ? p.capacity : len)) + 31) >> 5;
         total += t;
         if (i < b) before += t;
@@ -500,6 +500,10 @@ __global__ void __launch_bounds__(kD * kMaxGroups) attention_combine_kernel(cons
     total *= p.n_kv_heads;
     float* out = p.out + (static_cast<long long>(b) * n_q_heads + hq) * kD;
     const int nblk = (clamped_len(p.seq_lens, b, p.capacity) + 31) >> 5;
+    // Every CTA waits for the attention grid before it returns, also those with nothing to merge: this grid was
+    // launched as a programmatic dependent, so the next kernel of the stream is ordered against THIS grid only,
+    // and it must not retire while the attention grid is still writing `out`.
+    griddep_wait();
     if (nblk == 0) {  // empty sequence
         if (grp == 0) out[d] = 0.f;
         return;
@@ -509,7 +513,6 @@ __global__ void __launch_bounds__(kD * kMaxGroups) attention_combine_kernel(cons
     const int w_first = static_cast<int>(((lo + 1) * nw - 1) / total), w_last = static_cast<int>((hi * nw - 1) / total);
     if (w_first == w_last) return;  // one warp saw the whole (sequence, head) and wrote the output itself
     const long long s = static_cast<long long>(b) * p.n_kv_heads + hk;
-    griddep_wait();
     float M = -INFINITY, num = 0.f, den = 0.f;  // num: this group's share; den: a per-thread partial until the end
     for (int w0 = w_first; w0 <= w_last; w0 += nthr) {
         const int w = w0 + tid;
@@ -592,6 +595,7 @@ cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q1
     p.n_kv_heads = cache.n_kv_heads;
     p.group = n_q_heads / cache.n_kv_heads;
     p.capacity = cache.capacity;
+    count_launch(2);
     attention_decode_kernel<<<148, kWarps * 32, kSmem, st>>>(p);
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};

@@ -87,7 +87,7 @@ __device__ __forceinline__ long long cache_slot(long long row, int n_kv_heads, i
     const int h = static_cast<int>(row - t * n_kv_heads);
     const int b = seq_ids[t], pos = positions[t];
     if (b < 0 || b >= n_seqs || pos < 0 || pos >= capacity) {
-        atomicOr(status, RESQ_ERR_INDEX);
+        atomicOr(status, kStatusBitIndex);
         return -1;
     }
     const long long blk = (static_cast<long long>(b) * n_kv_heads + h) * (capacity / RESQ_KV_BLOCK) + pos / RESQ_KV_BLOCK;
@@ -321,6 +321,7 @@ int grid_for(long long tiles) {
 cudaError_t launch_project(const ProjectParams& p, cudaStream_t st) {
     const long long tiles = (p.q_rows + 15) / 16 + 2 * ((p.kv_rows + 15) / 16);
     if (tiles == 0) return cudaSuccess;
+    count_launch();
     kv_project_kernel<<<grid_for(tiles), kWarps * 32, 0, st>>>(p);
     return cudaGetLastError();
 }
@@ -328,6 +329,7 @@ cudaError_t launch_project(const ProjectParams& p, cudaStream_t st) {
 }  // namespace
 
 cudaError_t launch_uc_quantize(const float* W_C, int8_t* wq, float* s_u, cudaStream_t st) {
+    count_launch();
     uc_quantize_kernel<<<kD, 32, 0, st>>>(W_C, wq, s_u);
     return cudaGetLastError();
 }

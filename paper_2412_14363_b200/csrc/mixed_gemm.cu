@@ -140,7 +140,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
                 const int m0 = (tile % p.m_tiles) * 2 * BM + rank * BM;        // this CTA's token rows
                 const int n0 = (tile / p.m_tiles) * p.bn + rank * BN_HALF;     // this CTA's weight rows
                 for (int kb = 0; kb < kb_total; ++kb) {
-                    if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag, p.status)) { ok = false; break; }
                     // The even CTA arms its barrier for the bytes of both CTAs; the peer only sends its
                     // bytes there (if they land first, the pending arrival keeps the phase open).
                     const uint32_t full_addr = cluster_map(&sh->full[stage], 0);
@@ -170,16 +170,16 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
                 // INT4 columns are free once the previous tile's epilogue has copied them out.
-                if (!mbar_wait(&sh->acc4_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&sh->acc4_empty, acc_phase ^ 1, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
                 for (int kb = 0; kb < kb_total; ++kb) {
                     const bool seg4 = kb < p.kb4;
                     if (kb == p.kb4) {
                         // ... the INT8 columns once it has finished with the tile.
-                        if (!mbar_wait(&sh->acc8_empty, acc_phase ^ 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(&sh->acc8_empty, acc_phase ^ 1, abort_flag, p.status)) { ok = false; break; }
                         tc_fence_after();
                     }
-                    if (!mbar_wait(&sh->full[stage], phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&sh->full[stage], phase, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t a_desc = make_smem_desc_k128(smem_u32(sA + stage * A_BYTES));
                     const uint64_t b_desc = make_smem_desc_k128(smem_u32(sB + stage * B_BYTES));
@@ -228,7 +228,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
             const float sx4 = row_ok ? __ldg(p.s_x4 + row) : 0.f;
             const float zx8 = ASYM && row_ok ? __ldg(p.z_x8 + row) : 0.f;
             const float zx4 = ASYM && row_ok ? __ldg(p.z_x4 + row) : 0.f;
-            if (!mbar_wait(&sh->acc_full, acc_phase, abort_flag)) continue;  // flag is set; leave at the next sample
+            if (!mbar_wait(&sh->acc_full, acc_phase, abort_flag, p.status)) continue;  // flag is set; leave at the next sample
             acc_phase ^= 1;
             tc_fence_after();
             const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + ch * (BN / 2);
@@ -304,7 +304,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap tmA8, const __grid_constan
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();  // neither CTA leaves while the other may still read its shared memory or signal it
-    if (threadIdx.x == 0 && sh->abort_flag) atomicOr(p.status, RESQ_ERR_TIMEOUT);
+    if (threadIdx.x == 0 && sh->abort_flag) atomicOr(p.status, kStatusBitTimeout);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc_pair(tmem_base, kTmemCols);
@@ -329,12 +329,6 @@ bool make_map_u8(CUtensorMap* m, const void* base, uint64_t rows, uint64_t kbyte
 }
 
 }  // namespace
-
-// Tile width for a persistent grid.  The kernels take any multiple of 16 up to 256 (the B loads and
-// the TMEM offsets stay 256 wide), which would let the width be tuned so that the last round of tiles
-// is fuller; measured on B200, though, tiles of 240 and 192 columns ran 1.5-1.7 x slower per column
-// than 256-wide ones in both GEMMs, which costs far more than the partly filled round they save.
-int pick_tile_width(int /*m_tiles*/, int /*N*/, int /*sms*/) { return 256; }
 
 cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8, const int8_t* x4e,
                                     const float* s_x8, const float* s_x4, const int8_t* w8, const int8_t* w4e,
@@ -369,7 +363,9 @@ cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     p.m_tiles = (T + 2 * BM - 1) / (2 * BM);
-    p.bn = pick_tile_width(p.m_tiles, N, sms);
+    // The kernel takes any multiple of 16 up to BN here (B loads and TMEM offsets stay BN wide); tiles of 240 and
+    // 192 columns measured 1.5-1.7 x slower per column than 256-wide ones, far more than a fuller last round saves.
+    p.bn = BN;
     p.n_tiles = (N + p.bn - 1) / p.bn;
     p.kb8 = (r + BK - 1) / BK;
     p.kb4 = (K4 + BK - 1) / BK;
@@ -380,6 +376,7 @@ cudaError_t launch_mixed_gemm_tiles(int T, int N, int K, int r, const int8_t* x8
     p.status = device_status_ptr();
     const int tiles = p.m_tiles * p.n_tiles;
     const int pairs = tiles < sms / 2 ? tiles : sms / 2;
+    count_launch();
     if (asym) mixed_gemm_kernel<true><<<2 * pairs, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
     else mixed_gemm_kernel<false><<<2 * pairs, kThreads, kSmemBytes, st>>>(tA8, tA4, tB8, tB4, p);
     return cudaGetLastError();

@@ -205,7 +205,7 @@ project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
                 const Item it = item_info(p, item);
                 const int my_m = it.m0 + rank * BM, my_n = it.n0 + rank * BN_HALF;
                 for (int kb = it.kb0; kb < it.kb0 + it.nkb; ++kb) {
-                    if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag, p.status)) { ok = false; break; }
                     // The even CTA arms its barrier for the bytes of both CTAs; the peer only sends its bytes
                     // there (they may land before the barrier is armed: the pending arrival keeps the phase open).
                     const uint32_t full_addr = cluster_map(&sh->full[stage], 0);
@@ -234,11 +234,11 @@ project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
             bool ok = true;
             for (int item = pair; item < num_items && ok; item += npairs) {
                 const int nkb = item_info(p, item).nkb;
-                if (!mbar_wait(&sh->acc_empty[buf], acc_phase[buf] ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&sh->acc_empty[buf], acc_phase[buf] ^ 1, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + static_cast<uint32_t>(buf * BN);
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!mbar_wait(&sh->full[stage], phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&sh->full[stage], phase, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t a_desc = make_smem_desc_k128(smem_u32(sA + stage * A_BYTES));
                     const uint64_t b_desc = make_smem_desc_mn128(smem_u32(sB + stage * B_BYTES), B_BOX_BYTES);
@@ -266,7 +266,7 @@ project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
             if (et == 0) sh->epi_stop = *abort_flag;
             epi_barrier();
             if (sh->epi_stop) break;
-            if (!mbar_wait(&sh->acc_full[buf], acc_phase[buf], abort_flag)) continue;
+            if (!mbar_wait(&sh->acc_full[buf], acc_phase[buf], abort_flag, p.status)) continue;
             acc_phase[buf] ^= 1;
             tc_fence_after();
             const int lrow = rank * BM + quad * 32 + lane;  // row inside the pair's tile
@@ -295,7 +295,7 @@ project_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();  // neither CTA leaves while the other may still read its shared memory or signal it
-    if (threadIdx.x == 0 && sh->abort_flag) atomicOr(p.status, RESQ_ERR_TIMEOUT);
+    if (threadIdx.x == 0 && sh->abort_flag) atomicOr(p.status, kStatusBitTimeout);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc_pair(tmem_base, kTmemCols);
@@ -379,7 +379,7 @@ project_gemm_few_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
                 const Item it = item_info(p, item);
                 const int my_j = it.n0 + rank * BN_HALF;
                 for (int kb = it.kb0; kb < it.kb0 + it.nkb; ++kb) {
-                    if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag, p.status)) { ok = false; break; }
                     const uint32_t full_addr = cluster_map(&sh->full[stage], 0);
                     if (rank == 0) mbar_arrive_expect_tx(&sh->full[stage], 2 * (B_BYTES + x_bytes));
 #pragma unroll
@@ -405,11 +405,11 @@ project_gemm_few_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
             bool ok = true;
             for (int item = pair; item < num_items && ok; item += npairs) {
                 const int nkb = item_info(p, item).nkb;
-                if (!mbar_wait(&sh->acc_empty[buf], acc_phase[buf] ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&sh->acc_empty[buf], acc_phase[buf] ^ 1, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + static_cast<uint32_t>(buf * kFewMaxT);
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!mbar_wait(&sh->full[stage], phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&sh->full[stage], phase, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t a_desc = make_smem_desc_mn128(smem_u32(sP + stage * B_BYTES), B_BOX_BYTES);
                     const uint64_t b_desc = make_smem_desc_k128(smem_u32(sX + stage * FX_BYTES));
@@ -437,7 +437,7 @@ project_gemm_few_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
             if (et == 0) sh->epi_stop = *abort_flag;
             epi_barrier();
             if (sh->epi_stop) break;
-            if (!mbar_wait(&sh->acc_full[buf], acc_phase[buf], abort_flag)) continue;
+            if (!mbar_wait(&sh->acc_full[buf], acc_phase[buf], abort_flag, p.status)) continue;
             acc_phase[buf] ^= 1;
             tc_fence_after();
             const int jj = rank * BM + quad * 32 + lane;  // column inside the tile
@@ -464,7 +464,7 @@ project_gemm_few_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();
-    if (threadIdx.x == 0 && sh->abort_flag) atomicOr(p.status, RESQ_ERR_TIMEOUT);
+    if (threadIdx.x == 0 && sh->abort_flag) atomicOr(p.status, kStatusBitTimeout);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc_pair(tmem_base, kFewTmemCols);
@@ -502,6 +502,7 @@ cudaError_t launch_reduce(const Params& p, cudaStream_t st) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, project_reduce_kernel, p);
 }
 
@@ -554,6 +555,7 @@ cudaError_t launch_project_few(const void* X, const void* P, int T, int K, float
     }
     const int items = p.full_items + p.split_tiles * p.splits;
     const int pairs = items < all_pairs ? items : all_pairs;
+    count_launch();
     project_gemm_few_kernel<<<2 * pairs, kThreads, kFewSmemBytes, st>>>(tX, tP, p, ntok);
     if (cudaError_t le = cudaGetLastError(); le != cudaSuccess) return le;
     if (p.split_tiles > 0) {
@@ -618,6 +620,7 @@ cudaError_t launch_project_gemm(const void* X, const void* P, int T, int K, floa
             p.prows = 2 * BM;
         }
     }
+    count_launch();
     project_gemm_pair_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(tX, tP, p);
     if (cudaError_t le = cudaGetLastError(); le != cudaSuccess) return le;
     if (p.split_tiles > 0) return launch_reduce(p, st);

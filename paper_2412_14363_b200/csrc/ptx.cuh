@@ -55,19 +55,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Wall-clock limit of one wait.  A whole kernel of this library runs for milliseconds.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
-
+// `status` below is the device status block (internal.h): word 0 collects condition bits that kernels OR in; the
+// 64-bit word at byte offset 8 is the wall-clock limit of one wait in nanoseconds (default 2 s: a whole kernel of
+// this library runs for milliseconds).
 // Waits for the phase with the given parity to complete.  Returns false if the limit ran out or if
-// `abort_flag` (a shared-memory word any role may set) became non-zero.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// `abort_flag` (a shared-memory word any role may set) became non-zero.  `status` is the device status block;
+// the limit is read from it only when the first poll has failed.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, const int* status) {
     if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t limit = *reinterpret_cast<const volatile unsigned long long*>(status + 2);
     const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0xFF) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > limit) {
                 *abort_flag = 1;
                 return false;
             }

@@ -243,10 +243,10 @@ split_quantize_fast_kernel(const void* __restrict__ in, size_t in_row_bytes, siz
                       reinterpret_cast<const char*>(in) + (row0 + i) * in_row_bytes, row_bytes, &bar);
     }
     __syncthreads();
-    const bool landed = mbar_wait(&bar, 0, &abort_flag);
+    const bool landed = mbar_wait(&bar, 0, &abort_flag, status);
     if (__syncthreads_or(!landed)) {
         // The copy did not land in time: report it and leave the outputs of this group unwritten.
-        if (threadIdx.x == 0) atomicOr(status, RESQ_ERR_TIMEOUT);
+        if (threadIdx.x == 0) atomicOr(status, kStatusBitTimeout);
         return;
     }
 
@@ -355,7 +355,7 @@ __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* _
 // that cannot be folded costs a fast transform instead of a dense product), fused with the per-token
 // quantizer: C = X * H_K / sqrt(K), H_K = Sylvester(2^k) (x) H_m with coefficient index a * m + b, m = 1, or
 // m = 12 / 28 with Paley's second construction (q = 5 / 13).  One CTA per row: the row is widened to fp32
-// in shared memory, multiplied group-wise by the small factor (constant memory), run through the
+// in shared memory, multiplied group-wise by the small factor (a compile-time table), run through the
 // Sylvester butterflies up to five index bits per pass (32 values in registers),
 // scaled, and then quantized exactly as in the fast path above (absmax per segment, reciprocal-product
 // rounding with the exact fallback).  r = 0 gives the paper's uniform INT4 down_proj input.
@@ -620,11 +620,13 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
             attr[0].val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = attr;
             cfg.numAttrs = programmatic ? 1 : 0;
+            count_launch();
             return cudaLaunchKernelEx(&cfg, kern, in, in_row_stride_bytes, rows, K, r, rpc, q8, q4,
                                       static_cast<float*>(s8), static_cast<float*>(s4), q4_i8, device_status_ptr());
         }
     }
     const unsigned grid = static_cast<unsigned>(rows < 148u * 64u ? rows : 148u * 64u);
+    count_launch();
     if (in_is_f32)
         split_quantize_kernel<true><<<grid, kThreads, 0, st>>>(in, in_row_stride_bytes, rows, K, r, q8, q4, s8, s4,
                                                                scale_fp16 ? 1 : 0, q4_i8);
@@ -640,6 +642,7 @@ cudaError_t launch_unpack_int4(const uint8_t* packed, int8_t* out, size_t rows, 
     if (nwords == 0) return cudaSuccess;
     size_t blocks = (nwords + 255) / 256;
     if (blocks > 148 * 32) blocks = 148 * 32;
+    count_launch();
     if (codes_unsigned) unpack_int4_kernel<true><<<static_cast<unsigned>(blocks), 256, 0, st>>>(packed, out, nwords);
     else unpack_int4_kernel<false><<<static_cast<unsigned>(blocks), 256, 0, st>>>(packed, out, nwords);
     return cudaGetLastError();
@@ -686,6 +689,7 @@ cudaError_t launch_hadamard_quantize(const void* X, size_t rows, int K, int r, i
     const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(X);
     // 1024 threads per row only when rows do not outnumber the SMs: at 28672-wide rows (two 256-thread CTAs per SM)
     // the wide form measured slower for many rows (0.89 against 0.72 ms at 8192 rows).
+    count_launch();
     if (rows <= kWideMaxRows) {
         if (m == 1) hadamard_quantize_kernel<1, kWideThreads><<<grid, kWideThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);
         else if (m == 12) hadamard_quantize_kernel<12, kWideThreads><<<grid, kWideThreads, smem, st>>>(x, rows, K, kbits, r, inv_sqrt_k, q8, q4, s8, s4, q4_i8);

@@ -92,9 +92,9 @@ split_quantize_asym_kernel(const void* __restrict__ in, size_t in_row_bytes, siz
                       reinterpret_cast<const char*>(in) + (row0 + i) * in_row_bytes, row_bytes, &bar);
     }
     __syncthreads();
-    const bool landed = mbar_wait(&bar, 0, &abort_flag);
+    const bool landed = mbar_wait(&bar, 0, &abort_flag, status);
     if (__syncthreads_or(!landed)) {
-        if (threadIdx.x == 0) atomicOr(status, RESQ_ERR_TIMEOUT);
+        if (threadIdx.x == 0) atomicOr(status, kStatusBitTimeout);
         return;
     }
 
@@ -243,6 +243,7 @@ cudaError_t launch_split_quantize_asym(const void* in, bool in_is_f32, size_t ro
     }
     const size_t groups = (rows + rpc - 1) / rpc;
     if (groups > 0x7fffffffu) return cudaErrorNotSupported;
+    count_launch();
     kern<<<static_cast<unsigned>(groups), kThreads, smem, st>>>(in, in_row_stride_bytes, rows, K, r, rpc, u8, u4, s8, s4,
                                                             z8, z4, u4_u8, device_status_ptr());
     return cudaGetLastError();
@@ -250,6 +251,7 @@ cudaError_t launch_split_quantize_asym(const void* in, bool in_is_f32, size_t ro
 
 cudaError_t launch_weight_row_sums(const int8_t* w8, const uint8_t* w4, int N, int K, int r, int32_t* wsum8,
                                    int32_t* wsum4, cudaStream_t st) {
+    count_launch();
     weight_row_sums_kernel<<<(N + 7) / 8, 256, 0, st>>>(w8, w4, N, r, (K - r) / 2, wsum8, wsum4);
     return cudaGetLastError();
 }

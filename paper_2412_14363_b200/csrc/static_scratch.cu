@@ -46,8 +46,8 @@ using namespace resq;
 
 extern "C" int resq_project_quantize_static(const void* X, const void* P, int T, int K, int r, int8_t* x8,
                                             uint8_t* x4, float* s_x8, float* s_x4, int8_t* x4_i8, void* stream) {
-    if (T < 1 || K <= 0 || r <= 0 || r >= K || r % 32 != 0 || (K - r) % 32 != 0) return RESQ_ERR_SHAPE;
-    if (!X || !P || !x8 || !s_x8 || !s_x4 || (!x4 && !x4_i8)) return RESQ_ERR_NULL;
+    if (T < 1 || K <= 0 || r < 0 || r >= K || r % 32 != 0 || (K - r) % 32 != 0) return RESQ_ERR_SHAPE;
+    if (!X || !P || (!x8 && r > 0) || !s_x8 || !s_x4 || (!x4 && !x4_i8)) return RESQ_ERR_NULL;
     if (!aligned16(X) || !aligned16(P) || !aligned16(x8) || !aligned16(x4) || !aligned16(s_x8) ||
         !aligned16(s_x4) || !aligned16(x4_i8))
         return RESQ_ERR_ALIGN;

@@ -3,10 +3,9 @@ from __future__ import annotations
 
 import ctypes
 
-from . import ERR_CUDA, OK, ResqError, _check, _ptr, _stream, lib  # noqa: F401
+from . import ERR_CUDA, ERR_INDEX, OK, ResqError, _check, _ptr, _stream, lib  # noqa: F401
 
 KV_BLOCK, KV_BLOCK_BYTES = 32, 5632
-ERR_INDEX = 8
 KV_EXPORTS = ["resq_kv_cache_bytes", "resq_uc_quantize", "resq_query_project", "resq_kv_append", "resq_qkv_project_append",
               "resq_attention_workspace_bytes", "resq_attention_decode"]
 

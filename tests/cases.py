@@ -45,6 +45,13 @@ def config1() -> FoldedCase:
     return pca_case(16, 512, 512, 64, "normal", 256)
 
 
+def config2_basis() -> FoldedCase:
+    """The d = 2048 input dimension of the Llama-3.2-1B-shaped configuration on the real construction: Student-t
+    activations with 1 % of the channels x20, PCA on a separate 4096-token calibration batch, QR-of-Gaussian
+    rotations 256x256 and 1792x1792; 64 token rows and 512 output channels keep the oracle's layer in seconds."""
+    return pca_case(64, 2048, 512, 256, "t4", 4096)
+
+
 def synthetic_folded(T: int, K: int, N: int, r: int, seed_shift: int = 0):
     """Coefficients and projected weights drawn directly (no basis needed): bf16 t4 coefficients with
     outlier channels, fp32 Gaussian projected weights.  For shape sweeps of the kernels."""

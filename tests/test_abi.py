@@ -160,6 +160,7 @@ def test_options_and_error_text(resq):
     """Host-only entry points: an unknown option is refused, the known one toggles, and the CUDA error
     text is a string even when no CUDA error has occurred."""
     assert resq.lib.resq_set_option(12345, 1) == resq.ERR_SHAPE
+    assert resq.lib.resq_set_option(resq.OPT_WAIT_LIMIT_US, 0) == resq.ERR_SHAPE      # refused before any device call
     assert resq.lib.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 1) == resq.OK
     assert resq.lib.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 0) == resq.OK
     assert isinstance(resq.lib.resq_last_cuda_error(), bytes)

@@ -5,6 +5,7 @@ import pytest
 import torch
 
 import oracle
+import synth
 from tests.gpu_util import bf16_bits_from_dev, bf16_to_dev, dev, host
 from tests.test_gpu_parity import check_output, oracle_case, run_mixed_gemm
 
@@ -146,3 +147,48 @@ def test_decode_early_weights_back_to_back(resq):
     for (_, _, pw, res), (W, x8, x4, s8, s4, y, a8, a4, ws) in zip(cases, packs):
         assert (host(a8) == res.acc8).all() and (host(a4) == res.acc4).all()
         check_output(res, pw, host(y))
+
+
+@pytest.mark.parametrize("T,K,N,r", [(1, 14336, 4096, 1792), (4, 14336, 4096, 1792), (16, 14336, 512, 1792),
+                                     (16, 2304, 264, 288), (3, 2304, 72, 0)])
+def test_decode_linear_with_online_projection(resq, T, K, N, r):
+    """resq_linear with P given for up to 16 tokens -- the down_proj of a generation step through the public call:
+    few-token projection kernel, slice reduction, row quantizer, streaming kernel.  The codes the path forms lie
+    within +-1 of the oracle's (fp64-summed projection) on at most 0.1 % of the elements, the scales within the
+    accumulation bound, and the layer output is exact given those codes."""
+    X_bits = synth.f32_to_bf16_bits(synth.activations(T, K, "t4", seed=1300 + T))
+    P_bits = synth.f32_to_bf16_bits(synth.kron_orthogonal_bf16(K, inner=128 if K % 128 == 0 else 32))
+    Wp = synth.projected_weights_direct(N, K, seed=1301)
+    pw = oracle.pack_weights(Wp, r, scale_fp16=True)
+    desc = resq.layer_desc(K, N, r, resq.SCALE_FP16)
+    W = resq.resq_pack_weights(desc, dev(Wp), with_w4_i8=False)
+    ws = resq.alloc_workspace(desc, T, True, False)
+    X, P = bf16_to_dev(X_bits), bf16_to_dev(P_bits)
+    K4 = K - r
+    x8 = torch.empty((T, r), dtype=torch.int8, device="cuda") if r else None
+    x4 = torch.empty((T, K4 // 2), dtype=torch.uint8, device="cuda")
+    s8 = torch.full((T,), -1.0, dtype=torch.float32, device="cuda")
+    s4 = torch.full((T,), -1.0, dtype=torch.float32, device="cuda")
+    resq.resq_project_quantize(X, P, r, x8, x4, s8, s4, None, ws)       # the codes the layer call forms inside
+    y32 = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+    resq.resq_linear(W, X, P, y32, ws)
+    ybf = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    resq.resq_linear(W, X, P, ybf, ws)
+    assert resq.resq_device_status() == resq.OK
+    # against the oracle's projection + quantizer
+    C = oracle.project(X_bits, P_bits)
+    q8, q4, o8, o4 = oracle.split_quantize(C, r)
+    g4 = oracle.unpack_nibbles(host(x4)).astype(np.int32)
+    g8 = host(x8).astype(np.int32) if r else np.zeros((T, 0), np.int32)
+    assert np.abs(g4 - q4).max() <= 1 and (r == 0 or np.abs(g8 - q8).max() <= 1)
+    assert ((g8 != q8).sum() + (g4 != q4).sum()) / float(T * K) <= 1e-3
+    ulp = lambda a, b: np.abs(a.view(np.int32).astype(np.int64) - b.view(np.int32).astype(np.int64))
+    tol = K // 16 + 4
+    assert ulp(host(s4), o4).max() <= tol and (r == 0 or ulp(host(s8), o8).max() <= tol)
+    # exact given the path's own codes
+    gs8, gs4 = host(s8), host(s4)
+    acc8 = oracle.int_gemm(g8.astype(np.int8), pw.q8) if r else np.zeros((T, N), np.int32)
+    acc4 = oracle.int_gemm(g4.astype(np.int8), pw.q4)
+    e32, ebf = oracle.epilogue(acc8, acc4, gs8, gs4, pw.s8, pw.s4)
+    res = oracle.LayerResult(None, g8.astype(np.int8), g4.astype(np.int8), None, gs8, gs4, acc8, acc4, e32, ebf)
+    check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))

@@ -1,4 +1,4 @@
-"""Parity at the full sizes of the Llama-3-8B and Llama-3-70B prefill configurations, in the launch configuration
+"""Parity at the full sizes of the Llama-3.2-1B, Llama-3-8B and Llama-3-70B prefill configurations, in the launch configuration
 the benchmark times (all token rows, whole layers, the tile kernels), checked on sampled token rows that the
 oracle can afford: for those rows everything the layer produces is compared -- codes, scales, the fp32 output
 of every output channel."""
@@ -29,6 +29,9 @@ def _sample_rows(T):
 
 
 @pytest.mark.parametrize("T,K,N", [
+    (2048, 2048, 16384),    # Llama-3.2-1B gate|up
+    (2048, 2048, 3072),     # Llama-3.2-1B q|k|v (2048 + 2 x 512 output channels)
+    (2048, 2048, 2048),     # Llama-3.2-1B o
     (4096, 4096, 28672),    # 8B gate|up: the widest layer of the benchmark
     (4096, 4096, 6144),     # 8B q|k|v
     (8192, 8192, 10240),    # 70B q|k|v (8192 + 2 x 1024 output channels)
@@ -54,7 +57,7 @@ def test_folded_layer_full_size_sampled_rows(resq, T, K, N):
     check_output(res, pw, host(Y[torch.from_numpy(rows).to(dev)]))
 
 
-@pytest.mark.parametrize("T,K,N", [(4096, 14336, 4096), (8192, 28672, 8192)])
+@pytest.mark.parametrize("T,K,N", [(2048, 8192, 2048), (4096, 14336, 4096), (8192, 28672, 8192)])
 def test_down_proj_full_size_sampled_rows(resq, T, K, N):
     """down_proj with the online projection at full size: the kernel's codes on the sampled rows lie within +-1 of
     the oracle's on <= 0.1 %, and its output is exact given its own codes."""

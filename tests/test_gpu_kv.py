@@ -139,7 +139,7 @@ def test_fused_project_append_matches_the_two_calls(resq, kv, uc):
         assert (host(ca.data) != 7).any()
 
 
-def _attention_case(kv, seq_lens, Hq, Hkv, capacity, seed, v_scale=1.0, v_shift=0.3, fill=0xFF):
+def _attention_case(kv, seq_lens, Hq, Hkv, capacity, seed, v_scale=1.0, v_shift=0.3, fill=0xFF, device_consumer=False):
     """Cache image built on the CPU from the oracle's codes (no GPU kernel upstream), attention on both sides."""
     B = len(seq_lens)
     image = kv_util.empty_image(B, Hkv, capacity, fill)            # 0xFF: NaN scales in every unused slot
@@ -166,7 +166,17 @@ def _attention_case(kv, seq_lens, Hq, Hkv, capacity, seed, v_scale=1.0, v_shift=
     out = torch.full((B, Hq, D), float("nan"), dtype=torch.float32, device="cuda")
     ws = kv.attention_workspace(cache, Hq)
     ws.fill_(0xFF)
-    kv.resq_attention_decode(cache, dev(q16), dev(np.asarray(seq_lens, np.int32)), out, ws)
+    q16_d, lens_d = dev(q16), dev(np.asarray(seq_lens, np.int32))
+    if device_consumer:
+        # A kernel enqueued right behind the call on the same stream, with no host synchronization in between,
+        # must see the finished outputs: stream order is all a caller has between the attention and the o_proj
+        # quantizer that follows it.
+        spin = torch.empty(1 << 24, dtype=torch.float32, device="cuda")
+        spin.fill_(1.0)                                    # keeps the GPU busy so that the three launches queue up
+        kv.resq_attention_decode(cache, q16_d, lens_d, out, ws)
+        seen = out.clone()
+        return host(seen), ref, vmax
+    kv.resq_attention_decode(cache, q16_d, lens_d, out, ws)
     return host(out), ref, vmax
 
 
@@ -201,6 +211,18 @@ def test_attention_many_short_sequences(resq, kv):
     out, ref, vmax = _attention_case(kv, seq_lens, 8, 8, 64, seed=12)
     assert resq.resq_device_status() == resq.OK
     _assert_close(out, ref, vmax, 8, 8)
+
+
+def test_attention_outputs_are_complete_for_the_next_kernel_of_the_stream(resq, kv):
+    """64 sequences x 8 KV heads of at most one cache block each: every (sequence, head) is seen by a single warp,
+    so the merge kernel has nothing to add -- it must still hold the stream until the attention kernel has
+    written every output, which a device-side copy enqueued straight after the call observes."""
+    rng = np.random.default_rng(9)
+    seq_lens = [int(x) for x in rng.integers(0, 33, 64)]
+    for rep in range(3):
+        out, ref, vmax = _attention_case(kv, seq_lens, 32, 8, 32, seed=14 + rep, device_consumer=True)
+        assert resq.resq_device_status() == resq.OK
+        _assert_close(out, ref, vmax, 32, 8)
 
 
 @pytest.mark.parametrize("v_scale", [1e-7, 3e5])

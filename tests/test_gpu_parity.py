@@ -12,7 +12,7 @@ import torch
 
 import oracle
 import synth
-from tests.cases import config1, synthetic_folded
+from tests.cases import config1, config2_basis, synthetic_folded
 from tests.gpu_util import bf16_bits_from_dev, bf16_to_dev, dev, host
 
 pytestmark = pytest.mark.gpu
@@ -254,3 +254,24 @@ def test_linear_config1_end_to_end(resq, T):
     resq.resq_linear(W, bf16_to_dev(C_bits), None, ybf, ws)
     _check_status(resq)
     check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))
+
+
+def test_linear_d2048_pca_basis_end_to_end(resq):
+    """Whole layer on the PCA + rotation basis built at d = 2048 (the input width of the Llama-3.2-1B-shaped
+    configuration): weights projected by the oracle's U, coefficients bf16(X·U) as a folded projection delivers them."""
+    c = config2_basis()
+    pw = oracle.pack_weights(c.W_proj, c.r)
+    res = oracle.linear(c.C_bits, None, pw)
+    desc = resq.layer_desc(c.K, c.N, c.r)
+    W = resq.resq_pack_weights(desc, dev(c.W_proj))
+    assert (host(W.w8) == pw.q8).all() and (host(W.w4) == pw.w4_packed).all()
+    ws = resq.alloc_workspace(desc, c.T, False, True)
+    y32 = torch.empty((c.T, c.N), dtype=torch.float32, device="cuda")
+    resq.resq_linear(W, bf16_to_dev(c.C_bits), None, y32, ws)
+    ybf = torch.empty((c.T, c.N), dtype=torch.bfloat16, device="cuda")
+    resq.resq_linear(W, bf16_to_dev(c.C_bits), None, ybf, ws)
+    _check_status(resq)
+    check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))
+    # the quantized layer tracks the unquantized product (a sanity bound on the whole chain, not parity)
+    ref = c.X.astype(np.float64) @ c.W.astype(np.float64)
+    assert np.linalg.norm(host(y32) - ref) / np.linalg.norm(ref) < 0.25

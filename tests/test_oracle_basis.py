@@ -21,6 +21,34 @@ def test_U_is_orthogonal_and_layer_is_invariant_without_quantization():
     assert np.abs(split - ref).max() / np.abs(ref).max() < 1e-12
 
 
+def test_basis_at_d2048_orthogonal_invariant_and_ordered():
+    """The same construction at the 2048-wide input of the Llama-3.2-1B-shaped configuration (4096 calibration
+    tokens, r = 256): orthogonality, the unquantized invariance X·U·U^T·W = X·W with vanishing cross terms,
+    eigen-residuals, descending order, the trace identity, subspaces kept by the rotations, and the outlier
+    channels inside the high-precision subspace."""
+    from tests.cases import config2_basis
+    c = config2_basis()
+    U, r = c.U, c.r
+    assert np.abs(U.T @ U - np.eye(c.K)).max() < 1e-12
+    X, W = c.X.astype(np.float64), c.W.astype(np.float64)
+    ref = X @ W
+    assert np.abs((X @ U) @ (U.T @ W) - ref).max() / np.abs(ref).max() < 1e-12
+    split = (X @ U[:, :r]) @ (U[:, :r].T @ W) + (X @ U[:, r:]) @ (U[:, r:].T @ W)
+    assert np.abs(split - ref).max() / np.abs(ref).max() < 1e-12
+    G = basis.second_moment(c.X_calib)
+    assert (np.diff(c.lam) <= 1e-9 * c.lam[0]).all()
+    assert np.abs(G @ c.P - c.P * c.lam).max() < 1e-9 * c.lam[0]
+    assert np.isclose(c.lam.sum(), (c.X_calib.astype(np.float64) ** 2).sum() / c.X_calib.shape[0], rtol=1e-12)
+    rq = np.einsum("ij,ij->j", c.P[:, :r], G @ c.P[:, :r])
+    assert np.allclose(rq, c.lam[:r], rtol=1e-9)
+    assert np.abs(U[:, :r] @ U[:, :r].T - c.P[:, :r] @ c.P[:, :r].T).max() < 1e-11
+    out = synth.outlier_channels(c.K, synth.n_outliers(c.K))
+    assert ((c.P[out, :r] ** 2).sum(1) > 0.99).all()
+    # the coefficient layout the layer receives: bf16(X·U), high-variance block first
+    Cf = synth.bf16_bits_to_f32(c.C_bits).astype(np.float64)
+    assert (Cf[:, :r] ** 2).mean() > 4 * (Cf[:, r:] ** 2).mean()
+
+
 def test_pca_eigenpairs_descending_and_residuals():
     c = config1()
     G = basis.second_moment(c.X_calib)

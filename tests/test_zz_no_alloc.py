@@ -5,7 +5,11 @@ own pool, or they sit in a loop where cudaMalloc (which synchronises the whole d
 For them the fp32 staging panel is an 8 MiB array built into the library.  This file checks, through
 the C ABI, that the variant gives exactly what the regular entry point gives -- it runs the same two
 kernels, so codes and scales must be identical bit for bit -- on two calls in a row with different
-inputs (the array keeps the first call's contents, which the second must not see).
+inputs (the array keeps the first call's contents, which the second must not see).  For up to 64 token
+rows -- a generation step, the likeliest use -- the regular call given its full workspace cuts the
+projection along K and so adds in another order; there the variant is compared with the CPU oracle
+under the online path's own criterion, bit for bit with the regular call given a panel-only workspace,
+and within one code step of the regular call given its full workspace.
 
 Collected last on purpose: a run that stops at the first failure has then already run everything else.
 """
@@ -13,6 +17,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import synth
 from tests.gpu_util import bf16_to_dev, host
 
@@ -43,6 +48,50 @@ def test_static_scratch_variant_matches_regular_entry_point_twice():
             assert torch.equal(a, b)
         assert (host(got[2]) > 0).all() and (host(got[3]) > 0).all()
         assert np.abs(host(got[0])).max() == 127 and np.abs(host(got[4])).max() == 7
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("T,K,r", [(1, 14336, 1792), (16, 14336, 1792), (64, 14336, 1792), (5, 8192, 0)])
+def test_static_scratch_variant_few_rows_against_the_oracle(T, K, r):
+    import paper_2412_14363_b200 as resq
+    K4 = K - r
+    X_bits = synth.f32_to_bf16_bits(synth.activations(T, K, "t4", seed=950 + T))
+    P_bits = synth.f32_to_bf16_bits(synth.kron_orthogonal_bf16(K))
+    X, P = bf16_to_dev(X_bits), bf16_to_dev(P_bits)
+    q8, q4, o8, o4 = oracle.split_quantize(oracle.project(X_bits, P_bits), r)
+    x8 = lambda t: t[0] if r else None                           # r = 0: no INT8 segment, NULL accepted
+
+    def check_against_oracle(out):
+        g8, g4 = host(out[0]).astype(np.int32), host(out[4]).astype(np.int32)
+        assert (host(out[1]) == oracle.pack_nibbles(host(out[4]))).all()
+        assert np.abs(g4 - q4).max() <= 1 and (r == 0 or np.abs(g8 - q8).max() <= 1)
+        assert (((g8 != q8).sum() if r else 0) + (g4 != q4).sum()) / float(T * K) <= 1e-3
+        ulp = lambda a, b: np.abs(a.view(np.int32).astype(np.int64) - b.view(np.int32).astype(np.int64))
+        assert ulp(host(out[3]), o4).max() <= K // 16 + 4
+        if r:
+            assert ulp(host(out[2]), o8).max() <= K // 16 + 4
+        else:
+            assert (host(out[2]) == 0).all()                     # empty INT8 segment: scale 0
+
+    for _ in range(2):                                           # two calls in a row
+        got = _outputs(T, K, r)
+        resq.resq_project_quantize_static(X, P, r, x8(got), got[1], got[2], got[3], got[4])
+        assert resq.resq_device_status() == resq.OK
+        check_against_oracle(got)
+    # bit for bit what the regular call gives when its workspace holds the panel alone
+    panel_only = torch.empty(((T * K * 4 + 255) // 256) * 256, dtype=torch.uint8, device="cuda")
+    ref = _outputs(T, K, r)
+    resq.resq_project_quantize(X, P, r, x8(ref), ref[1], ref[2], ref[3], ref[4], panel_only)
+    for a, b in zip(got, ref):
+        assert torch.equal(a, b)
+    # the regular call with its full workspace adds the K slices in another order: one code step at most
+    full = _outputs(T, K, r)
+    resq.resq_project_quantize(X, P, r, x8(full), full[1], full[2], full[3], full[4],
+                               resq.alloc_workspace(resq.layer_desc(K, 8, r), T, True, True))
+    assert resq.resq_device_status() == resq.OK
+    check_against_oracle(full)
+    d4 = np.abs(host(full[4]).astype(np.int32) - host(got[4]).astype(np.int32))
+    assert d4.max() <= 1 and (d4 != 0).mean() <= 2e-3
 
 
 @pytest.mark.gpu
