@@ -3,8 +3,9 @@
 //
 // Work split.  The weight rows are cut into units of 8 output channels; CTA b of a persistent grid
 // (one CTA per SM) owns a contiguous, balanced range of units.  Inside the CTA the work is the
-// sequence of (item, chunk) pairs -- an item is a pair of units (16 channels), a chunk a slice of
-// its reduction dimension -- cut into eight equal runs, one per warp.  A warp that holds a whole item
+// sequence of (item, chunk) pairs -- an item is a pair of units (16 channels; the last item of a CTA
+// may be a single unit, whose copies bring 8 rows), a chunk a slice of its reduction dimension -- cut
+// into runs of equal cost, one per warp (an INT4 chunk counts about twice an INT8 chunk).  A warp that holds a whole item
 // finishes it alone; an item shared by several warps is summed in a shared-memory slot with integer
 // atomics and finished by whichever warp arrives last.  Integer sums do not depend on order, so the
 // result is the same bit for bit whatever the split; no warp ever waits for another, and there is no
@@ -18,8 +19,9 @@
 // below.  The rings together are as large as shared memory allows, so the bytes in flight per SM
 // do not depend on how fast the arithmetic runs.
 //
-// Arithmetic.  mma.sync.m16n8k32 (s8) with the tokens as the 16-row operand (shared by the item's
-// two units) and a unit's 8 channels as the 8-column operand; the reduction index may be permuted
+// Arithmetic.  mma.sync.m16n8k32 (s8) with the item's 16 weight rows (two units) as the 16-row operand and
+// up to 8 tokens as the 8-column operand (a second product per step for tokens 9-16), so that a step over
+// 64 bytes of each row costs as many products as there are token groups; the reduction index may be permuted
 // freely as long as both operands use the same permutation, so each thread simply takes 16
 // contiguous bytes of its row.  INT4 codes are never sign-extended one by one.  For a packed word w
 // (code 2j in the low, 2j+1 in the high nibble of byte j):
@@ -52,17 +54,17 @@ constexpr int kItemRows = 16;  // two units share the token operand
 constexpr int kMaxStages = 8;
 constexpr int kMinStages = 2;
 constexpr int kSmemLimit = 227 * 1024;
-constexpr int kControlBytes = 1024;
-constexpr int kSlotInts = 2 * 2 * 128;  // [half][acc8 | acc4][fragment element]: one shared item
+constexpr int kControlBytes = kWarps > 8 ? 2048 : 1024;
+constexpr int kSlotInts = 2 * 2 * 128;  // [token group][acc8 | acc4][fragment element]: one shared item
 constexpr int kSlotBytes = kWarps * kSlotInts * 4;
 constexpr uint32_t kHi = 0xF0F0F0F0u, kLo = 0x0F0F0F0Fu, kFlip = 0x08080808u;
 
 struct Params {
     int T, N, r, row4;     // row4 = (K - r) / 2: bytes of a packed INT4 weight row
     int c8, c4;            // chunks per row in the INT8 / INT4 segment
-    int units;             // N / 8
     int pitch8, pitch4;    // bytes per token of the staged activations (zero padded to whole chunks)
     int nstages;           // stages per warp
+    int ring_ofs;          // byte offset of the rings in shared memory (128-byte aligned)
     int early_weights;     // the launch allows an early start: the rings fill before the wait for the upstream kernel
     const int8_t* x8;
     const uint8_t* x4;
@@ -81,6 +83,14 @@ struct Params {
     int32_t* dbg8;
     int32_t* dbg4;
     int* status;
+    // Head of the NEXT few-token launch's weight stream, prefetched into L2 by this launch (0 stages = off): the
+    // geometry of that launch's work split, so that warp w of CTA b asks for what warp w of CTA b will load first.
+    int nx_stages, nx_grid, nx_uq, nx_urem, nx_c8, nx_c4, nx_chunk_words;
+    // Work split: CTA b owns units [b * uq + floor(b * urem / grid), ...): uq or uq + 1 of them; tab[0] / tab[1] hold the warps' run
+    // boundaries (run_boundary) for those two sizes.  nx_tab: the same for the next launch.
+    int uq, urem;
+    int tab[2][kWarps + 1];
+    int nx_tab[2][kWarps + 1];
 };
 
 struct __align__(16) Control {
@@ -91,13 +101,13 @@ struct __align__(16) Control {
 };
 static_assert(sizeof(Control) <= kControlBytes, "control block");
 
-// AU: the 16-row operand (the tokens) holds unsigned bytes.
-template <bool AU>
+// D (16 x 8, int32) += A (16 x 32, s8: weight rows) * B (32 x 8: token columns; BU: unsigned bytes).
+template <bool BU>
 __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
-    if constexpr (AU)
+    if constexpr (BU)
         asm volatile(
-            "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            "mma.sync.aligned.m16n8k32.row.col.s32.s8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
             : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
             : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
     else
@@ -110,13 +120,41 @@ __device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, ui
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// Two consecutive per-channel scales (channels n, n + 1; n even).
-__device__ __forceinline__ float2 load_scale2(const void* p, int n, int fp16) {
-    if (fp16) return __half22float2(*reinterpret_cast<const __half2*>(reinterpret_cast<const __half*>(p) + n));
-    return *reinterpret_cast<const float2*>(reinterpret_cast<const float*>(p) + n);
+// One per-channel scale: the raw bits now, the value when it is needed (an item's scales are requested when its
+// first chunk is, and used after its last: converting at once would make the warp wait for a DRAM round trip
+// before it touches the weights that are already in its ring).
+__device__ __forceinline__ uint32_t load_scale_raw(const void* p, int n, int fp16) {
+    if (fp16) return __ldg(reinterpret_cast<const unsigned short*>(p) + n);
+    return __ldg(reinterpret_cast<const uint32_t*>(p) + n);
+}
+__device__ __forceinline__ float scale_value(uint32_t raw, int fp16) {
+    return fp16 ? __half2float(__ushort_as_half(static_cast<unsigned short>(raw))) : __uint_as_float(raw);
 }
 
-// TT:     1 for T <= 8 (token rows 8..15 of the 16-row operand are zero and are not staged), 2 for T <= 16.
+// floor(a * b / d) for small non-negative a * b (< 2^20) and 0 < d < 2^12, without an integer division: the
+// quotient of (a * b + 0.5) by d stays clear of every integer by far more than fp32 rounding.
+__device__ __forceinline__ int small_muldiv(int a, int b, int d) {
+    return __float2int_rd(__fdividef(static_cast<float>(a * b) + 0.5f, static_cast<float>(d)));
+}
+
+// Cost of one chunk in the split of a CTA's work over its warps: an INT4 chunk takes about twice the
+// instructions of an INT8 chunk of the same bytes (two products per packed word plus the nibble logic).
+constexpr int kCost8 = 4, kCost4 = 9;
+
+// Where the run of warp w begins when the (item, chunk) sequence of a CTA with `items` items is cut into kWarps runs
+// of equal cost, packed as item << 16 | chunk; w = kWarps gives the end of the sequence.  Evaluated on the host
+// for the two CTA sizes of a launch (Params::tab), so that the kernel's prologue has no divisions.
+inline int run_boundary(int w, int items, int c8, int c4) {
+    if (w >= kWarps || items == 0) return items << 16;
+    const int cf = kCost8 * c8 + kCost4 * c4;
+    const long long pos = static_cast<long long>(items) * cf * w / kWarps;
+    const int item = static_cast<int>(pos / cf);
+    const int q = static_cast<int>(pos - static_cast<long long>(item) * cf);
+    const int chunk = q < kCost8 * c8 ? q / kCost8 : c8 + (q - kCost8 * c8) / kCost4;
+    return item << 16 | chunk;
+}
+
+// TT:     1 for T <= 8 (token rows 8..15 of the 16-row operand are zero), 2 for T <= 16.
 // CS:     64-byte steps per chunk (3 or 5).
 // kSplit: the INT4 activations are staged already split into their even / odd codes times 16 (twice
 //         the shared memory, a third of the logic operations); otherwise they stay packed and are
@@ -128,27 +166,39 @@ __device__ __forceinline__ float2 load_scale2(const void* p, int n, int fp16) {
 template <int TT, int CS, bool kSplit, bool ASYM>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_constant__ CUtensorMap tmW4,
+                         const __grid_constant__ CUtensorMap tmH8, const __grid_constant__ CUtensorMap tmH4,
+                         const __grid_constant__ CUtensorMap tmN8, const __grid_constant__ CUtensorMap tmN4,
                          const Params p) {
     extern __shared__ __align__(128) uint8_t smem[];
-    constexpr int TP = TT * 8;
     constexpr int kChunkBytes = CS * 64;
     constexpr int kStageBytes = kItemRows * kChunkBytes;
     Control* ctl = reinterpret_cast<Control*>(smem);
     int* slots = reinterpret_cast<int*>(smem + kControlBytes);                        // [kWarps][kSlotInts]
-    uint8_t* act8 = smem + kControlBytes + kSlotBytes;                                // [TP][pitch8]
-    uint8_t* act4 = act8 + static_cast<size_t>(TP) * p.pitch8;                        // kSplit: even [TP][pitch4], odd [TP][pitch4]; else packed [TP][pitch4]
-    uint8_t* rings = act4 + static_cast<size_t>(kSplit ? 2 : 1) * TP * p.pitch4;      // [kWarps][nstages][16][chunk]
+    // Staged activation codes: rows [0, T) are the tokens, row T is all zeros (what the 16-row operand reads for
+    // its rows beyond T).
+    const int TR = p.T + 1;
+    uint8_t* act8 = smem + kControlBytes + kSlotBytes;                                // [T + 1][pitch8]
+    uint8_t* act4 = act8 + static_cast<size_t>(TR) * p.pitch8;                        // kSplit: even [T + 1][pitch4], odd [T + 1][pitch4]; else packed [T + 1][pitch4]
+    uint8_t* rings = smem + p.ring_ofs;                                               // [kWarps][nstages][16][chunk]
     volatile int* abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        tma_prefetch_desc(&tmW8);
+        tma_prefetch_desc(&tmW4);
+    }
     const int g = lane >> 2, tig = lane & 3;
-    const int u0 = static_cast<int>(static_cast<long long>(p.units) * blockIdx.x / gridDim.x);
-    const int u1 = static_cast<int>(static_cast<long long>(p.units) * (blockIdx.x + 1) / gridDim.x);
+    const int bx = static_cast<int>(blockIdx.x);
+    const int nbx = static_cast<int>(gridDim.x);
+    const int u0 = bx * p.uq + small_muldiv(bx, p.urem, nbx), u1 = (bx + 1) * p.uq + small_muldiv(bx + 1, p.urem, nbx);
+    const int big = u1 - u0 - p.uq;                                                   // 1: this CTA owns uq + 1 units
     const int cta_items = (u1 - u0 + 1) >> 1;
+    const bool last_half = ((u1 - u0) & 1) != 0;
     const int nchunks = p.c8 + p.c4;
-    const int cta_chunks = cta_items * nchunks;
-    auto run_begin = [&](int w) { return static_cast<int>(static_cast<long long>(cta_chunks) * w / kWarps); };
-    const int cb = run_begin(warp), ce = run_begin(warp + 1);  // this warp's run of (item, chunk) pairs
+    const int* tab = p.tab[1 - big];
+    auto linear = [&](int packed) { return (packed >> 16) * nchunks + (packed & 0xFFFF); };
+    const int pb = tab[warp];
+    const int cb = linear(pb), ce = linear(tab[warp + 1]);                            // this warp's run of (item, chunk) pairs
     uint8_t* ring = rings + static_cast<size_t>(warp) * p.nstages * kStageBytes;
     uint64_t* full = ctl->full[warp];
 
@@ -172,17 +222,41 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         asm("lop3.b32 %0, %1, %2, %3, 0x28;" : "=r"(d) : "r"(w), "r"(rflip), "r"(rlo));  // (w ^ rflip) & rlo
         return d;
     };
-    // Issue cursor of this warp (only lane 0 uses it): next (item, chunk) to copy.
-    int is_idx = cb, is_item = cb / nchunks, is_chunk = cb - (cb / nchunks) * nchunks;
+    // Issue cursor of this warp (only lane 0 uses it): next (item, chunk) to copy.  A CTA's last item may be a
+    // single unit: its copies bring 8 rows (the maps with the 8-row box) instead of 16.
+    int is_idx = cb, is_item = pb >> 16, is_chunk = pb & 0xFFFF;
     auto issue = [&](int stage) {
         const int ub = u0 + 2 * is_item;
         const bool seg8 = is_chunk < p.c8;
+        const bool half = last_half && is_item == cta_items - 1;
         const int x = (seg8 ? is_chunk : is_chunk - p.c8) * (kChunkBytes / 4);  // in 32-bit elements: a multiple of 16
-        mbar_arrive_expect_tx(&full[stage], kStageBytes);
-        tma_load_2d_hint(ring + static_cast<size_t>(stage) * kStageBytes, seg8 ? &tmW8 : &tmW4, &full[stage], x, ub * kUnitRows,
-                         stream_policy);
+        mbar_arrive_expect_tx(&full[stage], half ? kStageBytes / 2 : kStageBytes);
+        const CUtensorMap* tm = half ? (seg8 ? &tmH8 : &tmH4) : (seg8 ? &tmW8 : &tmW4);
+        tma_load_2d_hint(ring + static_cast<size_t>(stage) * kStageBytes, tm, &full[stage], x, ub * kUnitRows, stream_policy);
         ++is_idx;
         if (++is_chunk == nchunks) { is_chunk = 0; ++is_item; }
+    };
+
+    // Once this warp has asked for the last of its own weights, it asks L2 for the first ring of the same warp of
+    // the next launch (no shared memory, no barrier involved: the lines simply are in L2 when that launch starts).
+    // HBM then keeps streaming through this launch's drain, the switch of grids and the next launch's ramp.
+    bool next_done = p.nx_stages == 0 || bx >= p.nx_grid;
+    auto prefetch_next = [&]() {
+        next_done = true;
+        const int nu0 = bx * p.nx_uq + small_muldiv(bx, p.nx_urem, p.nx_grid);
+        const int nbig = (bx + 1) * p.nx_uq + small_muldiv(bx + 1, p.nx_urem, p.nx_grid) - nu0 - p.nx_uq;
+        const int nch = p.nx_c8 + p.nx_c4;
+        const int* nt = p.nx_tab[1 - nbig];
+        const int q0 = nt[warp], q1 = nt[warp + 1];
+        int item = q0 >> 16, chunk = q0 & 0xFFFF;
+        const int len = ((q1 >> 16) - item) * nch + (q1 & 0xFFFF) - chunk;
+        const int count = len < p.nx_stages ? len : p.nx_stages;
+        for (int k = 0; k < count; ++k) {
+            const bool seg8 = chunk < p.nx_c8;
+            tma_prefetch_2d(seg8 ? &tmN8 : &tmN4, (seg8 ? chunk : chunk - p.nx_c8) * p.nx_chunk_words,
+                            (nu0 + 2 * item) * kUnitRows);
+            if (++chunk == nch) { chunk = 0; ++item; }
+        }
     };
 
     if (!p.early_weights) griddep_wait();
@@ -193,24 +267,40 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
     if (lane == 0 && first_burst > 0) {
         issue(0);
         issued = 1;
+        if (p.early_weights >= 2) {  // nothing of the preceding kernel is read before the wait below: fill the ring now
+            for (int s = 1; s < first_burst; ++s) issue(s);
+            issued = first_burst;
+        }
     }
     for (int i = threadIdx.x; i < kWarps * kSlotInts; i += kThreads) slots[i] = 0;
     if (threadIdx.x < kWarps) ctl->arrived[threadIdx.x] = 0;
     if (threadIdx.x == 0) ctl->abort_flag = 0;
     if (p.early_weights) griddep_wait();
 
-    // Token scales of the two accumulator rows this thread holds.
-    const float sx8a = g < p.T ? p.s_x8[g] : 0.f, sx4a = g < p.T ? p.s_x4[g] : 0.f;
-    const float sx8b = g + 8 < p.T ? p.s_x8[g + 8] : 0.f, sx4b = g + 8 < p.T ? p.s_x4[g + 8] : 0.f;
-    const float zx8a = ASYM && g < p.T ? p.z_x8[g] : 0.f, zx4a = ASYM && g < p.T ? p.z_x4[g] : 0.f;
-    const float zx8b = ASYM && g + 8 < p.T ? p.z_x8[g + 8] : 0.f, zx4b = ASYM && g + 8 < p.T ? p.z_x4[g + 8] : 0.f;
-    // Stage the activation codes: zero padded to the pitch, zero rows for tokens >= T.  The first
-    // batch of INT8 and of INT4 vectors is loaded before anything is stored (one round trip to L2 for
-    // the usual sizes); the rest of the ring goes out right behind those loads.
+    // The tokens are the 8 columns of the product (one group of 8 per TT): this thread feeds the codes of token g
+    // (and g + 8) and holds the sums of tokens 2 tig, 2 tig + 1 (and + 8).  Their scales and zero-points:
+    const bool a_ok = g < p.T, b_ok = TT == 2 && g + 8 < p.T;
+    float sx8t[TT][2], sx4t[TT][2], zx8t[TT][2], zx4t[TT][2];
+#pragma unroll
+    for (int tt = 0; tt < TT; ++tt)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int t = 8 * tt + 2 * tig + e;
+            const bool t_ok = t < p.T;
+            sx8t[tt][e] = t_ok ? p.s_x8[t] : 0.f;
+            sx4t[tt][e] = t_ok ? p.s_x4[t] : 0.f;
+            zx8t[tt][e] = ASYM && t_ok ? p.z_x8[t] : 0.f;
+            zx4t[tt][e] = ASYM && t_ok ? p.z_x4[t] : 0.f;
+        }
+    // Stage the activation codes of the T tokens, zero padded to the pitch (the weights arrive as zeros there, but an
+    // even INT4 weight code enters the product as code + 8), and the zero row.  The first batch of INT8 and
+    // of INT4 vectors is loaded before anything is stored (one round trip to L2 for the usual sizes); the rest of
+    // the ring goes out right behind those loads.  Meanwhile warp w sums the even-position INT4 codes of tokens
+    // w and w + 8 straight from global memory.
     {
         const int v8 = p.pitch8 >> 4, v4 = p.pitch4 >> 4;  // 16-byte vectors per token
         const int r8 = p.r >> 4, r4 = p.row4 >> 4;         // ... that hold data
-        const int n8 = TP * v8, n4 = TP * v4;
+        const int n8 = TR * v8, n4 = TR * v4;
         constexpr int kBatch = 4;
         auto load8 = [&](int base, uint4 (&v)[kBatch]) {
 #pragma unroll
@@ -248,12 +338,12 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                 uint8_t* dst = act4 + static_cast<size_t>(t) * p.pitch4 + (o << 4);
                 if (kSplit && ASYM) {
                     *reinterpret_cast<uint4*>(dst) = make_uint4(v[b].x & kLo, v[b].y & kLo, v[b].z & kLo, v[b].w & kLo);
-                    *reinterpret_cast<uint4*>(dst + static_cast<size_t>(TP) * p.pitch4) =
+                    *reinterpret_cast<uint4*>(dst + static_cast<size_t>(TR) * p.pitch4) =
                         make_uint4((v[b].x >> 4) & kLo, (v[b].y >> 4) & kLo, (v[b].z >> 4) & kLo, (v[b].w >> 4) & kLo);
                 } else if (kSplit) {
                     *reinterpret_cast<uint4*>(dst) =
                         make_uint4((v[b].x << 4) & kHi, (v[b].y << 4) & kHi, (v[b].z << 4) & kHi, (v[b].w << 4) & kHi);
-                    *reinterpret_cast<uint4*>(dst + static_cast<size_t>(TP) * p.pitch4) =
+                    *reinterpret_cast<uint4*>(dst + static_cast<size_t>(TR) * p.pitch4) =
                         make_uint4(v[b].x & kHi, v[b].y & kHi, v[b].z & kHi, v[b].w & kHi);
                 } else {
                     *reinterpret_cast<uint4*>(dst) = v[b];
@@ -263,9 +353,39 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         uint4 va[kBatch], vb[kBatch];
         load8(0, va);
         load4(0, vb);
+        // Sum of the even-position INT4 codes per token, from the global rows (up to four vectors in flight per lane).
+        constexpr int kTokIters = (8 * TT + kWarps - 1) / kWarps;
+        int se[kTokIters];
+#pragma unroll
+        for (int tt = 0; tt < kTokIters; ++tt) {
+            const int t = warp + kWarps * tt;
+            se[tt] = 0;
+            if (t < p.T) {
+                const uint4* row = reinterpret_cast<const uint4*>(p.x4 + static_cast<size_t>(t) * p.row4);
+                for (int i0 = 0; i0 < r4; i0 += 128) {
+                    uint4 v[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int i = i0 + 32 * k + lane;
+                        v[k] = i < r4 ? __ldg(row + i) : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        uint4 q = v[k];
+                        if (ASYM) q = make_uint4(q.x & kLo, q.y & kLo, q.z & kLo, q.w & kLo);
+                        else q = make_uint4((q.x << 4) & kHi, (q.y << 4) & kHi, (q.z << 4) & kHi, (q.w << 4) & kHi);
+                        se[tt] = __dp4a(static_cast<int>(q.x), 0x01010101, se[tt]);  // the lanes are < 128 when unsigned
+                        se[tt] = __dp4a(static_cast<int>(q.y), 0x01010101, se[tt]);
+                        se[tt] = __dp4a(static_cast<int>(q.z), 0x01010101, se[tt]);
+                        se[tt] = __dp4a(static_cast<int>(q.w), 0x01010101, se[tt]);
+                    }
+                }
+            }
+        }
         if (lane == 0) {
             for (int s = issued; s < first_burst; ++s) issue(s);
             issued = first_burst;
+            if (!next_done && is_idx >= ce) prefetch_next();
         }
         store8(0, va);
         store4(0, vb);
@@ -277,129 +397,111 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             load4(base, vb);
             store4(base, vb);
         }
-    }
-    __syncthreads();
-    // Sum of the even-position INT4 codes per token (warp w: tokens w and w + 8), from the staged rows.
 #pragma unroll
-    for (int tt = 0; tt < TT; ++tt) {
-        const int t = warp + 8 * tt;
-        int se = 0;
-        if (t < p.T) {
-            const uint8_t* row = act4 + static_cast<size_t>(t) * p.pitch4;
-            for (int i = lane; i < (p.pitch4 >> 4); i += 32) {
-                uint4 v = *reinterpret_cast<const uint4*>(row + (i << 4));
-                if (!kSplit) {
-                    if (ASYM) v = make_uint4(v.x & kLo, v.y & kLo, v.z & kLo, v.w & kLo);
-                    else v = make_uint4((v.x << 4) & kHi, (v.y << 4) & kHi, (v.z << 4) & kHi, (v.w << 4) & kHi);
-                }
-                se = __dp4a(static_cast<int>(v.x), 0x01010101, se);  // the lanes are < 128 when unsigned
-                se = __dp4a(static_cast<int>(v.y), 0x01010101, se);
-                se = __dp4a(static_cast<int>(v.z), 0x01010101, se);
-                se = __dp4a(static_cast<int>(v.w), 0x01010101, se);
-            }
+        for (int tt = 0; tt < kTokIters; ++tt) {
+            int v = se[tt];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == 0 && warp + kWarps * tt < p.T) ctl->s_even[warp + kWarps * tt] = ASYM ? v : v >> 4;  // signed codes: the lanes held 16 x the codes
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
-        if (lane == 0) ctl->s_even[t] = ASYM ? se : se >> 4;  // signed codes: the lanes held 16 x the codes
     }
     __syncthreads();
-    const int sev_a = ctl->s_even[g], sev_b = TT == 2 ? ctl->s_even[g + 8] : 0;
+    int sevt[TT][2];
+#pragma unroll
+    for (int tt = 0; tt < TT; ++tt)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) sevt[tt][e] = 8 * tt + 2 * tig + e < p.T ? ctl->s_even[8 * tt + 2 * tig + e] : 0;
 
-    const uint8_t* a8row = act8 + static_cast<size_t>(g) * p.pitch8 + 16 * tig;
-    const uint8_t* a4row = act4 + static_cast<size_t>(g) * p.pitch4 + 16 * tig;
+    const uint8_t* a8row = act8 + static_cast<size_t>(a_ok ? g : p.T) * p.pitch8 + 16 * tig;
+    const uint8_t* a4row = act4 + static_cast<size_t>(a_ok ? g : p.T) * p.pitch4 + 16 * tig;
+    const uint8_t* b8row = act8 + static_cast<size_t>(b_ok ? g + 8 : p.T) * p.pitch8 + 16 * tig;
+    const uint8_t* b4row = act4 + static_cast<size_t>(b_ok ? g + 8 : p.T) * p.pitch4 + 16 * tig;
+    const size_t odd_ofs = static_cast<size_t>(TR) * p.pitch4;  // kSplit: the odd codes follow the even ones
     const int wofs = g * kChunkBytes + 16 * tig;
 
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     int consumed = 0;
-    int idx = cb, item = cb / nchunks, c = cb - (cb / nchunks) * nchunks;
+    int idx = cb, item = pb >> 16, c = pb & 0xFFFF;
     while (idx < ce && ok) {
         // One segment: this warp's part of `item` (all of it, or a slice of its chunks).
         const int seg_begin = idx;
         const int ub = u0 + 2 * item;
         const int halves = u1 - ub >= 2 ? 2 : 1;
-        const int n0 = ub * kUnitRows + 2 * tig;  // first of this thread's two channels in half 0
+        const int n0 = ub * kUnitRows + g;  // this thread's channel in unit 0 of the item (unit 1: + 8)
         // Channel scales, fetched now and used after the reduction.
-        float2 sw8[2], sw4[2];
-        int2 ws8[2] = {}, ws4[2] = {};
+        uint32_t rw8[2], rw4[2];
+        int ws8[2] = {}, ws4[2] = {};
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int n = h < halves ? n0 + 8 * h : n0;
-            sw8[h] = load_scale2(p.s_w8, n, p.w_fp16);
-            sw4[h] = load_scale2(p.s_w4, n, p.w_fp16);
+            rw8[h] = load_scale_raw(p.s_w8, n, p.w_fp16);
+            rw4[h] = load_scale_raw(p.s_w4, n, p.w_fp16);
             if (ASYM) {
-                ws8[h] = *reinterpret_cast<const int2*>(p.wsum8 + n);
-                ws4[h] = *reinterpret_cast<const int2*>(p.wsum4 + n);
+                ws8[h] = __ldg(p.wsum8 + n);
+                ws4[h] = __ldg(p.wsum4 + n);
             }
         }
-        int acc8[2][4], accO[2][4], accE[2][4];
+        // Sums of this warp's part of the item: element i of group tt is unit i >> 1 (channel n0 + 8 (i >> 1)),
+        // token 8 tt + 2 tig + (i & 1).
+        int acc8[TT][4], accO[TT][4], accE[TT][4];
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
+        for (int tt = 0; tt < TT; ++tt)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc8[h][i] = accO[h][i] = accE[h][i] = 0;
+            for (int i = 0; i < 4; ++i) acc8[tt][i] = accO[tt][i] = accE[tt][i] = 0;
 
         for (; c < nchunks && idx < ce; ++c, ++idx) {
             if (!mbar_wait(&full[stage], phase, abort_flag, p.status)) { ok = false; break; }
             const uint8_t* w0 = ring + static_cast<size_t>(stage) * kStageBytes + wofs;
-            const uint8_t* w1 = w0 + 8 * kChunkBytes;
+            const uint8_t* w1 = w0 + 8 * kChunkBytes;  // a single unit: stale rows, their sums are never used
             if (c < p.c8) {
-                const uint8_t* xa = a8row + c * kChunkBytes;
+                const int co = c * kChunkBytes;
 #pragma unroll
                 for (int s = 0; s < CS; ++s) {
-                    const uint4 x = *reinterpret_cast<const uint4*>(xa + 64 * s);
-                    uint4 y = make_uint4(0, 0, 0, 0);
-                    if (TT == 2) y = *reinterpret_cast<const uint4*>(xa + 8 * p.pitch8 + 64 * s);
                     const uint4 wa = *reinterpret_cast<const uint4*>(w0 + 64 * s);
                     const uint4 wb = *reinterpret_cast<const uint4*>(w1 + 64 * s);
-                    mma_s8<ASYM>(acc8[0], x.x, y.x, x.y, y.y, wa.x, wa.y);
-                    mma_s8<ASYM>(acc8[1], x.x, y.x, x.y, y.y, wb.x, wb.y);
-                    mma_s8<ASYM>(acc8[0], x.z, y.z, x.w, y.w, wa.z, wa.w);
-                    mma_s8<ASYM>(acc8[1], x.z, y.z, x.w, y.w, wb.z, wb.w);
+                    const uint4 x = *reinterpret_cast<const uint4*>(a8row + co + 64 * s);
+                    mma_s8<ASYM>(acc8[0], wa.x, wb.x, wa.y, wb.y, x.x, x.y);
+                    mma_s8<ASYM>(acc8[0], wa.z, wb.z, wa.w, wb.w, x.z, x.w);
+                    if (TT == 2) {
+                        const uint4 y = *reinterpret_cast<const uint4*>(b8row + co + 64 * s);
+                        mma_s8<ASYM>(acc8[TT - 1], wa.x, wb.x, wa.y, wb.y, y.x, y.y);
+                        mma_s8<ASYM>(acc8[TT - 1], wa.z, wb.z, wa.w, wb.w, y.z, y.w);
+                    }
                 }
             } else {
-                const uint8_t* xa = a4row + (c - p.c8) * kChunkBytes;
+                const int co = (c - p.c8) * kChunkBytes;
 #pragma unroll
                 for (int s = 0; s < CS; ++s) {
-                    uint32_t xe[4], xo[4], ye[4], yo[4];
-                    if (kSplit) {
-                        const uint8_t* xod = xa + static_cast<size_t>(TP) * p.pitch4;
-                        const uint4 e = *reinterpret_cast<const uint4*>(xa + 64 * s);
-                        const uint4 o = *reinterpret_cast<const uint4*>(xod + 64 * s);
-                        xe[0] = e.x; xe[1] = e.y; xe[2] = e.z; xe[3] = e.w;
-                        xo[0] = o.x; xo[1] = o.y; xo[2] = o.z; xo[3] = o.w;
-                        uint4 e2 = make_uint4(0, 0, 0, 0), o2 = e2;
-                        if (TT == 2) {
-                            e2 = *reinterpret_cast<const uint4*>(xa + 8 * p.pitch4 + 64 * s);
-                            o2 = *reinterpret_cast<const uint4*>(xod + 8 * p.pitch4 + 64 * s);
-                        }
-                        ye[0] = e2.x; ye[1] = e2.y; ye[2] = e2.z; ye[3] = e2.w;
-                        yo[0] = o2.x; yo[1] = o2.y; yo[2] = o2.z; yo[3] = o2.w;
-                    } else {
-                        const uint4 x = *reinterpret_cast<const uint4*>(xa + 64 * s);
-                        uint4 y = make_uint4(0, 0, 0, 0);
-                        if (TT == 2) y = *reinterpret_cast<const uint4*>(xa + 8 * p.pitch4 + 64 * s);
-                        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            if (ASYM) {
-                                xe[j] = xs[j] & kLo; xo[j] = (xs[j] >> 4) & kLo;
-                                ye[j] = ys[j] & kLo; yo[j] = (ys[j] >> 4) & kLo;
-                            } else {
-                                xe[j] = (xs[j] << 4) & kHi; xo[j] = xs[j] & kHi;
-                                ye[j] = (ys[j] << 4) & kHi; yo[j] = ys[j] & kHi;
-                            }
-                        }
-                    }
                     const uint4 wa = *reinterpret_cast<const uint4*>(w0 + 64 * s);
                     const uint4 wb = *reinterpret_cast<const uint4*>(w1 + 64 * s);
-                    const uint32_t was[4] = {wa.x, wa.y, wa.z, wa.w}, wbs[4] = {wb.x, wb.y, wb.z, wb.w};
+                    // odd codes times 16 / even codes plus 8 of the two units' rows: the A fragments of two products
+                    const uint32_t ao[8] = {wa.x & kHi, wb.x & kHi, wa.y & kHi, wb.y & kHi, wa.z & kHi, wb.z & kHi, wa.w & kHi, wb.w & kHi};
+                    const uint32_t ae[8] = {even_codes(wa.x), even_codes(wb.x), even_codes(wa.y), even_codes(wb.y),
+                                            even_codes(wa.z), even_codes(wb.z), even_codes(wa.w), even_codes(wb.w)};
 #pragma unroll
-                    for (int j = 0; j < 4; j += 2) {
-                        mma_s8<ASYM>(accO[0], xo[j], yo[j], xo[j + 1], yo[j + 1], was[j] & kHi, was[j + 1] & kHi);
-                        mma_s8<ASYM>(accE[0], xe[j], ye[j], xe[j + 1], ye[j + 1], even_codes(was[j]), even_codes(was[j + 1]));
-                        mma_s8<ASYM>(accO[1], xo[j], yo[j], xo[j + 1], yo[j + 1], wbs[j] & kHi, wbs[j + 1] & kHi);
-                        mma_s8<ASYM>(accE[1], xe[j], ye[j], xe[j + 1], ye[j + 1], even_codes(wbs[j]), even_codes(wbs[j + 1]));
+                    for (int tt = 0; tt < TT; ++tt) {
+                        const uint8_t* row = tt == 0 ? a4row : b4row;
+                        uint32_t xe[4], xo[4];
+                        if (kSplit) {
+                            const uint4 e = *reinterpret_cast<const uint4*>(row + co + 64 * s);
+                            const uint4 o = *reinterpret_cast<const uint4*>(row + odd_ofs + co + 64 * s);
+                            xe[0] = e.x; xe[1] = e.y; xe[2] = e.z; xe[3] = e.w;
+                            xo[0] = o.x; xo[1] = o.y; xo[2] = o.z; xo[3] = o.w;
+                        } else {
+                            const uint4 x = *reinterpret_cast<const uint4*>(row + co + 64 * s);
+                            const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                if (ASYM) { xe[j] = xs[j] & kLo; xo[j] = (xs[j] >> 4) & kLo; }
+                                else { xe[j] = (xs[j] << 4) & kHi; xo[j] = xs[j] & kHi; }
+                            }
+                        }
+                        mma_s8<ASYM>(accO[tt], ao[0], ao[1], ao[2], ao[3], xo[0], xo[1]);
+                        mma_s8<ASYM>(accE[tt], ae[0], ae[1], ae[2], ae[3], xe[0], xe[1]);
+                        mma_s8<ASYM>(accO[tt], ao[4], ao[5], ao[6], ao[7], xo[2], xo[3]);
+                        mma_s8<ASYM>(accE[tt], ae[4], ae[5], ae[6], ae[7], xe[2], xe[3]);
                     }
                 }
             }
@@ -408,19 +510,20 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             if (lane == 0 && is_idx < ce) {
                 ++issued;
                 issue(stage);  // refill the stage just read
+                if (!next_done && is_idx >= ce) prefetch_next();
             }
             if (++stage == p.nstages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
 
         // This warp's sums of the segment: acc8 and acc4 + 8 * S_even's share (every shift exact).
-        int part[2][2][4];
+        int part[TT][2][4];
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
+        for (int tt = 0; tt < TT; ++tt)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                part[h][0][i] = acc8[h][i];
-                part[h][1][i] = ASYM ? (accO[h][i] >> 4) + accE[h][i] : (accO[h][i] >> 8) + (accE[h][i] >> 4);
+                part[tt][0][i] = acc8[tt][i];
+                part[tt][1][i] = ASYM ? (accO[tt][i] >> 4) + accE[tt][i] : (accO[tt][i] >> 8) + (accE[tt][i] >> 4);
             }
         const int item_begin = item * nchunks, item_end = item_begin + nchunks;
         bool finish = true;
@@ -428,7 +531,7 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             // Shared item: its slot belongs to the first warp whose run touches it.
             int first = kWarps, touching = 0;
             for (int w = 0; w < kWarps; ++w) {
-                const int b = run_begin(w), e = run_begin(w + 1);
+                const int b = linear(tab[w]), e = linear(tab[w + 1]);
                 if (b < e && b < item_end && e > item_begin) {
                     if (first == kWarps) first = w;
                     ++touching;
@@ -436,11 +539,11 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             }
             int* slot = slots + first * kSlotInts + lane * 4;
 #pragma unroll
-            for (int h = 0; h < 2; ++h)
+            for (int tt = 0; tt < TT; ++tt)
 #pragma unroll
                 for (int a = 0; a < 2; ++a)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) atomicAdd(slot + (h * 2 + a) * 128 + i, part[h][a][i]);
+                    for (int i = 0; i < 4; ++i) atomicAdd(slot + (tt * 2 + a) * 128 + i, part[tt][a][i]);
             __threadfence_block();
             __syncwarp();
             int prev = 0;
@@ -451,44 +554,39 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                 __threadfence_block();
                 const volatile int* vs = slot;
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
+                for (int tt = 0; tt < TT; ++tt)
 #pragma unroll
                     for (int a = 0; a < 2; ++a)
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) part[h][a][i] = vs[(h * 2 + a) * 128 + i];
+                        for (int i = 0; i < 4; ++i) part[tt][a][i] = vs[(tt * 2 + a) * 128 + i];
             }
         }
         if (finish) {
-            // Epilogue on the fragment this thread holds: element i of half h is token g + 8 * (i >> 1),
-            // channel n0 + 8 * h + (i & 1).
+            // Epilogue on the fragment this thread holds.
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 if (h >= halves) break;
+                const float sw8h = scale_value(rw8[h], p.w_fp16), sw4h = scale_value(rw4[h], p.w_fp16);
+                const int n = n0 + 8 * h;
 #pragma unroll
-                for (int tr = 0; tr < TT; ++tr) {
-                    const int t = g + 8 * tr;
-                    if (t >= p.T) continue;
-                    const float sx8 = tr ? sx8b : sx8a, sx4 = tr ? sx4b : sx4a;
-                    const int sev = 8 * (tr ? sev_b : sev_a);
-                    const int a8x = part[h][0][2 * tr], a8y = part[h][0][2 * tr + 1];
-                    const int a4x = part[h][1][2 * tr] - sev, a4y = part[h][1][2 * tr + 1] - sev;
-                    float yx = static_cast<float>(a8x) * (sx8 * sw8[h].x) + static_cast<float>(a4x) * (sx4 * sw4[h].x);
-                    float yy = static_cast<float>(a8y) * (sx8 * sw8[h].y) + static_cast<float>(a4y) * (sx4 * sw4[h].y);
-                    if (ASYM) {
-                        const float zx8 = tr ? zx8b : zx8a, zx4 = tr ? zx4b : zx4a;
-                        yx += zx8 * (static_cast<float>(ws8[h].x) * sw8[h].x) + zx4 * (static_cast<float>(ws4[h].x) * sw4[h].x);
-                        yy += zx8 * (static_cast<float>(ws8[h].y) * sw8[h].y) + zx4 * (static_cast<float>(ws4[h].y) * sw4[h].y);
+                for (int tt = 0; tt < TT; ++tt)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int t = 8 * tt + 2 * tig + e;
+                        if (t >= p.T) continue;
+                        const int a8v = part[tt][0][2 * h + e];
+                        const int a4v = part[tt][1][2 * h + e] - 8 * sevt[tt][e];
+                        float y = static_cast<float>(a8v) * (sx8t[tt][e] * sw8h) + static_cast<float>(a4v) * (sx4t[tt][e] * sw4h);
+                        if (ASYM)
+                            y += zx8t[tt][e] * (static_cast<float>(ws8[h]) * sw8h) + zx4t[tt][e] * (static_cast<float>(ws4[h]) * sw4h);
+                        const size_t o = static_cast<size_t>(t) * p.N + n;
+                        if (p.y_dtype == RESQ_Y_BF16) reinterpret_cast<__nv_bfloat16*>(p.Y)[o] = __float2bfloat16_rn(y);
+                        else reinterpret_cast<float*>(p.Y)[o] = y;
+                        if (p.dbg8) {
+                            p.dbg8[o] = a8v;
+                            p.dbg4[o] = a4v;
+                        }
                     }
-                    const size_t o = static_cast<size_t>(t) * p.N + n0 + 8 * h;
-                    if (p.y_dtype == RESQ_Y_BF16)
-                        *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(p.Y) + o) = __floats2bfloat162_rn(yx, yy);
-                    else
-                        *reinterpret_cast<float2*>(reinterpret_cast<float*>(p.Y) + o) = make_float2(yx, yy);
-                    if (p.dbg8) {
-                        *reinterpret_cast<int2*>(p.dbg8 + o) = make_int2(a8x, a8y);
-                        *reinterpret_cast<int2*>(p.dbg4 + o) = make_int2(a4x, a4y);
-                    }
-                }
             }
         }
         c = 0;
@@ -514,14 +612,15 @@ typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void
                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// [rows][row_bytes] matrix seen as 32-bit elements; box = chunk_bytes x 16 rows, dense in shared
-// memory (no swizzle), zero fill out of range.
-bool make_map_rows(CUtensorMap* m, const void* base, uint64_t rows, uint64_t row_bytes, uint32_t chunk_bytes) {
+// [rows][row_bytes] matrix seen as 32-bit elements; box = chunk_bytes x box_rows rows (16 for an item, 8 for a
+// single unit), dense in shared memory (no swizzle), zero fill out of range.
+bool make_map_rows(CUtensorMap* m, const void* base, uint64_t rows, uint64_t row_bytes, uint32_t chunk_bytes,
+                   uint32_t box_rows = kItemRows) {
     EncodeFn enc = reinterpret_cast<EncodeFn>(tensor_map_encode_fn());
     if (!enc) return false;
     cuuint64_t dims[2] = {row_bytes / 4, rows};
     cuuint64_t strides[1] = {row_bytes};
-    cuuint32_t box[2] = {chunk_bytes / 4, static_cast<cuuint32_t>(kItemRows)};
+    cuuint32_t box[2] = {chunk_bytes / 4, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -529,8 +628,7 @@ bool make_map_rows(CUtensorMap* m, const void* base, uint64_t rows, uint64_t row
 }
 
 template <int TT, int CS, bool SPLIT, bool ASYM>
-cudaError_t launch_variant(const CUtensorMap& t8, const CUtensorMap& t4, const Params& p, int grid, size_t smem,
-                           cudaStream_t st) {
+cudaError_t launch_variant(const CUtensorMap (&tm)[6], const Params& p, int grid, size_t smem, cudaStream_t st) {
     auto kern = mixed_gemm_stream_kernel<TT, CS, SPLIT, ASYM>;
     static bool attr_set[64] = {};
     int dev = 0;
@@ -552,13 +650,78 @@ cudaError_t launch_variant(const CUtensorMap& t8, const CUtensorMap& t4, const P
     cfg.attrs = attr;
     cfg.numAttrs = p.early_weights ? 1 : 0;
     count_launch();
-    return cudaLaunchKernelEx(&cfg, kern, t8, t4, p);
+    return cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
+}
+
+// How a launch cuts its work and its shared memory: chunk width, staging form, ring depth, grid.
+struct Plan {
+    int TT, cs, split, nstages, c8, c4, pitch8, pitch4, units, grid;
+    size_t fixed, smem;
+    bool ok;
+};
+
+Plan make_plan(int T, int N, int K, int r, int sms) {
+    Plan pl = {};
+    const int row4 = (K - r) / 2;
+    pl.units = N / kUnitRows;
+    if (pl.units >= (1 << 24)) return pl;  // the kernel's 32-bit unit arithmetic
+    pl.TT = T <= 8 ? 1 : 2;
+    // Configurations in order of preference: split staging of the INT4 activations before packed for T <= 8 and the
+    // reverse above, the larger chunk (5 steps) before the smaller (3 steps); the first that leaves every warp four
+    // stages wins, else the last one tried that leaves two.
+    for (int pass = 0; pass < 2 && !pl.ok; ++pass) {
+        const int need = pass == 0 ? 4 : kMinStages;
+        for (int k = 0; k < 2 && !pl.ok; ++k) {
+            const int sp = pl.TT == 1 ? 1 - k : k;  // measured: split staging pays for T <= 8 only
+            for (int c : {5, 3}) {
+                const int chunk = 64 * c;
+                pl.c8 = (r + chunk - 1) / chunk;
+                pl.c4 = (row4 + chunk - 1) / chunk;
+                pl.pitch8 = round_up(pl.c8 * chunk, 128) + 64;
+                pl.pitch4 = round_up(pl.c4 * chunk, 128) + 64;
+                pl.fixed = static_cast<size_t>(round_up(static_cast<int>(kControlBytes + kSlotBytes + static_cast<size_t>(T + 1) * pl.pitch8 +
+                                                                         static_cast<size_t>(sp ? 2 : 1) * (T + 1) * pl.pitch4), 128));
+                pl.cs = c;
+                pl.split = sp;
+                pl.nstages = pl.fixed < static_cast<size_t>(kSmemLimit)
+                                 ? static_cast<int>((kSmemLimit - pl.fixed) / kWarps / (static_cast<size_t>(kItemRows) * chunk))
+                                 : 0;
+                if (pl.nstages >= need) { pl.ok = true; break; }
+            }
+        }
+    }
+    if (!pl.ok) return pl;
+    if (pl.nstages > kMaxStages) pl.nstages = kMaxStages;
+    pl.smem = pl.fixed + static_cast<size_t>(kWarps) * pl.nstages * kItemRows * 64 * pl.cs;
+    pl.grid = pl.units < sms ? pl.units : sms;
+    return pl;
+}
+
+// Units per CTA (`urem` CTAs, spread evenly over the grid, own one more) and the warps' run boundaries for the two CTA sizes.
+void fill_split(const Plan& pl, int& uq, int& urem, int (&tab)[2][kWarps + 1]) {
+    uq = pl.units / pl.grid;
+    urem = pl.units % pl.grid;
+    for (int k = 0; k < 2; ++k)
+        for (int w = 0; w <= kWarps; ++w) tab[k][w] = run_boundary(w, (uq + 1 - k + 1) >> 1, pl.c8, pl.c4);
 }
 
 }  // namespace
 
 static int g_early_weights = 0;
-void set_decode_early_weights(int on) { g_early_weights = on ? 1 : 0; }
+void set_decode_early_weights(int on) { g_early_weights = on < 0 ? 0 : (on > 2 ? 2 : on); }
+
+// One-shot description of the few-token launch that will follow the next one (resq_decode_prefetch_next).
+static struct NextHint {
+    bool armed;
+    int T, N, K, r;
+    const int8_t* w8;
+    const uint8_t* w4;
+} g_next = {};
+static int g_prefetch_stages = kMaxStages;  // ring stages of the next launch that the current one asks L2 for
+void set_decode_next_weights(int T, int N, int K, int r, const int8_t* w8, const uint8_t* w4) {
+    g_next = NextHint{true, T, N, K, r, w8, w4};
+}
+void set_decode_prefetch_stages(int n) { g_prefetch_stages = n < 0 ? 0 : (n > kMaxStages ? kMaxStages : n); }
 
 // Returns cudaErrorNotSupported (nothing launched) when the staged activations leave no room for the rings.
 cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x8, const uint8_t* x4,
@@ -567,67 +730,62 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
                                      int32_t* dbg8, int32_t* dbg4, cudaStream_t st, const float* z_x8,
                                      const float* z_x4, const int32_t* wsum8, const int32_t* wsum4) {
     const bool asym = z_x8 != nullptr;  // then x8 / x4 hold unsigned codes
+    int dev = 0, sms = 148;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const Plan pl = make_plan(T, N, K, r, sms);
+    if (!pl.ok) return cudaErrorNotSupported;
     Params p;
     p.T = T; p.N = N; p.r = r; p.row4 = (K - r) / 2;
-    p.units = N / kUnitRows;
-    const int TT = T <= 8 ? 1 : 2, TP = 8 * TT;
-    // Configurations in order of preference: split staging of the INT4 activations before packed
-    // for T <= 8 and the reverse above, the
-    // larger chunk (5 steps) before the smaller (3 steps); the first that leaves every warp four
-    // stages wins, else the last one tried that leaves two.
-    int cs = 0, nstages = 0, split = 0;
-    size_t fixed = 0;
-    bool found = false;
-    for (int pass = 0; pass < 2 && !found; ++pass) {
-        const int need = pass == 0 ? 4 : kMinStages;
-        for (int k = 0; k < 2; ++k) {
-            const int sp = TT == 1 ? 1 - k : k;  // measured: split staging pays for T <= 8 only
-            for (int c : {5, 3}) {
-                const int chunk = 64 * c;
-                p.c8 = (r + chunk - 1) / chunk;
-                p.c4 = (p.row4 + chunk - 1) / chunk;
-                p.pitch8 = round_up(p.c8 * chunk, 128) + 64;
-                p.pitch4 = round_up(p.c4 * chunk, 128) + 64;
-                fixed = kControlBytes + kSlotBytes + static_cast<size_t>(TP) * p.pitch8 +
-                        static_cast<size_t>(sp ? 2 : 1) * TP * p.pitch4;
-                cs = c;
-                split = sp;
-                nstages = fixed < static_cast<size_t>(kSmemLimit)
-                              ? static_cast<int>((kSmemLimit - fixed) / kWarps / (static_cast<size_t>(kItemRows) * chunk))
-                              : 0;
-                if (nstages >= need) { found = true; break; }
-            }
-            if (found) break;
-        }
-    }
-    if (!found) return cudaErrorNotSupported;
-    if (nstages > kMaxStages) nstages = kMaxStages;
-    p.nstages = nstages;
+    fill_split(pl, p.uq, p.urem, p.tab);
+    p.c8 = pl.c8; p.c4 = pl.c4; p.pitch8 = pl.pitch8; p.pitch4 = pl.pitch4;
+    p.nstages = pl.nstages;
+    p.ring_ofs = static_cast<int>(pl.fixed);
     p.early_weights = g_early_weights;
     p.x8 = x8; p.x4 = x4; p.s_x8 = s_x8; p.s_x4 = s_x4; p.s_w8 = s_w8; p.s_w4 = s_w4;
     p.w_fp16 = w_scale_fp16 ? 1 : 0;
     p.z_x8 = z_x8; p.z_x4 = z_x4; p.wsum8 = wsum8; p.wsum4 = wsum4;
     p.Y = Y; p.y_dtype = y_dtype; p.dbg8 = dbg8; p.dbg4 = dbg8 ? dbg4 : nullptr;
     p.status = device_status_ptr();
-    const size_t smem = fixed + static_cast<size_t>(kWarps) * nstages * kItemRows * 64 * cs;
 
-    CUtensorMap t8, t4;
-    if (!make_map_rows(&t4, w4, N, p.row4, 64 * cs)) return cudaErrorInvalidValue;
+    // Maps: [0], [1] INT8 / INT4 weights with the 16-row box of an item, [2], [3] the same with the 8-row box of a
+    // single unit, [4], [5] the next launch's weights.
+    CUtensorMap tm[6];
+    CUtensorMap &t8 = tm[0], &t4 = tm[1], &n8 = tm[4], &n4 = tm[5];
+    if (!make_map_rows(&t4, w4, N, p.row4, 64 * pl.cs) || !make_map_rows(&tm[3], w4, N, p.row4, 64 * pl.cs, kUnitRows))
+        return cudaErrorInvalidValue;
     if (r > 0) {
-        if (!make_map_rows(&t8, w8, N, r, 64 * cs)) return cudaErrorInvalidValue;
+        if (!make_map_rows(&t8, w8, N, r, 64 * pl.cs) || !make_map_rows(&tm[2], w8, N, r, 64 * pl.cs, kUnitRows))
+            return cudaErrorInvalidValue;
     } else {
         t8 = t4;  // uniform INT4: no INT8 chunks are ever requested
+        tm[2] = tm[3];
     }
-    int dev = 0, sms = 148;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int grid = p.units < sms ? p.units : sms;
-    const int variant = (TT == 2 ? 4 : 0) + (cs == 5 ? 2 : 0) + split;
+    // The launch after this one, if the caller has described it: its maps and its work split.
+    n8 = t8;
+    n4 = t4;
+    p.nx_stages = 0; p.nx_grid = 0; p.nx_uq = 0; p.nx_urem = 0; p.nx_c8 = 0; p.nx_c4 = 1; p.nx_chunk_words = 16;
+    for (int k = 0; k < 2; ++k)
+        for (int w = 0; w <= kWarps; ++w) p.nx_tab[k][w] = 0;
+    if (g_next.armed) {
+        const NextHint h = g_next;
+        g_next.armed = false;
+        const Plan np = make_plan(h.T, h.N, h.K, h.r, sms);
+        if (np.ok && g_prefetch_stages > 0 && make_map_rows(&n4, h.w4, h.N, (h.K - h.r) / 2, 64 * np.cs) &&
+            (h.r == 0 || make_map_rows(&n8, h.w8, h.N, h.r, 64 * np.cs))) {
+            if (h.r == 0) n8 = n4;
+            p.nx_stages = np.nstages < g_prefetch_stages ? np.nstages : g_prefetch_stages;
+            p.nx_grid = np.grid; p.nx_c8 = np.c8; p.nx_c4 = np.c4;
+            fill_split(np, p.nx_uq, p.nx_urem, p.nx_tab);
+            p.nx_chunk_words = 16 * np.cs;
+        }
+    }
+    const int variant = (pl.TT == 2 ? 4 : 0) + (pl.cs == 5 ? 2 : 0) + pl.split;
 #define RESQ_STREAM_CASE(v, tt, c, sp)                                                               \
     case v:                                                                                          \
-        return asym ? launch_variant<tt, c, sp, true>(t8, t4, p, grid, smem, st)                     \
-                    : launch_variant<tt, c, sp, false>(t8, t4, p, grid, smem, st);
+        return asym ? launch_variant<tt, c, sp, true>(tm, p, pl.grid, pl.smem, st)       \
+                    : launch_variant<tt, c, sp, false>(tm, p, pl.grid, pl.smem, st);
     switch (variant) {
         RESQ_STREAM_CASE(0, 1, 3, false)
         RESQ_STREAM_CASE(1, 1, 3, true)
@@ -637,8 +795,8 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
         RESQ_STREAM_CASE(5, 2, 3, true)
         RESQ_STREAM_CASE(6, 2, 5, false)
         default:
-            return asym ? launch_variant<2, 5, true, true>(t8, t4, p, grid, smem, st)
-                        : launch_variant<2, 5, true, false>(t8, t4, p, grid, smem, st);
+            return asym ? launch_variant<2, 5, true, true>(tm, p, pl.grid, pl.smem, st)
+                        : launch_variant<2, 5, true, false>(tm, p, pl.grid, pl.smem, st);
     }
 #undef RESQ_STREAM_CASE
 }
