@@ -252,20 +252,6 @@ int resq_project_quantize_static(const void* X, const void* P, int T, int K, int
                                  float* s_x8, float* s_x4, int8_t* x4_i8, void* stream);
 
 /*
- * Generation is memory-bound (paper, Introduction): a step streams every packed weight once, and between two
- * few-token launches HBM would idle while one kernel drains and the next one ramps up.  This call describes the
- * few-token layer that will run AFTER the next one: the next resq_mixed_gemm / resq_linear call of this process
- * with T <= 16 then, once each of its warps has requested the last of its own weights, asks L2 for the first
- * bytes that the described launch will read (its first ring of copies: up to ~190 KB per SM, 28 MB in all), so
- * that HBM keeps streaming across the boundary and the described launch starts on L2 hits.  A hint only: results
- * never depend on it, nothing is written, and the described weights need not be used in the end (the lines are
- * then simply evicted).  next_W / next_desc describe packed weights as written by resq_pack_weights (w8, w4
- * used; both must stay valid until the hinted launch has run); next_T is the token count of that later launch
- * (1..16).  One-shot host state, consumed by the next few-token launch; not thread-safe.
- */
-int resq_decode_prefetch_next(const resq_layer_desc_t* next_desc, const resq_weights_t* next_W, int next_T);
-
-/*
  * Process-wide options (host state of the library; not thread-safe against concurrent calls).
  *  RESQ_OPT_DECODE_EARLY_WEIGHTS (default 0): when 1, the few-token kernel (T <= 16) is launched so
  *    that it may begin while the preceding kernel of the stream is still running; it then streams its
@@ -274,14 +260,13 @@ int resq_decode_prefetch_next(const resq_layer_desc_t* next_desc, const resq_wei
  *    the ramp of each short kernel behind the tail of the previous one.  The caller promises that the
  *    packed weights and their scales were complete before the preceding kernel was enqueued (true
  *    for weights packed at load time; false if resq_pack_weights is the preceding kernel).
- *  RESQ_OPT_DECODE_PREFETCH_STAGES (default 8): how much resq_decode_prefetch_next asks for, in ring stages of
- *    the described launch per warp (one stage = 16 weight rows x 192 or 320 bytes); 0 turns the prefetch off.
  *  RESQ_OPT_WAIT_LIMIT_US (default 2 000 000): wall-clock limit, in microseconds, of a single wait inside a
  *    kernel (for a copy to land, for a pipeline stage to be released).  Stored on the CURRENT device with a
- *    blocking copy; kernels enqueued afterwards on that device use it.  value >= 1.
+ *    blocking copy; kernels enqueued afterwards on that device use it.  value >= 1; the kernels look at the
+ *    limit only once a wait has lasted 100 us, so smaller values act as 100.
  * Returns RESQ_ERR_SHAPE for an unknown option or value.
  */
-enum { RESQ_OPT_DECODE_EARLY_WEIGHTS = 1, RESQ_OPT_WAIT_LIMIT_US = 2, RESQ_OPT_DECODE_PREFETCH_STAGES = 3 };
+enum { RESQ_OPT_DECODE_EARLY_WEIGHTS = 1, RESQ_OPT_WAIT_LIMIT_US = 2 };
 int resq_set_option(int option, int value);
 
 /* Inverse of the INT4 packing, for inspection: packed [rows][cols/2] -> int8 [rows][cols]. */

@@ -17,13 +17,13 @@ LIB_PATH = os.path.join(_HERE, "libresq.so")
 
 OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT, ERR_INDEX = range(9)
 SCALE_FP32, SCALE_FP16 = 0, 1
-OPT_DECODE_EARLY_WEIGHTS, OPT_WAIT_LIMIT_US, OPT_DECODE_PREFETCH_STAGES = 1, 2, 3
+OPT_DECODE_EARLY_WEIGHTS, OPT_WAIT_LIMIT_US = 1, 2
 Y_BF16, Y_FP32 = 0, 1
 
 EXPORTS = [
     "resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_bytes", "resq_workspace_bytes",
     "resq_pack_weights", "resq_pack_weights_projected", "resq_pack_projected_workspace_bytes", "resq_project", "resq_project_workspace_bytes", "resq_hadamard_quantize", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
-    "resq_unpack_int4", "resq_set_option", "resq_decode_prefetch_next",
+    "resq_unpack_int4", "resq_set_option",
     "resq_weight_row_sums", "resq_project_quantize_asym", "resq_mixed_gemm_asym", "resq_linear_asym",
     "resq_workspace_bytes_asym",
     "resq_device_status", "resq_launch_count", "resq_selftest_wait_runs_out", "resq_status_string", "resq_last_cuda_error",
@@ -81,7 +81,6 @@ lib.resq_linear_asym.argtypes = [_dp, _i, _vp, _vp, ctypes.POINTER(WeightsStruct
 lib.resq_workspace_bytes_asym.restype = _sz
 lib.resq_workspace_bytes_asym.argtypes = [_dp, _i, _i, _i]
 lib.resq_set_option.argtypes = [_i, _i]
-lib.resq_decode_prefetch_next.argtypes = [_dp, ctypes.POINTER(WeightsStruct), _i]
 lib.resq_device_status.argtypes = [_vp]
 lib.resq_selftest_wait_runs_out.argtypes = [_vp]
 lib.resq_launch_count.restype = ctypes.c_ulonglong
@@ -237,13 +236,6 @@ def resq_linear(W: Weights, X, P, Y, workspace):
 def resq_unpack_int4(packed, out):
     rows, half = packed.shape
     _check(lib.resq_unpack_int4(_ptr(packed), _ptr(out), rows, half * 2, _stream()), "resq_unpack_int4")
-
-
-def resq_decode_prefetch_next(W_next: Weights, T_next: int):
-    """Hint: the next few-token launch prefetches into L2 the head of `W_next` (the layer that runs after it)."""
-    ws = W_next.struct()
-    _check(lib.resq_decode_prefetch_next(ctypes.byref(W_next.desc), ctypes.byref(ws), int(T_next)),
-           "resq_decode_prefetch_next")
 
 
 def resq_set_option(option: int, value: int):

@@ -497,11 +497,6 @@ int resq_set_option(int option, int value) {
         set_decode_early_weights(value);
         return RESQ_OK;
     }
-    if (option == RESQ_OPT_DECODE_PREFETCH_STAGES) {
-        if (value < 0) return RESQ_ERR_SHAPE;
-        set_decode_prefetch_stages(value);
-        return RESQ_OK;
-    }
     if (option == RESQ_OPT_WAIT_LIMIT_US) {
         if (value < 1) return RESQ_ERR_SHAPE;
         int* p = device_status_ptr();
@@ -523,14 +518,6 @@ int resq_device_status(void* stream) {
         cudaMemcpy(p, &zero, sizeof(int), cudaMemcpyHostToDevice);
         return (v & kStatusBitTimeout) ? RESQ_ERR_TIMEOUT : RESQ_ERR_INDEX;  // one bit per condition
     }
-    return RESQ_OK;
-}
-
-int resq_decode_prefetch_next(const resq_layer_desc_t* next_desc, const resq_weights_t* next_W, int next_T) {
-    if (int e = check_desc(next_desc)) return e;
-    if (next_T < 1 || next_T > kDecodeMaxT) return RESQ_ERR_SHAPE;
-    if (int e = check_weights(next_W, next_desc->r)) return e;
-    set_decode_next_weights(next_T, next_desc->n_out, next_desc->K, next_desc->r, next_W->w8, next_W->w4);
     return RESQ_OK;
 }
 

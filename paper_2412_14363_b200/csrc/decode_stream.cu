@@ -61,6 +61,7 @@ constexpr uint32_t kHi = 0xF0F0F0F0u, kLo = 0x0F0F0F0Fu, kFlip = 0x08080808u;
 
 struct Params {
     int T, N, r, row4;     // row4 = (K - r) / 2: bytes of a packed INT4 weight row
+    int TR;                // staged activation rows: T, plus a zero row unless the tokens fill their groups of 8
     int c8, c4;            // chunks per row in the INT8 / INT4 segment
     int pitch8, pitch4;    // bytes per token of the staged activations (zero padded to whole chunks)
     int nstages;           // stages per warp
@@ -83,14 +84,10 @@ struct Params {
     int32_t* dbg8;
     int32_t* dbg4;
     int* status;
-    // Head of the NEXT few-token launch's weight stream, prefetched into L2 by this launch (0 stages = off): the
-    // geometry of that launch's work split, so that warp w of CTA b asks for what warp w of CTA b will load first.
-    int nx_stages, nx_grid, nx_uq, nx_urem, nx_c8, nx_c4, nx_chunk_words;
     // Work split: CTA b owns units [b * uq + floor(b * urem / grid), ...): uq or uq + 1 of them; tab[0] / tab[1] hold the warps' run
-    // boundaries (run_boundary) for those two sizes.  nx_tab: the same for the next launch.
+    // boundaries (run_boundary) for those two sizes.
     int uq, urem;
     int tab[2][kWarps + 1];
-    int nx_tab[2][kWarps + 1];
 };
 
 struct __align__(16) Control {
@@ -98,6 +95,7 @@ struct __align__(16) Control {
     int s_even[16];  // per token: sum of the even-position INT4 activation codes
     int arrived[kWarps];  // per slot: warps that have added their part
     int abort_flag;
+    uint64_t act_bar;  // completion of the bulk copies that stage the activation rows (packed staging only)
 };
 static_assert(sizeof(Control) <= kControlBytes, "control block");
 
@@ -139,7 +137,7 @@ __device__ __forceinline__ int small_muldiv(int a, int b, int d) {
 
 // Cost of one chunk in the split of a CTA's work over its warps: an INT4 chunk takes about twice the
 // instructions of an INT8 chunk of the same bytes (two products per packed word plus the nibble logic).
-constexpr int kCost8 = 4, kCost4 = 9;
+constexpr int kCost8 = 4, kCost4 = 7;
 
 // Where the run of warp w begins when the (item, chunk) sequence of a CTA with `items` items is cut into kWarps runs
 // of equal cost, packed as item << 16 | chunk; w = kWarps gives the end of the sequence.  Evaluated on the host
@@ -167,16 +165,15 @@ template <int TT, int CS, bool kSplit, bool ASYM>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_constant__ CUtensorMap tmW4,
                          const __grid_constant__ CUtensorMap tmH8, const __grid_constant__ CUtensorMap tmH4,
-                         const __grid_constant__ CUtensorMap tmN8, const __grid_constant__ CUtensorMap tmN4,
                          const Params p) {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int kChunkBytes = CS * 64;
     constexpr int kStageBytes = kItemRows * kChunkBytes;
     Control* ctl = reinterpret_cast<Control*>(smem);
     int* slots = reinterpret_cast<int*>(smem + kControlBytes);                        // [kWarps][kSlotInts]
-    // Staged activation codes: rows [0, T) are the tokens, row T is all zeros (what the 16-row operand reads for
-    // its rows beyond T).
-    const int TR = p.T + 1;
+    // Staged activation codes: rows [0, T) are the tokens, row T (when T is not a multiple of 8) is all zeros: what
+    // the token operand reads for its columns beyond T.
+    const int TR = p.TR;
     uint8_t* act8 = smem + kControlBytes + kSlotBytes;                                // [T + 1][pitch8]
     uint8_t* act4 = act8 + static_cast<size_t>(TR) * p.pitch8;                        // kSplit: even [T + 1][pitch4], odd [T + 1][pitch4]; else packed [T + 1][pitch4]
     uint8_t* rings = smem + p.ring_ofs;                                               // [kWarps][nstages][16][chunk]
@@ -235,28 +232,6 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         tma_load_2d_hint(ring + static_cast<size_t>(stage) * kStageBytes, tm, &full[stage], x, ub * kUnitRows, stream_policy);
         ++is_idx;
         if (++is_chunk == nchunks) { is_chunk = 0; ++is_item; }
-    };
-
-    // Once this warp has asked for the last of its own weights, it asks L2 for the first ring of the same warp of
-    // the next launch (no shared memory, no barrier involved: the lines simply are in L2 when that launch starts).
-    // HBM then keeps streaming through this launch's drain, the switch of grids and the next launch's ramp.
-    bool next_done = p.nx_stages == 0 || bx >= p.nx_grid;
-    auto prefetch_next = [&]() {
-        next_done = true;
-        const int nu0 = bx * p.nx_uq + small_muldiv(bx, p.nx_urem, p.nx_grid);
-        const int nbig = (bx + 1) * p.nx_uq + small_muldiv(bx + 1, p.nx_urem, p.nx_grid) - nu0 - p.nx_uq;
-        const int nch = p.nx_c8 + p.nx_c4;
-        const int* nt = p.nx_tab[1 - nbig];
-        const int q0 = nt[warp], q1 = nt[warp + 1];
-        int item = q0 >> 16, chunk = q0 & 0xFFFF;
-        const int len = ((q1 >> 16) - item) * nch + (q1 & 0xFFFF) - chunk;
-        const int count = len < p.nx_stages ? len : p.nx_stages;
-        for (int k = 0; k < count; ++k) {
-            const bool seg8 = chunk < p.nx_c8;
-            tma_prefetch_2d(seg8 ? &tmN8 : &tmN4, (seg8 ? chunk : chunk - p.nx_c8) * p.nx_chunk_words,
-                            (nu0 + 2 * item) * kUnitRows);
-            if (++chunk == nch) { chunk = 0; ++item; }
-        }
     };
 
     if (!p.early_weights) griddep_wait();
@@ -351,8 +326,42 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             }
         };
         uint4 va[kBatch], vb[kBatch];
-        load8(0, va);
-        load4(0, vb);
+        if constexpr (kSplit) {
+            load8(0, va);
+            load4(0, vb);
+        } else {
+            // Packed staging needs no arithmetic: one bulk copy per token row and segment, all in flight at once
+            // (16 rows of a 14336-wide layer are 129 KB), issued by the lanes of the last warp; the threads only
+            // write the zeros behind the rows and the zero row.
+            if (warp == kWarps - 1) {
+                if (lane == 0) {
+                    mbar_init(&ctl->act_bar, 1);
+                    fence_mbar_init();
+                    mbar_arrive_expect_tx(&ctl->act_bar, static_cast<uint32_t>(p.T) * static_cast<uint32_t>(p.r + p.row4));
+                }
+                __syncwarp();
+                for (int i = lane; i < 2 * p.T; i += 32) {
+                    const int t = i >> 1;
+                    if ((i & 1) == 0) {
+                        if (p.r > 0) bulk_load(act8 + static_cast<size_t>(t) * p.pitch8, p.x8 + static_cast<size_t>(t) * p.r, p.r, &ctl->act_bar);
+                    } else {
+                        bulk_load(act4 + static_cast<size_t>(t) * p.pitch4, p.x4 + static_cast<size_t>(t) * p.row4, p.row4, &ctl->act_bar);
+                    }
+                }
+            }
+            const int pv8 = v8 - r8, pv = pv8 + v4 - r4;  // vectors behind the data of a row: INT8, both segments
+            const uint4 z = make_uint4(0, 0, 0, 0);
+            for (int i = threadIdx.x; i < p.T * pv; i += kThreads) {
+                const int t = i / pv, o = i - t * pv;
+                if (o < pv8) *reinterpret_cast<uint4*>(act8 + static_cast<size_t>(t) * p.pitch8 + ((r8 + o) << 4)) = z;
+                else *reinterpret_cast<uint4*>(act4 + static_cast<size_t>(t) * p.pitch4 + ((r4 + o - pv8) << 4)) = z;
+            }
+            if (TR > p.T)
+                for (int i = threadIdx.x; i < v8 + v4; i += kThreads) {
+                    if (i < v8) *reinterpret_cast<uint4*>(act8 + static_cast<size_t>(p.T) * p.pitch8 + (i << 4)) = z;
+                    else *reinterpret_cast<uint4*>(act4 + static_cast<size_t>(p.T) * p.pitch4 + ((i - v8) << 4)) = z;
+                }
+        }
         // Sum of the even-position INT4 codes per token, from the global rows (up to four vectors in flight per lane).
         constexpr int kTokIters = (8 * TT + kWarps - 1) / kWarps;
         int se[kTokIters];
@@ -385,17 +394,18 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         if (lane == 0) {
             for (int s = issued; s < first_burst; ++s) issue(s);
             issued = first_burst;
-            if (!next_done && is_idx >= ce) prefetch_next();
         }
-        store8(0, va);
-        store4(0, vb);
-        for (int base = kBatch * kThreads; base < n8; base += kBatch * kThreads) {
-            load8(base, va);
-            store8(base, va);
-        }
-        for (int base = kBatch * kThreads; base < n4; base += kBatch * kThreads) {
-            load4(base, vb);
-            store4(base, vb);
+        if constexpr (kSplit) {
+            store8(0, va);
+            store4(0, vb);
+            for (int base = kBatch * kThreads; base < n8; base += kBatch * kThreads) {
+                load8(base, va);
+                store8(base, va);
+            }
+            for (int base = kBatch * kThreads; base < n4; base += kBatch * kThreads) {
+                load4(base, vb);
+                store4(base, vb);
+            }
         }
 #pragma unroll
         for (int tt = 0; tt < kTokIters; ++tt) {
@@ -406,6 +416,8 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         }
     }
     __syncthreads();
+    bool ok = true;
+    if constexpr (!kSplit) ok = mbar_wait(&ctl->act_bar, 0, abort_flag, p.status);  // the staged rows have landed
     int sevt[TT][2];
 #pragma unroll
     for (int tt = 0; tt < TT; ++tt)
@@ -421,7 +433,6 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
 
     int stage = 0;
     uint32_t phase = 0;
-    bool ok = true;
     int consumed = 0;
     int idx = cb, item = pb >> 16, c = pb & 0xFFFF;
     while (idx < ce && ok) {
@@ -445,11 +456,16 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         }
         // Sums of this warp's part of the item: element i of group tt is unit i >> 1 (channel n0 + 8 (i >> 1)),
         // token 8 tt + 2 tig + (i & 1).
-        int acc8[TT][4], accO[TT][4], accE[TT][4];
+        // With one token group a step issues two products per accumulator, each waiting for the one before: the two
+        // halves of a step then go to accumulators of their own (kAcc = 2), which halves the dependent chain.
+        constexpr int kAcc = TT == 1 ? 2 : 1;
+        int acc8[TT][kAcc][4], accO[TT][kAcc][4], accE[TT][kAcc][4];
 #pragma unroll
         for (int tt = 0; tt < TT; ++tt)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc8[tt][i] = accO[tt][i] = accE[tt][i] = 0;
+            for (int a = 0; a < kAcc; ++a)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc8[tt][a][i] = accO[tt][a][i] = accE[tt][a][i] = 0;
 
         for (; c < nchunks && idx < ce; ++c, ++idx) {
             if (!mbar_wait(&full[stage], phase, abort_flag, p.status)) { ok = false; break; }
@@ -462,12 +478,12 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                     const uint4 wa = *reinterpret_cast<const uint4*>(w0 + 64 * s);
                     const uint4 wb = *reinterpret_cast<const uint4*>(w1 + 64 * s);
                     const uint4 x = *reinterpret_cast<const uint4*>(a8row + co + 64 * s);
-                    mma_s8<ASYM>(acc8[0], wa.x, wb.x, wa.y, wb.y, x.x, x.y);
-                    mma_s8<ASYM>(acc8[0], wa.z, wb.z, wa.w, wb.w, x.z, x.w);
+                    mma_s8<ASYM>(acc8[0][0], wa.x, wb.x, wa.y, wb.y, x.x, x.y);
+                    mma_s8<ASYM>(acc8[0][kAcc - 1], wa.z, wb.z, wa.w, wb.w, x.z, x.w);
                     if (TT == 2) {
                         const uint4 y = *reinterpret_cast<const uint4*>(b8row + co + 64 * s);
-                        mma_s8<ASYM>(acc8[TT - 1], wa.x, wb.x, wa.y, wb.y, y.x, y.y);
-                        mma_s8<ASYM>(acc8[TT - 1], wa.z, wb.z, wa.w, wb.w, y.z, y.w);
+                        mma_s8<ASYM>(acc8[TT - 1][0], wa.x, wb.x, wa.y, wb.y, y.x, y.y);
+                        mma_s8<ASYM>(acc8[TT - 1][0], wa.z, wb.z, wa.w, wb.w, y.z, y.w);
                     }
                 }
             } else {
@@ -498,10 +514,10 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
                                 else { xe[j] = (xs[j] << 4) & kHi; xo[j] = xs[j] & kHi; }
                             }
                         }
-                        mma_s8<ASYM>(accO[tt], ao[0], ao[1], ao[2], ao[3], xo[0], xo[1]);
-                        mma_s8<ASYM>(accE[tt], ae[0], ae[1], ae[2], ae[3], xe[0], xe[1]);
-                        mma_s8<ASYM>(accO[tt], ao[4], ao[5], ao[6], ao[7], xo[2], xo[3]);
-                        mma_s8<ASYM>(accE[tt], ae[4], ae[5], ae[6], ae[7], xe[2], xe[3]);
+                        mma_s8<ASYM>(accO[tt][0], ao[0], ao[1], ao[2], ao[3], xo[0], xo[1]);
+                        mma_s8<ASYM>(accE[tt][0], ae[0], ae[1], ae[2], ae[3], xe[0], xe[1]);
+                        mma_s8<ASYM>(accO[tt][kAcc - 1], ao[4], ao[5], ao[6], ao[7], xo[2], xo[3]);
+                        mma_s8<ASYM>(accE[tt][kAcc - 1], ae[4], ae[5], ae[6], ae[7], xe[2], xe[3]);
                     }
                 }
             }
@@ -510,7 +526,6 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             if (lane == 0 && is_idx < ce) {
                 ++issued;
                 issue(stage);  // refill the stage just read
-                if (!next_done && is_idx >= ce) prefetch_next();
             }
             if (++stage == p.nstages) { stage = 0; phase ^= 1; }
         }
@@ -522,8 +537,11 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
         for (int tt = 0; tt < TT; ++tt)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                part[tt][0][i] = acc8[tt][i];
-                part[tt][1][i] = ASYM ? (accO[tt][i] >> 4) + accE[tt][i] : (accO[tt][i] >> 8) + (accE[tt][i] >> 4);
+                const int s8 = acc8[tt][0][i] + (kAcc == 2 ? acc8[tt][kAcc - 1][i] : 0);
+                const int sO = accO[tt][0][i] + (kAcc == 2 ? accO[tt][kAcc - 1][i] : 0);
+                const int sE = accE[tt][0][i] + (kAcc == 2 ? accE[tt][kAcc - 1][i] : 0);
+                part[tt][0][i] = s8;
+                part[tt][1][i] = ASYM ? (sO >> 4) + sE : (sO >> 8) + (sE >> 4);
             }
         const int item_begin = item * nchunks, item_end = item_begin + nchunks;
         bool finish = true;
@@ -602,6 +620,10 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             if (++stage == p.nstages) { stage = 0; phase ^= 1; }
         }
     }
+    if (!kSplit && !ok && threadIdx.x == kThreads - 32) {
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(&ctl->act_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+    }
     __syncthreads();
     if (threadIdx.x == 0 && ctl->abort_flag) atomicOr(p.status, kStatusBitTimeout);
 }
@@ -628,7 +650,7 @@ bool make_map_rows(CUtensorMap* m, const void* base, uint64_t rows, uint64_t row
 }
 
 template <int TT, int CS, bool SPLIT, bool ASYM>
-cudaError_t launch_variant(const CUtensorMap (&tm)[6], const Params& p, int grid, size_t smem, cudaStream_t st) {
+cudaError_t launch_variant(const CUtensorMap (&tm)[4], const Params& p, int grid, size_t smem, cudaStream_t st) {
     auto kern = mixed_gemm_stream_kernel<TT, CS, SPLIT, ASYM>;
     static bool attr_set[64] = {};
     int dev = 0;
@@ -650,12 +672,12 @@ cudaError_t launch_variant(const CUtensorMap (&tm)[6], const Params& p, int grid
     cfg.attrs = attr;
     cfg.numAttrs = p.early_weights ? 1 : 0;
     count_launch();
-    return cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
+    return cudaLaunchKernelEx(&cfg, kern, tm[0], tm[1], tm[2], tm[3], p);
 }
 
 // How a launch cuts its work and its shared memory: chunk width, staging form, ring depth, grid.
 struct Plan {
-    int TT, cs, split, nstages, c8, c4, pitch8, pitch4, units, grid;
+    int TT, TR, cs, split, nstages, c8, c4, pitch8, pitch4, units, grid;
     size_t fixed, smem;
     bool ok;
 };
@@ -666,6 +688,7 @@ Plan make_plan(int T, int N, int K, int r, int sms) {
     pl.units = N / kUnitRows;
     if (pl.units >= (1 << 24)) return pl;  // the kernel's 32-bit unit arithmetic
     pl.TT = T <= 8 ? 1 : 2;
+    pl.TR = T % 8 == 0 ? T : T + 1;  // a zero row for the token columns beyond T
     // Configurations in order of preference: split staging of the INT4 activations before packed for T <= 8 and the
     // reverse above, the larger chunk (5 steps) before the smaller (3 steps); the first that leaves every warp four
     // stages wins, else the last one tried that leaves two.
@@ -679,8 +702,8 @@ Plan make_plan(int T, int N, int K, int r, int sms) {
                 pl.c4 = (row4 + chunk - 1) / chunk;
                 pl.pitch8 = round_up(pl.c8 * chunk, 128) + 64;
                 pl.pitch4 = round_up(pl.c4 * chunk, 128) + 64;
-                pl.fixed = static_cast<size_t>(round_up(static_cast<int>(kControlBytes + kSlotBytes + static_cast<size_t>(T + 1) * pl.pitch8 +
-                                                                         static_cast<size_t>(sp ? 2 : 1) * (T + 1) * pl.pitch4), 128));
+                pl.fixed = static_cast<size_t>(round_up(static_cast<int>(kControlBytes + kSlotBytes + static_cast<size_t>(pl.TR) * pl.pitch8 +
+                                                                         static_cast<size_t>(sp ? 2 : 1) * pl.TR * pl.pitch4), 128));
                 pl.cs = c;
                 pl.split = sp;
                 pl.nstages = pl.fixed < static_cast<size_t>(kSmemLimit)
@@ -710,19 +733,6 @@ void fill_split(const Plan& pl, int& uq, int& urem, int (&tab)[2][kWarps + 1]) {
 static int g_early_weights = 0;
 void set_decode_early_weights(int on) { g_early_weights = on < 0 ? 0 : (on > 2 ? 2 : on); }
 
-// One-shot description of the few-token launch that will follow the next one (resq_decode_prefetch_next).
-static struct NextHint {
-    bool armed;
-    int T, N, K, r;
-    const int8_t* w8;
-    const uint8_t* w4;
-} g_next = {};
-static int g_prefetch_stages = kMaxStages;  // ring stages of the next launch that the current one asks L2 for
-void set_decode_next_weights(int T, int N, int K, int r, const int8_t* w8, const uint8_t* w4) {
-    g_next = NextHint{true, T, N, K, r, w8, w4};
-}
-void set_decode_prefetch_stages(int n) { g_prefetch_stages = n < 0 ? 0 : (n > kMaxStages ? kMaxStages : n); }
-
 // Returns cudaErrorNotSupported (nothing launched) when the staged activations leave no room for the rings.
 cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x8, const uint8_t* x4,
                                      const float* s_x8, const float* s_x4, const int8_t* w8, const uint8_t* w4,
@@ -738,6 +748,7 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
     if (!pl.ok) return cudaErrorNotSupported;
     Params p;
     p.T = T; p.N = N; p.r = r; p.row4 = (K - r) / 2;
+    p.TR = pl.TR;
     fill_split(pl, p.uq, p.urem, p.tab);
     p.c8 = pl.c8; p.c4 = pl.c4; p.pitch8 = pl.pitch8; p.pitch4 = pl.pitch4;
     p.nstages = pl.nstages;
@@ -750,9 +761,9 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
     p.status = device_status_ptr();
 
     // Maps: [0], [1] INT8 / INT4 weights with the 16-row box of an item, [2], [3] the same with the 8-row box of a
-    // single unit, [4], [5] the next launch's weights.
-    CUtensorMap tm[6];
-    CUtensorMap &t8 = tm[0], &t4 = tm[1], &n8 = tm[4], &n4 = tm[5];
+    // single unit.
+    CUtensorMap tm[4];
+    CUtensorMap &t8 = tm[0], &t4 = tm[1];
     if (!make_map_rows(&t4, w4, N, p.row4, 64 * pl.cs) || !make_map_rows(&tm[3], w4, N, p.row4, 64 * pl.cs, kUnitRows))
         return cudaErrorInvalidValue;
     if (r > 0) {
@@ -761,25 +772,6 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
     } else {
         t8 = t4;  // uniform INT4: no INT8 chunks are ever requested
         tm[2] = tm[3];
-    }
-    // The launch after this one, if the caller has described it: its maps and its work split.
-    n8 = t8;
-    n4 = t4;
-    p.nx_stages = 0; p.nx_grid = 0; p.nx_uq = 0; p.nx_urem = 0; p.nx_c8 = 0; p.nx_c4 = 1; p.nx_chunk_words = 16;
-    for (int k = 0; k < 2; ++k)
-        for (int w = 0; w <= kWarps; ++w) p.nx_tab[k][w] = 0;
-    if (g_next.armed) {
-        const NextHint h = g_next;
-        g_next.armed = false;
-        const Plan np = make_plan(h.T, h.N, h.K, h.r, sms);
-        if (np.ok && g_prefetch_stages > 0 && make_map_rows(&n4, h.w4, h.N, (h.K - h.r) / 2, 64 * np.cs) &&
-            (h.r == 0 || make_map_rows(&n8, h.w8, h.N, h.r, 64 * np.cs))) {
-            if (h.r == 0) n8 = n4;
-            p.nx_stages = np.nstages < g_prefetch_stages ? np.nstages : g_prefetch_stages;
-            p.nx_grid = np.grid; p.nx_c8 = np.c8; p.nx_c4 = np.c4;
-            fill_split(np, p.nx_uq, p.nx_urem, p.nx_tab);
-            p.nx_chunk_words = 16 * np.cs;
-        }
     }
     const int variant = (pl.TT == 2 ? 4 : 0) + (pl.cs == 5 ? 2 : 0) + pl.split;
 #define RESQ_STREAM_CASE(v, tt, c, sp)                                                               \

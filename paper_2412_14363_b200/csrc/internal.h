@@ -66,10 +66,6 @@ cudaError_t launch_mixed_gemm_stream(int T, int N, int K, int r, const int8_t* x
                                      const float* z_x4 = nullptr, const int32_t* wsum8 = nullptr,
                                      const int32_t* wsum4 = nullptr);  // z_x8 != NULL: asymmetric, unsigned codes
 void set_decode_early_weights(int on);
-// One-shot: the NEXT launch_mixed_gemm_stream prefetches into L2 the head of the weight stream of the launch
-// described here (the one that will follow it).  `stages`: ring stages of that launch to ask for (0 = off).
-void set_decode_next_weights(int T, int N, int K, int r, const int8_t* w8, const uint8_t* w4);
-void set_decode_prefetch_stages(int stages);
 
 // Online projection C = X·P (bf16 x bf16 -> fp32) on tcgen05 kind::f16, CTA pairs; writes fp32 C [T][K].
 // scratch (optional, project_split_scratch_bytes() bytes): lets a thinly filled last round of tiles be cut along K.

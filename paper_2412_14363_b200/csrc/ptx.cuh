@@ -60,18 +60,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // this library runs for milliseconds).
 // Waits for the phase with the given parity to complete.  Returns false if the limit ran out or if
 // `abort_flag` (a shared-memory word any role may set) became non-zero.  `status` is the device status block;
-// the limit is read from it only when the first poll has failed.
+// the limit is read from it (a global-memory round trip) only once a wait has lasted 100 us, far longer than any
+// wait of a healthy kernel, so limits below that act as 100 us.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, const int* status) {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t limit = *reinterpret_cast<const volatile unsigned long long*>(status + 2);
     const uint64_t t0 = global_timer_ns();
+    uint64_t limit = 0;
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0xFF) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > limit) {
-                *abort_flag = 1;
-                return false;
+            const uint64_t waited = global_timer_ns() - t0;
+            if (waited > 100000ull) {
+                if (limit == 0) limit = *reinterpret_cast<const volatile unsigned long long*>(status + 2);
+                if (waited > limit) {
+                    *abort_flag = 1;
+                    return false;
+                }
             }
         }
     }
@@ -89,12 +94,6 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* tmap, ui
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(x), "r"(y)
         : "memory");
-}
-// Asks L2 for the lines of a 2-D tile (no destination, no completion to wait for).  x as for tma_load_2d.
-__device__ __forceinline__ void tma_prefetch_2d(const void* tmap, int x, int y) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y)
-                 : "memory");
 }
 // Untiled bulk copy global -> shared, completion counted in bytes on `bar`.  Both addresses must be
 // 16-byte aligned and `bytes` a multiple of 16.
