@@ -44,10 +44,21 @@ __device__ __forceinline__ Chunk<F32> load_chunk(const void* row, int c) {
 
 template <bool F32>
 __device__ __forceinline__ float chunk_absmax(const Chunk<F32>& c) {
-    float m = 0.f;
+    if constexpr (F32) {
+        float m = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(c.get(i)));
-    return m;
+        for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(c.get(i)));
+        return m;
+    } else {
+        // bf16 pairs: clear the signs, then compare as packed bf16 (exact: max selects one of its inputs)
+        __nv_bfloat162 m = __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t a = c.w[i] & 0x7FFF7FFFu;
+            m = __hmax2(m, *reinterpret_cast<const __nv_bfloat162*>(&a));
+        }
+        return fmaxf(__low2float(m), __high2float(m));
+    }
 }
 
 // code = clamp(round-half-even(x / s)); IEEE division, no reciprocal.
@@ -167,15 +178,18 @@ split_quantize_kernel(const void* __restrict__ in, size_t in_row_bytes, size_t r
 // twice from shared memory: once for the two absmax values, once for the codes.
 //
 // Rounding.  The definition is code = round-half-even(fl(x / s)) with an IEEE division.  Here
-// t = fma(x, inv, M) with inv = RN(1 / s) and M = 1.5 * 2^23 rounds the exact product x * inv to the
-// nearest integer (ties to even) in one instruction, and the low byte of t's bit pattern is the
-// two's-complement code.  x * inv and fl(x / s) both lie within 2^-16 of x / s for |x / s| <= 128, so
-// the two roundings can only disagree when x * inv is within 2^-16 of a half-integer; whenever the
-// residual of a chunk comes within 2^-15 of one half, the chunk is redone with the true division.
+// t = fma(x, v, M) with M = 1.5 * 2^23 rounds the exact product x * v to the nearest integer (ties to
+// even) in one instruction, and the low byte of t's bit pattern is the two's-complement code.  It is
+// evaluated for two factors that bracket 1 / s, v_lo = RN(inv (1 - 2^-20)) and v_hi = RN(inv (1 + 2^-20))
+// with inv = RN(1 / s): fl(x / s) lies between x * v_lo and x * v_hi (the division and the reciprocal
+// are each off by at most 2^-24 relative, the bracket is 2^-21 wide at least on either side), rounding to
+// nearest is monotone, so when both products round to the same integer, that integer is the defined code;
+// when they differ (the quotient is within |x / s| * 2^-19 of a half-integer, ties included) the chunk is
+// redone with the true division.
 constexpr int kFastGroupBytes = 32 * 1024;
 constexpr int kFastMaxRowBytes = 200 * 1024;
 constexpr float kMagic = 12582912.f;                    // 1.5 * 2^23
-constexpr float kTieGuard = 0.5f - 0.000030517578125f;  // 1/2 - 2^-15
+constexpr float kBracket = 9.5367431640625e-07f;        // 2^-20
 
 template <bool F32>
 __device__ __forceinline__ Chunk<F32> lds_chunk(const uint8_t* row, int c) {
@@ -194,16 +208,15 @@ __device__ __forceinline__ Chunk<F32> lds_chunk(const uint8_t* row, int c) {
 
 template <bool F32>
 __device__ __forceinline__ void fast_codes(const Chunk<F32>& ch, float s, float inv, bool exact_only, uint32_t (&t)[8]) {
-    float dmax = 0.f;
+    const float v_lo = fmaf(inv, -kBracket, inv), v_hi = fmaf(inv, kBracket, inv);
+    uint32_t differ = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const float x = ch.get(i);
-        const float tf = fmaf(x, inv, kMagic);
-        const float d = fmaf(x, inv, -(tf - kMagic));
-        dmax = fmaxf(dmax, fabsf(d));
-        t[i] = __float_as_uint(tf);
+        t[i] = __float_as_uint(fmaf(x, v_lo, kMagic));
+        differ |= t[i] ^ __float_as_uint(fmaf(x, v_hi, kMagic));
     }
-    if (exact_only || !(dmax < kTieGuard)) {
+    if (exact_only || differ != 0) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) t[i] = __float_as_uint(rintf(__fdiv_rn(ch.get(i), s)) + kMagic);
     }
@@ -259,15 +272,39 @@ split_quantize_fast_kernel(const void* __restrict__ in, size_t in_row_bytes, siz
 
     float a8 = 0.f, a4 = 0.f;
     if (live) {
-        for (int c = j; c < rchunks; c += tpr) a8 = fmaxf(a8, chunk_absmax(lds_chunk<F32>(srow, c)));
-        float m0 = 0.f, m1 = 0.f;  // two chains: the INT4 segment is 7/8 of the row
-        int c = rchunks + j;
-        for (; c + tpr < nchunks; c += 2 * tpr) {
-            m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
-            m1 = fmaxf(m1, chunk_absmax(lds_chunk<F32>(srow, c + tpr)));
+        if constexpr (F32) {
+            for (int c = j; c < rchunks; c += tpr) a8 = fmaxf(a8, chunk_absmax(lds_chunk<F32>(srow, c)));
+            float m0 = 0.f, m1 = 0.f;  // two chains: the INT4 segment is 7/8 of the row
+            int c = rchunks + j;
+            for (; c + tpr < nchunks; c += 2 * tpr) {
+                m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
+                m1 = fmaxf(m1, chunk_absmax(lds_chunk<F32>(srow, c + tpr)));
+            }
+            if (c < nchunks) m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
+            a4 = fmaxf(m0, m1);
+        } else {
+            // bf16 rows: sign bits cleared, maxima kept as packed pairs until the end (two operations per pair)
+            const uint4* v = reinterpret_cast<const uint4*>(srow);
+            uint32_t m8 = 0, m4a = 0, m4b = 0;
+            auto acc = [](uint32_t& m, const uint4 u) {
+                const uint32_t w[4] = {u.x & 0x7FFF7FFFu, u.y & 0x7FFF7FFFu, u.z & 0x7FFF7FFFu, u.w & 0x7FFF7FFFu};
+                __nv_bfloat162 mm = *reinterpret_cast<const __nv_bfloat162*>(&m);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) mm = __hmax2(mm, *reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+                m = *reinterpret_cast<const uint32_t*>(&mm);
+            };
+            for (int c = j; c < rchunks; c += tpr) acc(m8, v[c]);
+            int c = rchunks + j;
+#pragma unroll 2
+            for (; c + tpr < nchunks; c += 2 * tpr) {
+                acc(m4a, v[c]);
+                acc(m4b, v[c + tpr]);
+            }
+            if (c < nchunks) acc(m4a, v[c]);
+            auto unpack = [](uint32_t m) { return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u)); };
+            a8 = unpack(m8);
+            a4 = fmaxf(unpack(m4a), unpack(m4b));
         }
-        if (c < nchunks) m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
-        a4 = fmaxf(m0, m1);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {

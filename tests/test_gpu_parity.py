@@ -275,3 +275,44 @@ def test_linear_d2048_pca_basis_end_to_end(resq):
     # the quantized layer tracks the unquantized product (a sanity bound on the whole chain, not parity)
     ref = c.X.astype(np.float64) @ c.W.astype(np.float64)
     assert np.linalg.norm(host(y32) - ref) / np.linalg.norm(ref) < 0.25
+
+
+@pytest.mark.parametrize("T,K,N,r,fp16", [
+    (1280, 8192, 3840, 1024, False),   # 75 tiles on 74 CTA pairs: one tile in the last round
+    (1250, 8192, 3832, 1024, True),    # the same with ragged rows and columns
+    (1280, 8192, 3840, 6144, False),   # an INT8 segment three times as long as the INT4 one
+    (1280, 8192, 3840, 0, False),      # uniform INT4 over 64 K blocks
+    (2304, 8192, 2304, 1024, False),   # 81 tiles: seven in the last round
+])
+def test_mixed_gemm_long_reduction_thin_last_round(resq, T, K, N, r, fp16):
+    """Reductions of 64 K blocks with a thin last round of the persistent grid (the accumulators reach their
+    largest magnitudes of the parity suite, the ring wraps ten times per tile): both accumulators bit for bit on
+    the rows of the last tiles and on sampled rows elsewhere; two runs agree bit for bit."""
+    C_bits, Wp = synthetic_folded(T, K, N, r, seed_shift=300 + (r // 1024))
+    pw = oracle.pack_weights(Wp, r, scale_fp16=fp16)
+    q8, q4, s8, s4 = oracle.split_quantize(oracle.bf16_bits_to_f32(C_bits), r)
+    desc = resq.layer_desc(K, N, r, resq.SCALE_FP16 if fp16 else resq.SCALE_FP32)
+    sdt = torch.float16 if fp16 else torch.float32
+    W = resq.Weights(desc, dev(pw.q8), dev(pw.w4_packed), dev(pw.s8).to(sdt), dev(pw.s4).to(sdt), dev(pw.q4))
+    ws = resq.alloc_workspace(desc, T, False, True)
+    ws.fill_(0x5A)
+    x8, x4e, sx8, sx4 = dev(q8), dev(q4), dev(s8), dev(s4)
+    outs = []
+    for _ in range(2):
+        y32 = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+        a8 = torch.full((T, N), -1, dtype=torch.int32, device="cuda")
+        a4 = torch.full((T, N), -1, dtype=torch.int32, device="cuda")
+        resq.resq_mixed_gemm(W, x8 if r else None, None, sx8, sx4, y32, ws, a8, a4, x4_i8=x4e)
+        _check_status(resq)
+        outs.append((host(a8), host(a4), host(y32)))
+    for a, b in zip(outs[0], outs[1]):
+        assert (a.view(np.uint32) == b.view(np.uint32)).all()
+    rows = np.unique(np.concatenate([np.arange(max(0, T - 256), T), np.arange(0, T, 97), [255, 256, 1023, 1024]]))
+    rows = rows[rows < T]
+    acc8 = oracle.int_gemm(q8[rows], pw.q8) if r else np.zeros((rows.size, N), np.int32)
+    acc4 = oracle.int_gemm(q4[rows], pw.q4)
+    assert (outs[0][0][rows] == acc8).all()
+    assert (outs[0][1][rows] == acc4).all()
+    y_ref, ybf = oracle.epilogue(acc8, acc4, s8[rows], s4[rows], pw.s8, pw.s4)
+    res = oracle.LayerResult(None, q8[rows], q4[rows], None, s8[rows], s4[rows], acc8, acc4, y_ref, ybf)
+    check_output(res, pw, outs[0][2][rows])
