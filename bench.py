@@ -598,6 +598,16 @@ def kv_leg(resq, torch, dev, peaks, steps, n_seqs=16, seq_len=8192, prefill_T=40
     idsp = torch.zeros(T, dtype=torch.int32, device=dev)
     appp_ms = timed(lambda i: kv.resq_kv_append(caches[i % 2], kp, vp, idsp, pos[:T], wq, s_u), steps)
     qpp_ms = timed(lambda i: kv.resq_query_project(qp, wq, s_u, qp16), steps)
+    # many-query (causal prefill) attention of the last Tp tokens of one full sequence: every row streams its own prefix
+    Tp = min(1024, seq_len)
+    qa16 = torch.empty((Tp, KV_HQ, KV_D), dtype=torch.float16, device=dev)
+    kv.resq_query_project(qp[:Tp], wq, s_u, qa16)
+    oa = torch.empty((Tp, KV_HQ, KV_D), dtype=torch.float32, device=dev)
+    qs = torch.zeros(Tp, dtype=torch.int32, device=dev)
+    ql = torch.arange(seq_len - Tp + 1, seq_len + 1, dtype=torch.int32, device=dev)
+    wsq = torch.empty(int(resq.lib.resq_attention_queries_workspace_bytes(Tp, KV_HQ, KV_HKV, KV_D)), dtype=torch.uint8, device=dev)
+    mq_ms = timed(lambda i: kv.resq_attention_queries(caches[i % 2], qa16, qs, ql, oa, wsq), max(3, steps // 4))
+    mq_blocks = int(((ql + 31) // 32).sum().item()) * KV_HKV
     app_bytes = T * KV_HKV * (2 * 2 * KV_D + 2 * 88)
     qp_bytes = T * KV_HQ * (2 * KV_D + 2 * KV_D)
     st = resq.resq_device_status()
@@ -613,7 +623,11 @@ def kv_leg(resq, torch, dev, peaks, steps, n_seqs=16, seq_len=8192, prefill_T=40
             "prefill_tokens": T, "prefill_kv_append_us": round(appp_ms * 1e3, 2),
             "prefill_kv_append_gbs": round(app_bytes / (appp_ms * 1e-3) / 1e9, 1),
             "prefill_query_project_us": round(qpp_ms * 1e3, 2),
-            "prefill_query_project_gbs": round(qp_bytes / (qpp_ms * 1e-3) / 1e9, 1)}
+            "prefill_query_project_gbs": round(qp_bytes / (qpp_ms * 1e-3) / 1e9, 1),
+            "many_query_attention": {"queries": Tp, "prefix_positions": f"{seq_len - Tp + 1}..{seq_len}",
+                                     "us": round(mq_ms * 1e3, 1),
+                                     "cache_block_reads_gbs": round(mq_blocks * 5632 / (mq_ms * 1e-3) / 1e9, 1),
+                                     "note": "each query row streams its own prefix (L2-resident): batched single-query passes"}}
 
 
 # --------------------------------------------------------------------------------------- our arm

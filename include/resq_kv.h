@@ -105,6 +105,20 @@ size_t resq_attention_workspace_bytes(int n_seqs, int n_q_heads, int n_kv_heads,
 int resq_attention_decode(const resq_kv_cache_t* cache, const void* q16, int n_q_heads, const int32_t* seq_lens,
                           float* out, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Many-query attention over the cache (prefill, chunked prefill, speculative steps; Section 4.3 Eq. 8 with the cache
+ * of Section 5.1): query row i -- q16 half [n_queries][n_q_heads][d_head] -- attends the first q_len[i] positions of
+ * cache sequence q_seq[i] (int32 [n_queries] each); out fp32 [n_queries][n_q_heads][d_head].  Causal attention of
+ * tokens appended at positions p_i is q_len[i] = p_i + 1, after the tokens have been appended.  The arithmetic per
+ * query row is that of resq_attention_decode (same kernels, same tolerance; the fp32 partial sums of a row are merged
+ * in the order its cache blocks fall on the grid's warps): every row streams its own prefix of the cache (from L2
+ * when rows share a sequence), so the cost grows with the sum of the q_len, not with the tile products of a
+ * tensor-core prefill kernel.  An out-of-range q_seq[i] is reported as RESQ_ERR_INDEX by resq_device_status (the row's
+ * output is then unspecified); q_len is clamped like seq_lens.  n_queries >= 1. */
+size_t resq_attention_queries_workspace_bytes(int n_queries, int n_q_heads, int n_kv_heads, int d_head);
+int resq_attention_queries(const resq_kv_cache_t* cache, const void* q16, int n_q_heads, int n_queries,
+                           const int32_t* q_seq, const int32_t* q_len, float* out, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -93,3 +93,27 @@ def attention_decode(q16, K_hat, V_hat, seq_lens, n_q_heads: int, n_kv_heads: in
             p /= p.sum()
             out[b, h] = p @ V
     return out
+
+
+def attention_queries(q16, K_hat, V_hat, q_seq, q_len, n_q_heads: int, n_kv_heads: int):
+    """Many-query attention on the dequantized cache, fp64: query row i attends the first q_len[i] positions of
+    sequence q_seq[i] (causal attention of a token at position p is q_len = p + 1).  The textbook definition, one
+    row at a time: out[i][h] = softmax(q[i][h] K^T / sqrt(d)) V over those positions; an empty prefix gives 0.
+
+    q16 [n][Hq][d]; K_hat / V_hat [B][Hkv][S][d] fp64 (lists of arrays)."""
+    q = np.asarray(q16, np.float64)
+    n, Hq, d = q.shape
+    assert Hq == n_q_heads and Hq % n_kv_heads == 0
+    g = Hq // n_kv_heads
+    out = np.zeros((n, Hq, d), np.float64)
+    for i in range(n):
+        b, L = int(q_seq[i]), int(q_len[i])
+        if L == 0:
+            continue
+        for h in range(Hq):
+            K = K_hat[b][h // g][:L]
+            V = V_hat[b][h // g][:L]
+            sc = (K @ q[i, h]) / np.sqrt(float(d))
+            p = np.exp(sc - sc.max())
+            out[i, h] = (p / p.sum()) @ V
+    return out

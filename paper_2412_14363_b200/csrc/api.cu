@@ -607,6 +607,24 @@ int resq_attention_decode(const resq_kv_cache_t* cache, const void* q16, int n_q
 
 unsigned long long resq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+size_t resq_attention_queries_workspace_bytes(int n_queries, int n_q_heads, int n_kv_heads, int d_head) {
+    return resq_attention_workspace_bytes(n_queries, n_q_heads, n_kv_heads, d_head);
+}
+
+int resq_attention_queries(const resq_kv_cache_t* cache, const void* q16, int n_q_heads, int n_queries,
+                           const int32_t* q_seq, const int32_t* q_len, float* out, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+    if (int e = check_cache(cache)) return e;
+    const size_t need = resq_attention_queries_workspace_bytes(n_queries, n_q_heads, cache->n_kv_heads, cache->d_head);
+    if (need == 0) return RESQ_ERR_SHAPE;
+    if (!q16 || !q_seq || !q_len || !out) return RESQ_ERR_NULL;
+    if (!workspace || workspace_bytes < need) return RESQ_ERR_WORKSPACE;
+    if (!aligned16(q16) || !aligned16(out) || !aligned16(workspace)) return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_attention_decode(*cache, q16, n_q_heads, q_len, out, workspace,
+                                               static_cast<cudaStream_t>(stream), n_queries, q_seq));
+}
+
 const char* resq_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 const char* resq_status_string(int s) {

@@ -80,8 +80,11 @@ cudaError_t launch_qkv_project_append(const resq_kv_cache_t* cache, const void* 
                                       const void* k, const void* v, long long T, const int32_t* seq_ids,
                                       const int32_t* positions, const int8_t* wq, const float* s_u, cudaStream_t st);
 size_t attention_scratch_bytes(int n_seqs, int n_kv_heads);
+// n_rows >= 0 with seq_map: the many-query form -- q16 / out / seq_lens have n_rows rows and row i reads the first
+// seq_lens[i] positions of cache sequence seq_map[i]; scratch: attention_scratch_bytes(n_rows, n_kv_heads).
 cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q16, int n_q_heads, const int32_t* seq_lens,
-                                    float* out, void* scratch, cudaStream_t st);
+                                    float* out, void* scratch, cudaStream_t st, int n_rows = -1,
+                                    const int32_t* seq_map = nullptr);
 
 // Driver entry point for tensor-map encoding (resolved once, without linking libcuda).
 void* tensor_map_encode_fn();

@@ -40,10 +40,12 @@ struct AttnParams {
     const uint8_t* cache;
     const __half* q;
     const int32_t* seq_lens;
+    const int32_t* seq_map;  // NULL: query row b reads cache sequence b; else the cache sequence of query row b
     float* partial;
     float* out;
     int* status;
-    int n_seqs, n_kv_heads, group, capacity;
+    int n_seqs, n_kv_heads, group, capacity;  // n_seqs: query rows (= cache sequences when seq_map is NULL)
+    int n_cache_seqs;
 };
 
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -214,7 +216,14 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attention_decode_kernel(const 
     const int blocks_cap = p.capacity / RESQ_KV_BLOCK;
     auto issue = [&](int stage) {  // lane 0 copies the producer cursor's block; every lane moves the cursor
         if (lane == 0) {
-            const uint8_t* src = p.cache + ((static_cast<long long>(prod.b) * p.n_kv_heads + prod.h) * blocks_cap + prod.blk) * kBlk;
+            int cb = prod.b;
+            if (p.seq_map) {
+                cb = p.seq_map[prod.b];
+                if (cb < 0 || cb >= p.n_cache_seqs) {  // reported by the merge kernel; read a valid block meanwhile
+                    cb = 0;
+                }
+            }
+            const uint8_t* src = p.cache + ((static_cast<long long>(cb) * p.n_kv_heads + prod.h) * blocks_cap + prod.blk) * kBlk;
             mbar_arrive_expect_tx(&full[stage], kBlk);
             bulk_load(ring + stage * kBlk, src, kBlk, &full[stage]);
         }
@@ -484,6 +493,7 @@ __global__ void __launch_bounds__(kD * kMaxGroups) attention_combine_kernel(cons
     for (int i = tid; i < p.n_seqs; i += nthr) {
         const int len = p.seq_lens[i];
         if (blockIdx.x == 0 && (len < 0 || len > p.capacity)) atomicOr(p.status, kStatusBitIndex);
+        if (blockIdx.x == 0 && p.seq_map && (p.seq_map[i] < 0 || p.seq_map[i] >= p.n_cache_seqs)) atomicOr(p.status, kStatusBitIndex);
         const int t = ((len < 0 ? 0 : (len > p.capacity ? p.capacity : len)) + 31) >> 5;
         total += t;
         if (i < b) before += t;
@@ -573,7 +583,8 @@ size_t attention_scratch_bytes(int n_seqs, int n_kv_heads) {
 }
 
 cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q16, int n_q_heads, const int32_t* seq_lens,
-                                    float* out, void* scratch, cudaStream_t st) {
+                                    float* out, void* scratch, cudaStream_t st, int n_rows, const int32_t* seq_map) {
+    if (n_rows < 0) n_rows = cache.n_seqs;  // single-query form: one query row per cache sequence
     static bool configured[64] = {};
     int dev = 0;
     if (cudaError_t e = cudaGetDevice(&dev); e != cudaSuccess) return e;
@@ -591,7 +602,9 @@ cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q1
     p.partial = static_cast<float*>(scratch);
     p.out = out;
     p.status = device_status_ptr();
-    p.n_seqs = cache.n_seqs;
+    p.seq_map = seq_map;
+    p.n_seqs = n_rows;
+    p.n_cache_seqs = cache.n_seqs;
     p.n_kv_heads = cache.n_kv_heads;
     p.group = n_q_heads / cache.n_kv_heads;
     p.capacity = cache.capacity;
@@ -599,9 +612,9 @@ cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q1
     attention_decode_kernel<<<148, kWarps * 32, kSmem, st>>>(p);
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cache.n_seqs * n_q_heads, 1, 1);
+    cfg.gridDim = dim3(n_rows * n_q_heads, 1, 1);
     // few (sequence, head) pairs share the grid's warps: each has many records, so four groups of threads add them
-    const int merge_threads = cache.n_seqs * cache.n_kv_heads <= 64 ? kD * kMaxGroups : kD;
+    const int merge_threads = n_rows * cache.n_kv_heads <= 64 ? kD * kMaxGroups : kD;
     cfg.blockDim = dim3(merge_threads, 1, 1);
     cfg.dynamicSmemBytes = static_cast<size_t>(merge_threads) * (sizeof(long long) + sizeof(float)) + (merge_threads / kD) * kD * sizeof(float);
     cfg.stream = st;

@@ -7,7 +7,8 @@ from . import ERR_CUDA, ERR_INDEX, OK, ResqError, _check, _ptr, _stream, lib  # 
 
 KV_BLOCK, KV_BLOCK_BYTES = 32, 5632
 KV_EXPORTS = ["resq_kv_cache_bytes", "resq_uc_quantize", "resq_query_project", "resq_kv_append", "resq_qkv_project_append",
-              "resq_attention_workspace_bytes", "resq_attention_decode"]
+              "resq_attention_workspace_bytes", "resq_attention_decode", "resq_attention_queries_workspace_bytes",
+              "resq_attention_queries"]
 
 
 class KvCacheStruct(ctypes.Structure):
@@ -26,6 +27,9 @@ lib.resq_qkv_project_append.argtypes = [_cp, _vp, _i, _vp, _vp, _vp, _i64, _vp, 
 lib.resq_attention_workspace_bytes.restype = _sz
 lib.resq_attention_workspace_bytes.argtypes = [_i, _i, _i, _i]
 lib.resq_attention_decode.argtypes = [_cp, _vp, _i, _vp, _vp, _vp, _sz, _vp]
+lib.resq_attention_queries_workspace_bytes.restype = _sz
+lib.resq_attention_queries_workspace_bytes.argtypes = [_i, _i, _i, _i]
+lib.resq_attention_queries.argtypes = [_cp, _vp, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]
 
 
 class KvCache:
@@ -87,3 +91,17 @@ def resq_attention_decode(cache: KvCache, q16, seq_lens, out, workspace):
     """q16 half [n_seqs][n_q_heads][128], seq_lens int32 [n_seqs], out fp32 [n_seqs][n_q_heads][128]."""
     _check(lib.resq_attention_decode(ctypes.byref(cache.c), _ptr(q16), q16.shape[1], _ptr(seq_lens), _ptr(out),
                                      _ptr(workspace), workspace.numel(), _stream()), "resq_attention_decode")
+
+
+def resq_attention_queries(cache: KvCache, q16, q_seq, q_len, out, workspace=None):
+    """q16 half [n_queries][n_q_heads][128]; query row i attends the first q_len[i] positions of cache sequence
+    q_seq[i] (int32 tensors); out fp32 of q16's shape.  Allocates the scratch if none is given."""
+    import torch
+    n, hq = q16.shape[0], q16.shape[1]
+    if workspace is None:
+        nbytes = int(lib.resq_attention_queries_workspace_bytes(n, hq, cache.n_kv_heads, cache.d_head))
+        if nbytes == 0:
+            raise ResqError(2, "resq_attention_queries_workspace_bytes")
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=cache.data.device)
+    _check(lib.resq_attention_queries(ctypes.byref(cache.c), _ptr(q16), hq, n, _ptr(q_seq), _ptr(q_len), _ptr(out),
+                                      _ptr(workspace), workspace.numel(), _stream()), "resq_attention_queries")

@@ -270,3 +270,56 @@ def test_end_to_end_append_then_attend(resq, kv, uc):
     Yq, _, _ = okv.project_int8(q.reshape(-1, D), *okv.quantize_uc(W_C))
     ref = okv.attention_decode(okv.query_fp16(Yq).reshape(B, Hq, D), K_hat, V_hat, [S] * B, Hq, Hkv)
     _assert_close(host(out), ref, vmax, Hq, Hkv)
+
+
+@pytest.mark.parametrize("prefix,Tq,Hq,Hkv", [(0, 37, 8, 2), (50, 70, 4, 4), (3, 200, 32, 8)])
+def test_attention_many_queries_causal(resq, kv, uc, prefix, Tq, Hq, Hkv):
+    """Prefill-shaped attention through the public calls: Tq new tokens of one sequence (after `prefix` cached ones)
+    and a few of another are projected and appended, then every new token attends its own causal prefix of the
+    quantized cache in ONE call.  Against the oracle's many-query definition on the oracle's own codes, within the
+    single-query tolerance; rows with an empty prefix give 0; a bad sequence index is reported."""
+    W_C, wq, s_u = uc
+    S = prefix + Tq
+    cap = ((S + 31) // 32) * 32
+    cache = kv.KvCache(3, Hkv, cap)
+    cache.data.fill_(0xFF)
+    K_hat = [[None] * Hkv for _ in range(3)]
+    V_hat = [[None] * Hkv for _ in range(3)]
+    vmax = np.zeros((3, Hkv))
+    for b, n in ((2, S), (0, 5)):
+        k = synth.head_vectors(n, Hkv, D, stream=800 + b, lead=1.0, scale=1.5)
+        v = synth.head_vectors(n, Hkv, D, stream=810 + b, lead=4.0, shift=0.3)
+        kv.resq_kv_append(cache, bf16_to_dev(synth.f32_to_bf16_bits(k)), bf16_to_dev(synth.f32_to_bf16_bits(v)),
+                          dev(np.full(n, b, np.int32)), dev(np.arange(n, dtype=np.int32)), wq, s_u)
+        hk, hv = _oracle_records(k, v, W_C)
+        dk, dv = okv.kv_dequantize(hk).reshape(n, Hkv, D), okv.kv_dequantize(hv).reshape(n, Hkv, D)
+        for h in range(Hkv):
+            K_hat[b][h], V_hat[b][h], vmax[b, h] = dk[:, h], dv[:, h], np.abs(dv[:, h]).max()
+    # query rows: the Tq new tokens of sequence 2 (causal), three rows of sequence 0, one row with an empty prefix
+    q_seq = np.r_[np.full(Tq, 2), [0, 0, 0], [2]].astype(np.int32)
+    q_len = np.r_[np.arange(prefix + 1, S + 1), [1, 3, 5], [0]].astype(np.int32)
+    n = q_seq.size
+    q = synth.head_vectors(n, Hq, D, stream=820, lead=1.0, scale=1.5)
+    q16 = torch.empty((n, Hq, D), dtype=torch.float16, device="cuda")
+    kv.resq_query_project(bf16_to_dev(synth.f32_to_bf16_bits(q)), wq, s_u, q16)
+    out = torch.full((n, Hq, D), float("nan"), dtype=torch.float32, device="cuda")
+    kv.resq_attention_queries(cache, q16, dev(q_seq), dev(q_len), out)
+    assert resq.resq_device_status() == resq.OK
+    ref = okv.attention_queries(host(q16), K_hat, V_hat, q_seq, q_len, Hq, Hkv)
+    got = host(out)
+    assert np.isfinite(got).all() and (got[-1] == 0).all()
+    g = Hq // Hkv
+    for i in range(n):
+        for h in range(Hq):
+            assert np.abs(got[i, h] - ref[i, h]).max() <= 1e-3 * vmax[q_seq[i], h // g], (i, h)
+    # the last causal row sees the whole sequence: the single-query call on that sequence agrees within tolerance
+    one = torch.empty((3, Hq, D), dtype=torch.float32, device="cuda")
+    q3 = torch.zeros((3, Hq, D), dtype=torch.float16, device="cuda")
+    q3[2] = q16[Tq - 1]
+    kv.resq_attention_decode(cache, q3, dev(np.array([0, 0, S], np.int32)), one, kv.attention_workspace(cache, Hq))
+    assert np.abs(host(one)[2] - got[Tq - 1]).max() <= 2e-3 * vmax[2].max()
+    # an out-of-range sequence index is reported
+    bad = q_seq.copy()
+    bad[0] = 3
+    kv.resq_attention_queries(cache, q16, dev(bad), dev(q_len), out)
+    assert resq.resq_device_status() == kv.ERR_INDEX

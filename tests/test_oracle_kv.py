@@ -160,3 +160,40 @@ def test_mixed_cache_beats_uniform_4bit_on_high_variance_heads():
     uni = kv.attention_decode(q, [[uniform4(Kf)]], [[uniform4(Vf)]], [S], 1, 1)
     e_mixed, e_uni = np.linalg.norm(mixed - exact), np.linalg.norm(uni - exact)
     assert e_mixed < 0.5 * e_uni
+
+
+def test_attention_queries_against_masked_matrix_form_and_special_cases():
+    """Many-query attention pinned by an independent formulation -- causal self-attention written as one masked
+    score matrix per head (mask, row softmax, matrix product) -- and by what the definition fixes: a query of
+    prefix length 1 returns the first value vector, equal keys give the running mean of the values, an empty
+    prefix gives 0, rows may come in any order and may address different sequences."""
+    rng = np.random.default_rng(21)
+    d, Hq, Hkv, S = 16, 4, 2, 9
+    K, V = _cache(rng, 2, Hkv, S, d)
+    q = rng.standard_normal((S, Hq, d)).astype(np.float16)
+    # causal prefill of sequence 1: token at position p attends positions <= p
+    out = kv.attention_queries(q, K, V, np.ones(S, int), np.arange(1, S + 1), Hq, Hkv)
+    for h in range(Hq):
+        sc = q[:, h].astype(np.float64) @ K[1][h // 2].T / math.sqrt(d)           # [S queries][S keys]
+        sc = np.where(np.tril(np.ones((S, S), bool)), sc, -np.inf)
+        w = np.exp(sc - sc.max(1, keepdims=True))
+        ref = (w / w.sum(1, keepdims=True)) @ V[1][h // 2]
+        assert np.abs(out[:, h] - ref).max() < 1e-13
+        assert np.allclose(out[0, h], V[1][h // 2][0], rtol=0, atol=1e-15)         # prefix of one position
+    # a permutation of the rows permutes the outputs; rows of different sequences do not interact
+    perm = rng.permutation(S)
+    seqs = np.r_[np.ones(S, int), np.zeros(3, int)]
+    lens = np.r_[np.arange(1, S + 1)[perm], [0, 4, S]]
+    qq = np.concatenate([q[perm], q[:3]])
+    out2 = kv.attention_queries(qq, K, V, seqs, lens, Hq, Hkv)
+    assert np.array_equal(out2[:S], out[perm])
+    assert (out2[S] == 0).all()                                                    # empty prefix
+    single = kv.attention_decode(q[1:3], K, V, [4, S], Hq, Hkv)                    # the single-query definition
+    assert np.allclose(out2[S + 1], kv.attention_decode(q[1:2], [K[0]], [V[0]], [4], Hq, Hkv)[0], atol=1e-15)
+    assert single.shape == (2, Hq, d)
+    # equal keys: uniform weights over the prefix -> running means of the values
+    for h in range(Hkv):
+        K[1][h][:] = K[1][h][0]
+    out3 = kv.attention_queries(q, K, V, np.ones(S, int), np.arange(1, S + 1), Hq, Hkv)
+    for p in range(S):
+        assert np.allclose(out3[p, 3], V[1][1][:p + 1].mean(0), atol=1e-14)

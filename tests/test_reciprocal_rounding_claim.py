@@ -1,10 +1,12 @@
-"""Host-side check of the claim the fast quantizer kernel rests on.
+"""Host-side checks of the claims the fast quantizer kernels rest on.
 
-The kernel replaces code = rint(fl(x / s)) (the definition, Eq. 1 with round-half-even and an IEEE
-fp32 division) by rint(x * inv) with inv = RN(1 / s), evaluated exactly by a fused multiply-add, and
-falls back to the division whenever x * inv comes within 2^-15 of a half-integer.  Claim: outside that
-guard band both roundings agree for every |x / s| <= 128.  Checked here with exact rationals on random
-and on adversarial near-tie inputs; the defined value comes from the oracle's quantizer.
+Symmetric quantizer: the kernel replaces code = rint(fl(x / s)) (the definition, Eq. 1 with round-half-even and
+an IEEE fp32 division) by the rounding of two exact products, x * v_lo and x * v_hi with
+v_lo = RN(inv (1 - 2^-20)), v_hi = RN(inv (1 + 2^-20)), inv = RN(1 / s), and falls back to the division whenever
+the two roundings differ.  Claim: whenever they agree, they are the defined code, for every |x / s| <= 128.
+Asymmetric quantizer: rint(d * inv) evaluated exactly, with a fallback whenever the product comes within 2^-14
+of a half-integer.  Both are checked here with exact rationals on random and on adversarial near-tie inputs; the
+defined values come from the oracle's quantizers.
 """
 from fractions import Fraction
 
@@ -23,7 +25,14 @@ def _rint_half_even(q: Fraction) -> int:
     return f
 
 
-def test_product_rounding_agrees_outside_guard_band():
+def _f32(q: Fraction) -> np.float32:
+    """Rounds an exact rational that a double holds exactly (at most 53 significant bits) to fp32 once."""
+    d = float(q)
+    assert Fraction(d) == q
+    return np.float32(d)
+
+
+def test_bracketing_products_agree_only_on_the_defined_code():
     rng = np.random.default_rng(3)
     checked = fallbacks = 0
     for qmax in (127, 7):
@@ -31,6 +40,8 @@ def test_product_rounding_agrees_outside_guard_band():
             a = np.float32(np.exp(rng.uniform(-20, 20)))
             s = np.float32(a / np.float32(qmax))
             inv = np.float32(np.float32(1.0) / s)  # numpy's fp32 division is correctly rounded
+            v_lo = _f32(Fraction(float(inv)) * (1 - Fraction(1, 2 ** 20)))   # fma(inv, -2^-20, inv): one rounding
+            v_hi = _f32(Fraction(float(inv)) * (1 + Fraction(1, 2 ** 20)))
             k = rng.integers(-qmax, qmax, 200).astype(np.float32) + np.float32(0.5)
             near = ((k * s).astype(np.float32).view(np.int32) + rng.integers(-4, 5, 200).astype(np.int32)).view(np.float32)
             rand = (rng.uniform(-1, 1, 200) * a).astype(np.float32)
@@ -42,10 +53,10 @@ def test_product_rounding_agrees_outside_guard_band():
             assert s_o == s
             codes = codes[1:]
             for xv, code in zip(x, codes):
-                p = Fraction(float(xv)) * Fraction(float(inv))
-                n = _rint_half_even(p)
-                if abs(p - n) < GUARD:
-                    assert n == int(code), (float(xv), float(s), n, int(code))
+                n_lo = _rint_half_even(Fraction(float(xv)) * Fraction(float(v_lo)))
+                n_hi = _rint_half_even(Fraction(float(xv)) * Fraction(float(v_hi)))
+                if n_lo == n_hi:
+                    assert n_lo == int(code), (float(xv), float(s), n_lo, int(code))
                     checked += 1
                 else:
                     fallbacks += 1
