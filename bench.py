@@ -630,6 +630,55 @@ def kv_leg(resq, torch, dev, peaks, steps, n_seqs=16, seq_len=8192, prefill_T=40
                                      "note": "each query row streams its own prefix (L2-resident): batched single-query passes"}}
 
 
+# --------------------------------------------------------------------------------------- projection GEMM study
+def project_study(resq, torch, dev, peaks, T, launches=60):
+    """The online projection GEMM of the block's down_proj alone, `launches` times back to back, with the SM clock
+    sampled alongside: time per launch, TFLOP/s, and SM cycles per K block of one CTA pair (time x median MHz over
+    the K blocks a pair executes), so that runs at different clocks or widths can be compared."""
+    import synth
+    name, K, N, _ = [l for l in LAYERS if l[3]][0]
+    X = synth.t_activations(T, K, dev, "t4", seed=synth.SEED_ACT)
+    P = synth.t_kron_orthogonal_bf16(K, dev)
+    C = torch.empty((min(T, 4096), K), dtype=torch.float32, device=dev)
+    ws = torch.empty(resq.resq_project_workspace_bytes(), dtype=torch.uint8, device=dev)
+    rows = C.shape[0]
+    Xp = X[:rows].contiguous()
+    for _ in range(3):
+        resq.resq_project(Xp, P, C, ws)
+    torch.cuda.synchronize()
+    gpu_id = str(getattr(torch.cuda.get_device_properties(dev), "uuid", 0))
+    if not gpu_id.startswith("GPU-") and "-" in gpu_id:
+        gpu_id = "GPU-" + gpu_id
+    sampler = ClockSampler(gpu_id)
+    sampler.start()
+    evs = []
+    for _ in range(launches):
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        resq.resq_project(Xp, P, C, ws)
+        b.record()
+        evs.append((a, b))
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = sorted(a.elapsed_time(b) for a, b in evs)
+    med = ms[len(ms) // 2]
+    tiles = ((rows + 255) // 256) * ((K + 255) // 256)
+    kblocks_per_pair = tiles / 74.0 * (K / 64.0)   # 64 bf16 elements (128 bytes) per K block
+    mhz = clocks.get("sm_mhz") or 0.0
+    st = resq.resq_device_status()
+    if st != resq.OK:
+        raise SystemExit(f"device status {st}: {resq.status_string(st)}")
+    return {"layer": f"{name} {K}x{K} P, {rows} token rows", "launches": launches, "ms_median": round(med, 4),
+            "ms_min": round(ms[0], 4), "ms_max": round(ms[-1], 4),
+            "tflops_median": round(2.0 * rows * K * K / (med * 1e-3) / 1e12, 1),
+            "frac_of_bf16_burst": round(2.0 * rows * K * K / (med * 1e-3) / 1e12 / peaks["bf16_burst"], 4),
+            "frac_of_bf16_sustained": round(2.0 * rows * K * K / (med * 1e-3) / 1e12 / peaks["bf16_sustained"], 4),
+            "sm_mhz_median": mhz, "clocks": clocks,
+            "sm_cycles_per_k_block": round(med * 1e-3 * mhz * 1e6 / kblocks_per_pair, 1) if mhz else None,
+            "ideal_cycles_per_k_block": 256.0,   # 256 x 256 x 64 MACs per pair and K block at 8192 dense bf16 MACs per SM-clock
+            "tiles": tiles, "rounds_of_74_pairs": round(tiles / 74.0, 2)}
+
+
 # --------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import numpy as np
@@ -648,6 +697,9 @@ def run_ours(args):
     peaks = load_peaks()
     T = T_PREFILL
 
+    if args.project_study:  # profiling runs: the projection GEMM alone with the clock alongside
+        print(json.dumps({"project_gemm_study": project_study(resq, torch, dev, peaks, T)}))
+        return
     only = [x for x in args.layers.split(",") if x]
     layers = build_layers(dev, only=only)
     for L in layers:
@@ -988,6 +1040,8 @@ def main():
     ap.add_argument("--no-decode", action="store_true", help="skip the few-token leg (profiling runs)")
     ap.add_argument("--decode-only", action="store_true", help="run only the few-token leg (profiling runs)")
     ap.add_argument("--no-kv", action="store_true", help="skip the attention-block leg (profiling runs)")
+    ap.add_argument("--project-study", action="store_true", help="time the projection GEMM alone with SM clocks (profiling runs)")
+    ap.add_argument("--tokens", type=int, default=0, help="override the prefill token count (profiling runs)")
     ap.add_argument("--kv-only", action="store_true", help="run only the attention-block leg (profiling runs)")
     ap.add_argument("--kv-seqs", type=int, default=16, help="sequences in the attention-block leg")
     ap.add_argument("--kv-len", type=int, default=8192, help="cached positions per sequence in the attention-block leg")
@@ -995,6 +1049,9 @@ def main():
     ap.add_argument("--layers", default="", help="comma-separated subset of qkv,o,gate_up,down (profiling runs)")
     args = ap.parse_args()
     select_model(args.model)
+    if args.tokens > 0:
+        global T_PREFILL
+        T_PREFILL = args.tokens
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # Plain `python bench.py --gpus N`: start the N ranks here, one process per GPU, the way a launcher would.
         sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
