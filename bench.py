@@ -675,7 +675,7 @@ def project_study(resq, torch, dev, peaks, T, launches=60):
             "frac_of_bf16_sustained": round(2.0 * rows * K * K / (med * 1e-3) / 1e12 / peaks["bf16_sustained"], 4),
             "sm_mhz_median": mhz, "clocks": clocks,
             "sm_cycles_per_k_block": round(med * 1e-3 * mhz * 1e6 / kblocks_per_pair, 1) if mhz else None,
-            "ideal_cycles_per_k_block": 256.0,   # 256 x 256 x 64 MACs per pair and K block at 8192 dense bf16 MACs per SM-clock
+            "nominal_cycles_per_k_block": round(256 * 256 * 64 * 2 / (2 * NOMINAL["bf16_tflops"] * 1e12 / 148 / 1.965e9), 1),   # 256 x 256 x 64 multiply-adds per pair
             "tiles": tiles, "rounds_of_74_pairs": round(tiles / 74.0, 2)}
 
 

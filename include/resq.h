@@ -102,6 +102,23 @@ int resq_pack_weights(const resq_layer_desc_t* desc, const float* W_proj, int8_t
                       void* s_w8, void* s_w4, int8_t* w4_i8, void* stream);
 
 /*
+ * Eq. 3 with the rounding of the paper's experiments (Section 5.1: "apply GPTQ for weight quantization"; Frantar et
+ * al., 2022) instead of round-to-nearest.  W_proj as for resq_pack_weights.  U_inv: fp32 [K][K], the upper triangular
+ * Cholesky factor of the inverse of the layer's damped input Hessian H = (2/n) X^T X + 0.01 mean(diag) I, X being
+ * calibration inputs of the layer in the projected basis (H^-1 = U_inv^T U_inv; the factorisation is the caller's:
+ * any LAPACK, offline).  dead_cols: optional bytes [K], non-zero where H had a zero diagonal entry (an input that was
+ * never active): those weights are set to 0.  Per output channel: the scales are those of resq_pack_weights on the
+ * rows as given; columns are visited in order, column j is rounded to code_j = clamp(round-half-even(w_j / s)), and
+ * (w_j - code_j s) / U_inv[j][j] times U_inv[j][j+1:] is subtracted from the columns not yet visited.  All of it in
+ * fp64, one rounding per operation in this order, so the codes are reproducible bit for bit.  An offline step: the
+ * sweep is a chain of K dependent steps per row.  K * 9 bytes (a row in shared memory) must not exceed 200 KB, else
+ * RESQ_ERR_SHAPE.  Outputs as resq_pack_weights.
+ */
+int resq_pack_weights_gptq(const resq_layer_desc_t* desc, const float* W_proj, const float* U_inv,
+                           const uint8_t* dead_cols, int8_t* w8, uint8_t* w4, void* s_w8, void* s_w4, int8_t* w4_i8,
+                           void* stream);
+
+/*
  * Eq. 3 with the projection done here (Section 4.3: the bases are multiplied into the weights offline): W_raw is
  * the unprojected weight as bf16 [n_out][K] (row n = the K input weights of output channel n), U the basis as
  * bf16 [K][K] (row i = input feature, column j = coefficient, as P of resq_project_quantize).  Forms

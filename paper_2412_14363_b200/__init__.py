@@ -22,7 +22,7 @@ Y_BF16, Y_FP32 = 0, 1
 
 EXPORTS = [
     "resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_bytes", "resq_workspace_bytes",
-    "resq_pack_weights", "resq_pack_weights_projected", "resq_pack_projected_workspace_bytes", "resq_project", "resq_project_workspace_bytes", "resq_hadamard_quantize", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
+    "resq_pack_weights", "resq_pack_weights_gptq", "resq_pack_weights_projected", "resq_pack_projected_workspace_bytes", "resq_project", "resq_project_workspace_bytes", "resq_hadamard_quantize", "resq_project_quantize", "resq_project_quantize_static", "resq_mixed_gemm", "resq_linear",
     "resq_unpack_int4", "resq_set_option",
     "resq_weight_row_sums", "resq_project_quantize_asym", "resq_mixed_gemm_asym", "resq_linear_asym",
     "resq_workspace_bytes_asym",
@@ -60,6 +60,7 @@ for _n in ("resq_w8_bytes", "resq_w4_bytes", "resq_w4_i8_bytes", "resq_scale_byt
 lib.resq_workspace_bytes.restype = _sz
 lib.resq_workspace_bytes.argtypes = [_dp, _i, _i, _i]
 lib.resq_pack_weights.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.resq_pack_weights_gptq.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.resq_pack_projected_workspace_bytes.restype = _sz
 lib.resq_pack_projected_workspace_bytes.argtypes = [_dp]
 lib.resq_pack_weights_projected.argtypes = [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
@@ -147,6 +148,26 @@ def resq_pack_weights(desc: LayerDesc, W_proj, with_w4_i8: bool = True) -> Weigh
                 torch.empty((desc.n_out, K4), dtype=torch.int8, device=dev) if with_w4_i8 else None)
     _check(lib.resq_pack_weights(ctypes.byref(desc), _ptr(W_proj), _ptr(w.w8), _ptr(w.w4), _ptr(w.s_w8),
                                  _ptr(w.s_w4), _ptr(w.w4_i8), _stream()), "resq_pack_weights")
+    return w
+
+
+def resq_pack_weights_gptq(desc: LayerDesc, W_proj, U_inv, dead_cols=None, with_w4_i8: bool = True) -> Weights:
+    """W_proj fp32 [n_out][K], U_inv fp32 [K][K] (upper Cholesky factor of the inverse Hessian), dead_cols uint8 [K] or
+    None: GPTQ rounding instead of round-to-nearest (buffers allocated here)."""
+    import torch
+    assert W_proj.is_cuda and W_proj.dtype == torch.float32 and tuple(W_proj.shape) == (desc.n_out, desc.K)
+    assert U_inv.dtype == torch.float32 and tuple(U_inv.shape) == (desc.K, desc.K) and U_inv.is_contiguous()
+    dev = W_proj.device
+    K4 = desc.K - desc.r
+    sdt = torch.float16 if desc.w_scale_dtype == SCALE_FP16 else torch.float32
+    w = Weights(desc,
+                torch.empty((desc.n_out, desc.r), dtype=torch.int8, device=dev),
+                torch.empty((desc.n_out, K4 // 2), dtype=torch.uint8, device=dev),
+                torch.empty(desc.n_out, dtype=sdt, device=dev),
+                torch.empty(desc.n_out, dtype=sdt, device=dev),
+                torch.empty((desc.n_out, K4), dtype=torch.int8, device=dev) if with_w4_i8 else None)
+    _check(lib.resq_pack_weights_gptq(ctypes.byref(desc), _ptr(W_proj), _ptr(U_inv), _ptr(dead_cols), _ptr(w.w8), _ptr(w.w4),
+                                      _ptr(w.s_w8), _ptr(w.s_w4), _ptr(w.w4_i8), _stream()), "resq_pack_weights_gptq")
     return w
 
 

@@ -151,6 +151,19 @@ int resq_pack_weights(const resq_layer_desc_t* d, const float* W_proj, int8_t* w
                                              static_cast<size_t>(d->K) * 4, static_cast<cudaStream_t>(stream)));
 }
 
+int resq_pack_weights_gptq(const resq_layer_desc_t* d, const float* W_proj, const float* U_inv, const uint8_t* dead_cols,
+                           int8_t* w8, uint8_t* w4, void* s_w8, void* s_w4, int8_t* w4_i8, void* stream) {
+    if (int e = check_desc(d)) return e;
+    if (!W_proj || !U_inv || (!w8 && d->r > 0) || !w4 || !s_w8 || !s_w4) return RESQ_ERR_NULL;
+    if (!aligned16(W_proj) || !aligned16(U_inv) || !aligned16(w8) || !aligned16(w4) || !aligned16(s_w8) ||
+        !aligned16(s_w4) || !aligned16(w4_i8))
+        return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    const cudaError_t e = launch_pack_gptq(W_proj, U_inv, dead_cols, d->n_out, d->K, d->r, w8, w4, s_w8, s_w4,
+                                           d->w_scale_dtype == RESQ_SCALE_FP16, w4_i8, static_cast<cudaStream_t>(stream));
+    return e == cudaErrorNotSupported ? RESQ_ERR_SHAPE : cuda_status(e);
+}
+
 size_t resq_pack_projected_workspace_bytes(const resq_layer_desc_t* d) {
     if (check_desc(d)) return 0;
     return align_up(static_cast<size_t>(d->n_out < kPanelRows ? d->n_out : kPanelRows) * d->K * 4);

@@ -28,6 +28,12 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
                                   uint8_t* q4, void* s8, void* s4, bool scale_fp16, int8_t* q4_i8,
                                   size_t in_row_stride, cudaStream_t st, bool programmatic = false);
 
+// GPTQ rounding of the rows of W [N][K] fp32 with the upper Cholesky factor U [K][K] fp32 of the inverse Hessian
+// (Section 5.1); dead: optional [K] bytes, non-zero = the column's weights are zeroed.  Returns cudaErrorNotSupported
+// when a row (9 bytes per weight) does not fit in shared memory.
+cudaError_t launch_pack_gptq(const float* W, const float* U, const uint8_t* dead, int N, int K, int r, int8_t* w8,
+                             uint8_t* w4, void* s8, void* s4, bool scale_fp16, int8_t* w4e, cudaStream_t st);
+
 // Hadamard transform of the bf16 rows (H_K / sqrt(K), K = 2^k * {1, 12, 28}) fused with the split quantizer
 // (r may be 0).  Returns cudaErrorNotSupported for other K or rows wider than 200 KB of fp32.
 cudaError_t launch_hadamard_quantize(const void* X, size_t rows, int K, int r, int8_t* q8, uint8_t* q4, float* s8,
