@@ -53,6 +53,7 @@ constexpr int kUnitRows = 8;
 constexpr int kItemRows = 16;  // two units share the token operand
 constexpr int kMaxStages = 8;
 constexpr int kMinStages = 2;
+constexpr int kEarlyStages = 8;  // ring stages a warp requests before the activations are staged (1: 36.3 us for the 8B block at one token, 2: 33.6, 3: 32.7, 8: 32.5)
 constexpr int kSmemLimit = 227 * 1024;
 constexpr int kControlBytes = kWarps > 8 ? 2048 : 1024;
 constexpr int kSlotInts = 2 * 2 * 128;  // [token group][acc8 | acc4][fragment element]: one shared item
@@ -95,7 +96,7 @@ struct __align__(16) Control {
     int s_even[16];  // per token: sum of the even-position INT4 activation codes
     int arrived[kWarps];  // per slot: warps that have added their part
     int abort_flag;
-    uint64_t act_bar;  // completion of the bulk copies that stage the activation rows (packed staging only)
+    uint64_t act_bar[kWarps];  // per warp: completion of the bulk copies it issued to stage activation rows (packed staging only)
 };
 static_assert(sizeof(Control) <= kControlBytes, "control block");
 
@@ -333,19 +334,27 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             // Packed staging needs no arithmetic: one bulk copy per token row and segment, all in flight at once
             // (16 rows of a 14336-wide layer are 129 KB), issued by the lanes of the last warp; the threads only
             // write the zeros behind the rows and the zero row.
-            if (warp == kWarps - 1) {
+            // Copy i of the 2 T copies (token i / 2, INT8 segment when i is even) is issued by lane i / kWarps of
+            // warp i % kWarps: a warp's copies complete on its own barrier, and no warp issues more than four.
+            {
+                const int mine = (2 * p.T - warp + kWarps - 1) / kWarps;  // copies i = warp + kWarps * l, l < mine
                 if (lane == 0) {
-                    mbar_init(&ctl->act_bar, 1);
+                    uint32_t bytes = 0;
+                    for (int l = 0; l < mine; ++l) {
+                        const int i = warp + kWarps * l;
+                        bytes += (i & 1) ? static_cast<uint32_t>(p.row4) : static_cast<uint32_t>(p.r);
+                    }
+                    mbar_init(&ctl->act_bar[warp], 1);
                     fence_mbar_init();
-                    mbar_arrive_expect_tx(&ctl->act_bar, static_cast<uint32_t>(p.T) * static_cast<uint32_t>(p.r + p.row4));
+                    mbar_arrive_expect_tx(&ctl->act_bar[warp], bytes);
                 }
                 __syncwarp();
-                for (int i = lane; i < 2 * p.T; i += 32) {
-                    const int t = i >> 1;
+                if (lane < mine) {
+                    const int i = warp + kWarps * lane, t = i >> 1;
                     if ((i & 1) == 0) {
-                        if (p.r > 0) bulk_load(act8 + static_cast<size_t>(t) * p.pitch8, p.x8 + static_cast<size_t>(t) * p.r, p.r, &ctl->act_bar);
+                        if (p.r > 0) bulk_load(act8 + static_cast<size_t>(t) * p.pitch8, p.x8 + static_cast<size_t>(t) * p.r, p.r, &ctl->act_bar[warp]);
                     } else {
-                        bulk_load(act4 + static_cast<size_t>(t) * p.pitch4, p.x4 + static_cast<size_t>(t) * p.row4, p.row4, &ctl->act_bar);
+                        bulk_load(act4 + static_cast<size_t>(t) * p.pitch4, p.x4 + static_cast<size_t>(t) * p.row4, p.row4, &ctl->act_bar[warp]);
                     }
                 }
             }
@@ -392,8 +401,11 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             }
         }
         if (lane == 0) {
-            for (int s = issued; s < first_burst; ++s) issue(s);
-            issued = first_burst;
+            // Part of the ring now, the rest once the activations are staged: a copy instruction waits for room in
+            // the SM's copy queue, and a warp held there holds up the barrier below and with it the first product.
+            const int now = first_burst < kEarlyStages ? first_burst : kEarlyStages;
+            for (int s = issued; s < now; ++s) issue(s);
+            if (issued < now) issued = now;
         }
         if constexpr (kSplit) {
             store8(0, va);
@@ -417,7 +429,10 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
     }
     __syncthreads();
     bool ok = true;
-    if constexpr (!kSplit) ok = mbar_wait(&ctl->act_bar, 0, abort_flag, p.status);  // the staged rows have landed
+    if constexpr (!kSplit) {  // the staged rows have landed
+#pragma unroll 1
+        for (int w = 0; w < kWarps && ok; ++w) ok = mbar_wait(&ctl->act_bar[w], 0, abort_flag, p.status);
+    }
     int sevt[TT][2];
 #pragma unroll
     for (int tt = 0; tt < TT; ++tt)
@@ -434,6 +449,7 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
     int stage = 0;
     uint32_t phase = 0;
     int consumed = 0;
+    int iss_stage = issued == p.nstages ? 0 : issued;  // the stage the next copy goes into (lane 0)
     int idx = cb, item = pb >> 16, c = pb & 0xFFFF;
     while (idx < ce && ok) {
         // One segment: this warp's part of `item` (all of it, or a slice of its chunks).
@@ -523,9 +539,15 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
             }
             ++consumed;
             __syncwarp();
-            if (lane == 0 && is_idx < ce) {
-                ++issued;
-                issue(stage);  // refill the stage just read
+            if (lane == 0) {
+                // Copies go into the ring's stages in order.  One per chunk read keeps a full ring full; until the
+                // ring is as deep as it gets, two per chunk read: it deepens while the first chunks are consumed
+                // instead of holding up the first product.
+                for (int k = 0; k < 2 && is_idx < ce && issued - consumed < p.nstages; ++k) {
+                    issue(iss_stage);
+                    if (++iss_stage == p.nstages) iss_stage = 0;
+                    ++issued;
+                }
             }
             if (++stage == p.nstages) { stage = 0; phase ^= 1; }
         }
@@ -622,7 +644,8 @@ mixed_gemm_stream_kernel(const __grid_constant__ CUtensorMap tmW8, const __grid_
     }
     if (!kSplit && !ok && threadIdx.x == kThreads - 32) {
         const uint64_t t0 = global_timer_ns();
-        while (!mbar_try_wait(&ctl->act_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+        for (int w = 0; w < kWarps; ++w)
+            while (!mbar_try_wait(&ctl->act_bar[w], 0) && global_timer_ns() - t0 < 100000000ull) {}
     }
     __syncthreads();
     if (threadIdx.x == 0 && ctl->abort_flag) atomicOr(p.status, kStatusBitTimeout);
