@@ -634,6 +634,7 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
     if (!scale_fp16 && row_bytes <= static_cast<size_t>(kFastMaxRowBytes) && in_row_stride_bytes % 16 == 0) {
         int rpc = 1;  // rows per CTA: 1, 2, 4 or 8, about kFastGroupBytes of staging
         while (rpc < 8 && row_bytes * rpc * 2 <= static_cast<size_t>(kFastGroupBytes)) rpc *= 2;
+        while (rpc > 1 && rows / rpc < 148) rpc /= 2;  // few rows (a generation step): all threads of a CTA on one row
         const size_t smem = row_bytes * rpc;
         auto kern = in_is_f32 ? split_quantize_fast_kernel<true> : split_quantize_fast_kernel<false>;
         static bool attr_set[2][64] = {};
@@ -656,7 +657,10 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
             attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
             attr[0].val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = attr;
-            cfg.numAttrs = programmatic ? 1 : 0;
+            // The kernel waits for the preceding grid itself (griddepcontrol.wait on entry), so it may always be
+            // scheduled while that grid drains; for the few rows of a generation step this hides most of its launch.
+            (void)programmatic;
+            cfg.numAttrs = 1;
             count_launch();
             return cudaLaunchKernelEx(&cfg, kern, in, in_row_stride_bytes, rows, K, r, rpc, q8, q4,
                                       static_cast<float*>(s8), static_cast<float*>(s4), q4_i8, device_status_ptr());
