@@ -119,6 +119,19 @@ int resq_attention_queries(const resq_kv_cache_t* cache, const void* q16, int n_
                            const int32_t* q_seq, const int32_t* q_len, float* out, void* workspace,
                            size_t workspace_bytes, void* stream);
 
+/* Causal attention of a run of T new tokens of ONE sequence over the cache, on the tensor cores (prefill and chunked
+ * prefill; Section 4.3 Eq. 8 with the cache of Section 5.1): token t -- q16 half [T][n_q_heads][d_head], at position
+ * pos0 + t of cache sequence `seq` -- attends positions 0 .. pos0 + t, which must have been appended (the T new
+ * tokens included); out fp32 [T][n_q_heads][d_head].  seq, pos0 and T are host values: 0 <= seq < n_seqs, pos0 >= 0,
+ * T >= 1, pos0 + T <= capacity, else RESQ_ERR_SHAPE.  No workspace.
+ * The same definition as resq_attention_queries with q_seq[t] = seq, q_len[t] = pos0 + t + 1, evaluated tile-wise: 128
+ * (token, query head) rows that share a KV head meet 64 cache positions at a time, every cache block is read once per
+ * such tile.  The score products run on the integer codes held exactly in half (scales and zero-points applied in
+ * fp32), the softmax is fp32 with the row maximum found in a first pass over the keys, the softmax weights times the
+ * value scales are rounded to half before the second product, accumulation is fp32. */
+int resq_attention_prefill(const resq_kv_cache_t* cache, const void* q16, int n_q_heads, int seq, int pos0, int T,
+                           float* out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -638,6 +638,17 @@ int resq_attention_queries(const resq_kv_cache_t* cache, const void* q16, int n_
                                                static_cast<cudaStream_t>(stream), n_queries, q_seq));
 }
 
+int resq_attention_prefill(const resq_kv_cache_t* cache, const void* q16, int n_q_heads, int seq, int pos0, int T,
+                           float* out, void* stream) {
+    if (int e = check_cache(cache)) return e;
+    if (resq_attention_workspace_bytes(1, n_q_heads, cache->n_kv_heads, cache->d_head) == 0) return RESQ_ERR_SHAPE;
+    if (seq < 0 || seq >= cache->n_seqs || pos0 < 0 || T < 1 || pos0 > cache->capacity - T) return RESQ_ERR_SHAPE;
+    if (!q16 || !out) return RESQ_ERR_NULL;
+    if (!aligned16(q16) || !aligned16(out)) return RESQ_ERR_ALIGN;
+    if (int e = check_arch()) return e;
+    return cuda_status(launch_attention_prefill(*cache, q16, n_q_heads, seq, pos0, T, out, static_cast<cudaStream_t>(stream)));
+}
+
 const char* resq_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 const char* resq_status_string(int s) {

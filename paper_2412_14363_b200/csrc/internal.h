@@ -92,6 +92,10 @@ cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q1
                                     float* out, void* scratch, cudaStream_t st, int n_rows = -1,
                                     const int32_t* seq_map = nullptr);
 
+// Causal attention of T new tokens of sequence `seq` (positions pos0 .. pos0 + T - 1) on the tensor cores.
+cudaError_t launch_attention_prefill(const resq_kv_cache_t& cache, const void* q16, int n_q_heads, int seq, int pos0,
+                                     int T, float* out, cudaStream_t st);
+
 // Driver entry point for tensor-map encoding (resolved once, without linking libcuda).
 void* tensor_map_encode_fn();
 

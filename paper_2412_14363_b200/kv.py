@@ -8,7 +8,7 @@ from . import ERR_CUDA, ERR_INDEX, OK, ResqError, _check, _ptr, _stream, lib  # 
 KV_BLOCK, KV_BLOCK_BYTES = 32, 5632
 KV_EXPORTS = ["resq_kv_cache_bytes", "resq_uc_quantize", "resq_query_project", "resq_kv_append", "resq_qkv_project_append",
               "resq_attention_workspace_bytes", "resq_attention_decode", "resq_attention_queries_workspace_bytes",
-              "resq_attention_queries"]
+              "resq_attention_queries", "resq_attention_prefill"]
 
 
 class KvCacheStruct(ctypes.Structure):
@@ -30,6 +30,7 @@ lib.resq_attention_decode.argtypes = [_cp, _vp, _i, _vp, _vp, _vp, _sz, _vp]
 lib.resq_attention_queries_workspace_bytes.restype = _sz
 lib.resq_attention_queries_workspace_bytes.argtypes = [_i, _i, _i, _i]
 lib.resq_attention_queries.argtypes = [_cp, _vp, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.resq_attention_prefill.argtypes = [_cp, _vp, _i, _i, _i, _i, _vp, _vp]
 
 
 class KvCache:
@@ -105,3 +106,10 @@ def resq_attention_queries(cache: KvCache, q16, q_seq, q_len, out, workspace=Non
         workspace = torch.empty(nbytes, dtype=torch.uint8, device=cache.data.device)
     _check(lib.resq_attention_queries(ctypes.byref(cache.c), _ptr(q16), hq, n, _ptr(q_seq), _ptr(q_len), _ptr(out),
                                       _ptr(workspace), workspace.numel(), _stream()), "resq_attention_queries")
+
+
+def resq_attention_prefill(cache: KvCache, q16, seq: int, pos0: int, out):
+    """q16 half [T][n_q_heads][128]: token t, at position pos0 + t of cache sequence `seq`, attends positions
+    0 .. pos0 + t (already appended); out fp32 of q16's shape."""
+    _check(lib.resq_attention_prefill(ctypes.byref(cache.c), _ptr(q16), q16.shape[1], int(seq), int(pos0), q16.shape[0],
+                                      _ptr(out), _stream()), "resq_attention_prefill")
