@@ -608,6 +608,16 @@ def kv_leg(resq, torch, dev, peaks, steps, n_seqs=16, seq_len=8192, prefill_T=40
     wsq = torch.empty(int(resq.lib.resq_attention_queries_workspace_bytes(Tp, KV_HQ, KV_HKV, KV_D)), dtype=torch.uint8, device=dev)
     mq_ms = timed(lambda i: kv.resq_attention_queries(caches[i % 2], qa16, qs, ql, oa, wsq), max(3, steps // 4))
     mq_blocks = int(((ql + 31) // 32).sum().item()) * KV_HKV
+    # the same rows tile-wise on the tensor cores, then the causal attention of the whole sequence
+    pf_ms = timed(lambda i: kv.resq_attention_prefill(caches[i % 2], qa16, 0, seq_len - Tp, oa), max(3, steps // 4))
+    pf_flops = 4.0 * KV_D * KV_HQ * float(ql.sum().item())
+    Tf = min(seq_len, 8192)
+    qf16 = torch.empty((Tf, KV_HQ, KV_D), dtype=torch.float16, device=dev)
+    for t0 in range(0, Tf, T):
+        kv.resq_query_project(qp[:min(T, Tf - t0)], wq, s_u, qf16[t0:t0 + min(T, Tf - t0)])
+    of = torch.empty((Tf, KV_HQ, KV_D), dtype=torch.float32, device=dev)
+    full_ms = timed(lambda i: kv.resq_attention_prefill(caches[i % 2], qf16, 0, 0, of), max(3, steps // 4))
+    full_flops = 4.0 * KV_D * KV_HQ * (Tf * (Tf + 1) / 2)
     app_bytes = T * KV_HKV * (2 * 2 * KV_D + 2 * 88)
     qp_bytes = T * KV_HQ * (2 * KV_D + 2 * KV_D)
     st = resq.resq_device_status()
@@ -627,7 +637,14 @@ def kv_leg(resq, torch, dev, peaks, steps, n_seqs=16, seq_len=8192, prefill_T=40
             "many_query_attention": {"queries": Tp, "prefix_positions": f"{seq_len - Tp + 1}..{seq_len}",
                                      "us": round(mq_ms * 1e3, 1),
                                      "cache_block_reads_gbs": round(mq_blocks * 5632 / (mq_ms * 1e-3) / 1e9, 1),
-                                     "note": "each query row streams its own prefix (L2-resident): batched single-query passes"}}
+                                     "note": "each query row streams its own prefix (L2-resident): batched single-query passes"},
+            "prefill_attention": {"kernel": "attention_prefill_kernel (tcgen05 kind::f16, 128 rows x 64 positions per step)",
+                                  "chunk": {"queries": Tp, "prefix_positions": f"{seq_len - Tp + 1}..{seq_len}",
+                                            "us": round(pf_ms * 1e3, 1), "tflops": round(pf_flops / (pf_ms * 1e-3) / 1e12, 1),
+                                            "vs_many_query_call": round(mq_ms / pf_ms, 2)},
+                                  "whole_sequence": {"tokens": Tf, "us": round(full_ms * 1e3, 1),
+                                                     "tflops": round(full_flops / (full_ms * 1e-3) / 1e12, 1)},
+                                  "flops": "4 d_head per (query head, attended position): both products, causal part only"}}
 
 
 # --------------------------------------------------------------------------------------- projection GEMM study

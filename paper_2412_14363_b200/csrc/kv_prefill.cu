@@ -2,18 +2,22 @@
 // Section 5.1) on the tcgen05 tensor cores: the prefill form, where every cache block is read once per tile of
 // 128 (token, query head) rows instead of once per query.
 //
-// One CTA of 128 threads owns 128 rows that share a KV head -- 128 / g consecutive tokens times the g query heads
+// One CTA of 256 threads owns 128 rows that share a KV head -- 128 / g consecutive tokens times the g query heads
 // of the group -- and walks the cache of its sequence in steps of 64 positions (two cache blocks, brought in whole
-// by bulk copies, double buffered).  Per step:
+// by bulk copies, double buffered).  Two threads share a row: thread (row, h) handles the 32 positions of cache
+// block h of the step; their partial maxima and sums meet in shared memory between the passes and at the end.
+// Two CTAs fit on an SM (256 TMEM columns and about 108 KB of shared memory each), so one's tensor-core work and
+// waits overlap the other's expansion and softmax arithmetic.  Per step:
 //   keys     the 8-bit and 4-bit CODES are expanded to fp16 integers (exact) into a K-major operand tile; the
 //            tensor core forms S8 = Q[:, :16]·C8^T and S4 = Q[:, 16:]·C4^T as two TMEM accumulators, and the thread
 //            that owns a row applies the per-position scales and zero-points in fp32:
 //                score = (s8·S8 + z8·sum(q[:16]) + s4·S4 + z4·sum(q[16:])) / sqrt(d).
-//   softmax  fp32, one thread per row (TMEM lane = row).  Two passes over the cache: the first finds each row's
-//            maximum score (and the largest value scale, for the normalisation below), the second forms
-//            p = exp(score - max), so the output accumulator never has to be rescaled.
+//   softmax  fp32 (TMEM lane = row).  Two passes over the cache: the first finds each row's maximum score (and the
+//            tile's largest value scale, for the normalisation below), the second forms p = exp(score - max), so the
+//            output accumulator never has to be rescaled.  Steps that lie wholly below the tile's first position
+//            skip the causal comparison.
 //   values   P8' = half(p · s8_v · 2^-E) and P4' = half(p · s4_v · 2^-E) are written as two K-major operand tiles
-//            (2^E = the row's largest value scale rounded down to a power of two, so the products stay in half's
+//            (2^E = the tile's largest value scale rounded down to a power of two, so the products stay in half's
 //            normal range), the value codes are expanded, transposed, into an operand tile [coefficient][position],
 //            (centred: code - 128, code - 8) and the tensor core accumulates O[:, :16] += P8'·C8v,
 //            O[:, 16:] += P4'·C4v in TMEM.  The zero-points (plus the centres times the scales) enter as
@@ -45,9 +49,13 @@ constexpr int kKVBytes = 16384;           // keys [64 pos][128 coef] (two halves
 constexpr int kPBytes = 16384;            // [128 rows][64 pos]
 constexpr int kRawBytes = 2 * kBlockBytes;
 constexpr uint32_t kTmemCols = 256;       // S8: 0..63, S4: 64..127, O: 128..255
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;
 
 struct Shared {
+    float4 colK[kStep];    // per position of the step: key (s8, z8, s4, z4) times log2(e) / sqrt(d)
+    float4 colV[kStep];    // value (s8 2^-E, z8 + 128 s8, s4 2^-E, z4 + 8 s4)
+    float xch[3][2][kRows];  // partial results of the two threads of a row
+    float vmax[kStep];
     uint64_t load[2];
     uint64_t mma;
     uint32_t tmem_base;
@@ -94,65 +102,114 @@ __device__ __forceinline__ uint32_t pack_h2(float a, float b) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// Keys of the step: position j = tid % 64, coefficient half a = tid / 64 -> eight 16-byte chunks of tile row j.
+// Keys of the step: position j = tid % 64, quarter tid / 64 of the row's sixteen 16-byte chunks.
 __device__ __forceinline__ void expand_keys(const uint8_t* raw, uint8_t* tile, int tid) {
-    const int j = tid & 63, a = tid >> 6;
+    const int j = tid & 63, qtr = tid >> 6;
     const uint8_t* blk = raw + (j >> 5) * kBlockBytes;
     const int jp = j & 31;
-    uint8_t* row = tile + a * (kStep * 128) + j * 128;
+    uint8_t* row = tile + (qtr >> 1) * (kStep * 128) + j * 128;
     const int sw = j & 7;
     const uint32_t* k4 = reinterpret_cast<const uint32_t*>(blk + kOffK4 + jp * 56);
-    if (a == 0) {
+    const int c0 = 4 * (qtr & 1);  // first chunk inside the 128-byte half row
+    if (qtr == 0) {
         const uint4 k8 = *reinterpret_cast<const uint4*>(blk + jp * 16);
         *reinterpret_cast<uint4*>(row + ((0 ^ sw) << 4)) = make_uint4(bytes_to_h2<0x4140>(k8.x), bytes_to_h2<0x4342>(k8.x),
                                                                       bytes_to_h2<0x4140>(k8.y), bytes_to_h2<0x4342>(k8.y));
         *reinterpret_cast<uint4*>(row + ((1 ^ sw) << 4)) = make_uint4(bytes_to_h2<0x4140>(k8.z), bytes_to_h2<0x4342>(k8.z),
                                                                       bytes_to_h2<0x4140>(k8.w), bytes_to_h2<0x4342>(k8.w));
 #pragma unroll
-        for (int w = 0; w < 6; ++w) {
-            const uint32_t x = k4[w];
-            *reinterpret_cast<uint4*>(row + (((2 + w) ^ sw) << 4)) =
+        for (int i = 0; i < 2; ++i) {
+            const uint32_t x = k4[i];
+            *reinterpret_cast<uint4*>(row + (((2 + i) ^ sw) << 4)) =
                 make_uint4(nibbles_to_h2(x, 0), nibbles_to_h2(x, 4), nibbles_to_h2(x, 8), nibbles_to_h2(x, 12));
         }
     } else {
+        const int w0 = 4 * qtr - 2;
 #pragma unroll
-        for (int w = 6; w < 14; ++w) {
-            const uint32_t x = k4[w];
-            *reinterpret_cast<uint4*>(row + (((w - 6) ^ sw) << 4)) =
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t x = k4[w0 + i];
+            *reinterpret_cast<uint4*>(row + (((c0 + i) ^ sw) << 4)) =
                 make_uint4(nibbles_to_h2(x, 0), nibbles_to_h2(x, 4), nibbles_to_h2(x, 8), nibbles_to_h2(x, 12));
         }
     }
 }
 
 // Values of the step, transposed: tile row n = output column, 64 positions (128 bytes) per row.
-__device__ __forceinline__ void store_value(uint8_t* tile, int n, int j, uint16_t h) {
-    *reinterpret_cast<uint16_t*>(tile + n * 128 + ((((j >> 3) ^ (n & 7)) << 4) | ((j & 7) << 1))) = h;
+__device__ __forceinline__ void store_value(uint8_t* tile, int n, int j, uint32_t h) {
+    *reinterpret_cast<uint16_t*>(tile + n * 128 + ((((j >> 3) ^ (n & 7)) << 4) | ((j & 7) << 1))) = static_cast<uint16_t>(h);
+}
+__device__ __forceinline__ void expand_value_word(uint8_t* tile, int w, int j, uint32_t x) {
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+        const uint32_t h2 = nibbles_to_h2<kBias4>(x, 4 * m);
+        store_value(tile, 16 + 8 * w + 2 * m, j, h2 & 0xFFFF);
+        store_value(tile, 16 + 8 * w + 2 * m + 1, j, h2 >> 16);
+    }
 }
 __device__ __forceinline__ void expand_values(const uint8_t* raw, uint8_t* tile, int tid) {
-    const int j = tid & 63, a = tid >> 6;
+    const int j = tid & 63, qtr = tid >> 6;
     const uint8_t* blk = raw + (j >> 5) * kBlockBytes;
     const int jp = j & 31;
     const uint32_t* v4 = reinterpret_cast<const uint32_t*>(blk + kOffV4 + jp * 56);
-    if (a == 0) {
+    if (qtr == 0) {
         const uint4 v8 = *reinterpret_cast<const uint4*>(blk + kOffV8 + jp * 16);
         const uint32_t w8[4] = {v8.x, v8.y, v8.z, v8.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const uint32_t lo = bytes_to_h2<0x4140, kBias8>(w8[i]), hi = bytes_to_h2<0x4342, kBias8>(w8[i]);
-            store_value(tile, 4 * i + 0, j, static_cast<uint16_t>(lo & 0xFFFF));
-            store_value(tile, 4 * i + 1, j, static_cast<uint16_t>(lo >> 16));
-            store_value(tile, 4 * i + 2, j, static_cast<uint16_t>(hi & 0xFFFF));
-            store_value(tile, 4 * i + 3, j, static_cast<uint16_t>(hi >> 16));
+            store_value(tile, 4 * i + 0, j, lo & 0xFFFF);
+            store_value(tile, 4 * i + 1, j, lo >> 16);
+            store_value(tile, 4 * i + 2, j, hi & 0xFFFF);
+            store_value(tile, 4 * i + 3, j, hi >> 16);
         }
-    }
-    const int w0 = a == 0 ? 0 : 6, w1 = a == 0 ? 6 : 14;
-    for (int w = w0; w < w1; ++w) {
-        const uint32_t x = v4[w];
+        expand_value_word(tile, 0, j, v4[0]);
+        expand_value_word(tile, 1, j, v4[1]);
+    } else {
+        const int w0 = 4 * qtr - 2;
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            const uint32_t h2 = nibbles_to_h2<kBias4>(x, 4 * m);
-            store_value(tile, 16 + 8 * w + 2 * m, j, static_cast<uint16_t>(h2 & 0xFFFF));
-            store_value(tile, 16 + 8 * w + 2 * m + 1, j, static_cast<uint16_t>(h2 >> 16));
+        for (int i = 0; i < 4; ++i) expand_value_word(tile, w0 + i, j, v4[w0 + i]);
+    }
+}
+
+// First pass over sixteen positions of one row: the running maximum of the scores.
+template <bool MASKED>
+__device__ __forceinline__ void scores_max(const uint32_t (&a8)[16], const uint32_t (&a4)[16], const float4* colK, int jb,
+                                           int pos_i, float qsum8, float qsum4, float& m2) {
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        const float4 k = colK[c];
+        const float sc = fmaf(k.x, __uint_as_float(a8[c]), fmaf(k.z, __uint_as_float(a4[c]), fmaf(k.y, qsum8, k.w * qsum4)));
+        if (!MASKED || jb + c <= pos_i) m2 = fmaxf(m2, sc);
+    }
+}
+
+// Second pass over sixteen positions of one row: softmax weights, their sums, and the two half-precision operand
+// chunks (16 positions = 32 bytes of the row in each of P8' and P4').
+template <bool MASKED>
+__device__ __forceinline__ void scores_weights(const uint32_t (&a8)[16], const uint32_t (&a4)[16], const float4* colK,
+                                               const float4* colV, int jb, int pos_i, float qsum8, float qsum4, float m2,
+                                               float& l, float& zsum8, float& zsum4, uint32_t (&w8)[8], uint32_t (&w4)[8]) {
+    float prev8 = 0.f, prev4 = 0.f;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        const float4 k = colK[c];
+        const float sc = fmaf(k.x, __uint_as_float(a8[c]), fmaf(k.z, __uint_as_float(a4[c]), fmaf(k.y, qsum8, k.w * qsum4)));
+        float p8 = 0.f, p4 = 0.f;
+        if (!MASKED || jb + c <= pos_i) {
+            const float pr = exp2f(sc - m2);
+            const float4 v = colV[c];
+            l += pr;
+            zsum8 = fmaf(pr, v.y, zsum8);
+            zsum4 = fmaf(pr, v.w, zsum4);
+            p8 = pr * v.x;
+            p4 = pr * v.z;
+        }
+        if (c & 1) {
+            w8[c >> 1] = pack_h2(prev8, p8);
+            w4[c >> 1] = pack_h2(prev4, p4);
+        } else {
+            prev8 = p8;
+            prev4 = p4;
         }
     }
 }
@@ -168,13 +225,15 @@ __global__ void __launch_bounds__(kThreads, 2) attention_prefill_kernel(const Pr
     Shared* sh = reinterpret_cast<Shared*>(raw + 2 * kRawBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5;
+    const int row = tid & (kRows - 1), half = tid >> 7;  // thread (row, half): cache block `half` of every step
     const int tile = static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x);  // long tiles first
     const int kvh = blockIdx.y;
-    const int R = tile * kRows + tid;
+    const int R = tile * kRows + row;
     const bool row_ok = R < p.T * p.g;
     const int tq = row_ok ? R / p.g : 0;
     const int hq = kvh * p.g + (row_ok ? R % p.g : 0);
     const int pos_i = row_ok ? p.pos0 + tq : -1;
+    const int pos_first = p.pos0 + (tile * kRows) / p.g;  // position of the tile's first row: the smallest
     const int tq_max = min(p.T - 1, (tile * kRows + kRows - 1) / p.g);
     const int last_pos = p.pos0 + tq_max;
     const int n_steps = last_pos / kStep + 1;
@@ -194,11 +253,12 @@ __global__ void __launch_bounds__(kThreads, 2) attention_prefill_kernel(const Pr
         tmem_relinquish();
     }
 
-    // ---- query tile: row = tid, coefficients in the tile's permutation; sums of the two segments
+    // ---- query tile: thread (row, half) writes half of the row's chunks, in the tile's permutation, and both
+    // threads of a row form the sums of the two segments
     float qsum8 = 0.f, qsum4 = 0.f;
     {
         const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(tq) * p.Hq + hq) * 128);
-        const int sw = tid & 7;
+        const int sw = row & 7;
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
             uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
@@ -216,7 +276,8 @@ __global__ void __launch_bounds__(kThreads, 2) attention_prefill_kernel(const Pr
                 v = make_uint4(__byte_perm(v.x, v.z, 0x5410), __byte_perm(v.x, v.z, 0x7632), __byte_perm(v.y, v.w, 0x5410),
                                __byte_perm(v.y, v.w, 0x7632));
             }
-            *reinterpret_cast<uint4*>(Qs + (c >> 3) * (kRows * 128) + tid * 128 + (((c & 7) ^ sw) << 4)) = v;
+            if ((c >> 3) == half)
+                *reinterpret_cast<uint4*>(Qs + (c >> 3) * (kRows * 128) + row * 128 + (((c & 7) ^ sw) << 4)) = v;
         }
     }
     fence_proxy_async_smem();
@@ -224,7 +285,7 @@ __global__ void __launch_bounds__(kThreads, 2) attention_prefill_kernel(const Pr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sh->tmem_base;
-    const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
 
     auto issue_load = [&](int gs) {
         const bool full = gs >= n_steps;
@@ -253,7 +314,7 @@ __global__ void __launch_bounds__(kThreads, 2) attention_prefill_kernel(const Pr
     const uint64_t p_desc8 = make_smem_desc_k128(smem_u32(P8)), p_desc4 = make_smem_desc_k128(smem_u32(P4));
 
     const float kScoreScale = 1.4426950408889634f * 0.08838834764831845f;  // log2(e) / sqrt(128)
-    float m2 = -INFINITY, vmax = 0.f, l = 0.f, zsum8 = 0.f, zsum4 = 0.f, out_scale = 1.f, p_scale = 1.f;
+    float m2 = -INFINITY, vmax_col = 0.f, l = 0.f, zsum8 = 0.f, zsum4 = 0.f, out_scale = 1.f, p_scale = 1.f;
     uint32_t mma_phase = 0;
     int bad = 0;
     int loads_issued = 0;
@@ -266,7 +327,16 @@ __global__ void __launch_bounds__(kThreads, 2) attention_prefill_kernel(const Pr
     for (int gs = 0; gs < total; ++gs) {
         const bool second = gs >= n_steps;
         const int s = second ? gs - n_steps : gs;
-        if (gs == n_steps) {  // between the passes: the normalisation of the value scales
+        const int j0 = s * kStep;
+        if (gs == n_steps) {
+            // between the passes: the two threads of a row merge their maxima; the tile's largest value scale gives
+            // the power of two that normalises the second product's left operand
+            sh->xch[0][half][row] = m2;
+            if (tid < kStep) sh->vmax[tid] = vmax_col;
+            __syncthreads();
+            m2 = fmaxf(sh->xch[0][0][row], sh->xch[0][1][row]);
+            float vmax = 0.f;
+            for (int i = 0; i < kStep; ++i) vmax = fmaxf(vmax, sh->vmax[i]);
             int e = 0;
             if (vmax > 0.f) e = min(max(ilogbf(vmax), -100), 100);
             p_scale = ldexpf(1.f, -e);
@@ -279,6 +349,16 @@ __global__ void __launch_bounds__(kThreads, 2) attention_prefill_kernel(const Pr
         const uint8_t* rb = raw + (gs & 1) * kRawBytes;
         if (!mbar_wait(&sh->load[gs & 1], (gs >> 1) & 1, &sh->abort_flag, p.status)) bad = 1;
         expand_keys(rb, KV, tid);
+        if (tid < kStep) {  // the step's per-position constants
+            const uint8_t* blk = rb + (tid >> 5) * kBlockBytes;
+            const float4 k = reinterpret_cast<const float4*>(blk + kOffKm)[tid & 31];
+            const float4 v = reinterpret_cast<const float4*>(blk + kOffVm)[tid & 31];
+            sh->colK[tid] = make_float4(k.x * kScoreScale, k.y * kScoreScale, k.z * kScoreScale, k.w * kScoreScale);
+            if (second)
+                sh->colV[tid] = make_float4(v.x * p_scale, fmaf(128.f, v.x, v.y), v.z * p_scale, fmaf(8.f, v.z, v.w));
+            else if (j0 + tid <= last_pos)
+                vmax_col = fmaxf(vmax_col, fmaxf(v.x, v.z));
+        }
         fence_proxy_async_smem();
         tc_fence_before();
         if (__syncthreads_or(bad)) {
@@ -298,65 +378,33 @@ __global__ void __launch_bounds__(kThreads, 2) attention_prefill_kernel(const Pr
         mma_phase ^= 1;
         tc_fence_after();
 
-        const int j0 = s * kStep;
+        const bool masked = j0 + kStep - 1 > pos_first;  // uniform over the CTA
 #pragma unroll 1
-        for (int hb = 0; hb < 2; ++hb) {  // one cache block (32 positions) at a time
-            uint32_t a8[32], a4[32];
+        for (int part = 0; part < 2; ++part) {  // sixteen positions at a time
+            const int col = 32 * half + 16 * part;
+            uint32_t a8[16], a4[16];
             __syncwarp();  // TMEM loads are warp-wide instructions
-            tmem_ld32(lane_addr + 32 * hb, a8);
-            tmem_ld32(lane_addr + 64 + 32 * hb, a4);
+            tmem_ld16(lane_addr + col, a8);
+            tmem_ld16(lane_addr + 64 + col, a4);
             tmem_ld_wait();
-            const uint8_t* blk = rb + hb * kBlockBytes;
-            const float4* km = reinterpret_cast<const float4*>(blk + kOffKm);
-            const float4* vm = reinterpret_cast<const float4*>(blk + kOffVm);
-            const int jb = j0 + 32 * hb;
             if (!second) {
-#pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    if (jb + c <= pos_i) {
-                        const float4 k = km[c];
-                        const float sc = (k.x * __uint_as_float(a8[c]) + k.y * qsum8 + k.z * __uint_as_float(a4[c]) +
-                                          k.w * qsum4) * kScoreScale;
-                        m2 = fmaxf(m2, sc);
-                        const float4 v = vm[c];
-                        vmax = fmaxf(vmax, fmaxf(v.x, v.z));
-                    }
-                }
+                if (masked)
+                    scores_max<true>(a8, a4, sh->colK + col, j0 + col, pos_i, qsum8, qsum4, m2);
+                else
+                    scores_max<false>(a8, a4, sh->colK + col, j0 + col, pos_i, qsum8, qsum4, m2);
             } else {
-                uint32_t w4[16], w8[16];
-                float prev4 = 0.f, prev8 = 0.f;
-#pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    float p4 = 0.f, p8 = 0.f;
-                    if (jb + c <= pos_i) {
-                        const float4 k = km[c];
-                        const float sc = (k.x * __uint_as_float(a8[c]) + k.y * qsum8 + k.z * __uint_as_float(a4[c]) +
-                                          k.w * qsum4) * kScoreScale;
-                        const float pr = exp2f(sc - m2);
-                        const float4 v = vm[c];
-                        l += pr;
-                        zsum8 = fmaf(pr, fmaf(128.f, v.x, v.y), zsum8);
-                        zsum4 = fmaf(pr, fmaf(8.f, v.z, v.w), zsum4);
-                        p8 = pr * (v.x * p_scale);
-                        p4 = pr * (v.z * p_scale);
-                    }
-                    if (c & 1) {
-                        w8[c >> 1] = pack_h2(prev8, p8);
-                        w4[c >> 1] = pack_h2(prev4, p4);
-                    } else {
-                        prev8 = p8;
-                        prev4 = p4;
-                    }
-                }
-                const int sw = tid & 7;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int chunk = 4 * hb + c;
-                    *reinterpret_cast<uint4*>(P8 + tid * 128 + ((chunk ^ sw) << 4)) =
-                        make_uint4(w8[4 * c], w8[4 * c + 1], w8[4 * c + 2], w8[4 * c + 3]);
-                    *reinterpret_cast<uint4*>(P4 + tid * 128 + ((chunk ^ sw) << 4)) =
-                        make_uint4(w4[4 * c], w4[4 * c + 1], w4[4 * c + 2], w4[4 * c + 3]);
-                }
+                uint32_t w8[8], w4[8];
+                if (masked)
+                    scores_weights<true>(a8, a4, sh->colK + col, sh->colV + col, j0 + col, pos_i, qsum8, qsum4, m2, l,
+                                         zsum8, zsum4, w8, w4);
+                else
+                    scores_weights<false>(a8, a4, sh->colK + col, sh->colV + col, j0 + col, pos_i, qsum8, qsum4, m2, l,
+                                          zsum8, zsum4, w8, w4);
+                const int sw = row & 7, chunk = col >> 3;
+                *reinterpret_cast<uint4*>(P8 + row * 128 + ((chunk ^ sw) << 4)) = make_uint4(w8[0], w8[1], w8[2], w8[3]);
+                *reinterpret_cast<uint4*>(P8 + row * 128 + (((chunk + 1) ^ sw) << 4)) = make_uint4(w8[4], w8[5], w8[6], w8[7]);
+                *reinterpret_cast<uint4*>(P4 + row * 128 + ((chunk ^ sw) << 4)) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                *reinterpret_cast<uint4*>(P4 + row * 128 + (((chunk + 1) ^ sw) << 4)) = make_uint4(w4[4], w4[5], w4[6], w4[7]);
             }
         }
         if (second) {
@@ -390,10 +438,17 @@ __global__ void __launch_bounds__(kThreads, 2) attention_prefill_kernel(const Pr
     }
 
     if (!bad) {  // uniform over the CTA: the TMEM loads are warp-wide instructions, only the stores depend on the row
+        sh->xch[0][half][row] = l;
+        sh->xch[1][half][row] = zsum8;
+        sh->xch[2][half][row] = zsum4;
+        __syncthreads();
+        l = sh->xch[0][0][row] + sh->xch[0][1][row];
+        zsum8 = sh->xch[1][0][row] + sh->xch[1][1][row];
+        zsum4 = sh->xch[2][0][row] + sh->xch[2][1][row];
         const float inv = l > 0.f ? 1.f / l : 0.f;
         float* dst = p.out + (static_cast<size_t>(tq) * p.Hq + hq) * 128;
 #pragma unroll 1
-        for (int qd = 0; qd < 4; ++qd) {
+        for (int qd = 2 * half; qd < 2 * half + 2; ++qd) {  // thread (row, half): output columns [64 half, 64 half + 64)
             uint32_t o[32];
             __syncwarp();
             tmem_ld32(lane_addr + 128 + 32 * qd, o);
