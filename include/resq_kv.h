@@ -39,11 +39,16 @@
  *        offset 2304  km   [32][4]   fp32    s8, z8, s4, z4 of the key
  *        offset 2816  v8, offset 3328 v4, offset 5120 vm: the same for the value
  * so one block is one contiguous 5632-byte transfer.  88 bytes per head vector instead of 256 in bf16.
+ * For d_head = 64 every code array is half as wide (k8 [32][8] at 0, k4 [32][28] at 256, km at 1152, the value
+ * half at 1664: 3328 bytes per block, 52 per head vector); resq_kv_block_bytes() gives the block size of a geometry.
  *
  * Conventions are those of resq.h: device pointers unless marked host, caller-owned memory, no allocation,
  * no stream synchronisation, 16-byte aligned pointers, status codes of resq_status_t, arguments validated
- * on the host before anything is enqueued.  d_head must be 128; capacity % 32 == 0;
- * n_q_heads / n_kv_heads must be an integer between 1 and 8.  Indices that live on the device (seq_ids,
+ * on the host before anything is enqueued.  d_head must be 128 or 64; capacity % 32 == 0;
+ * n_q_heads / n_kv_heads must be an integer between 1 and 8.  d_head = 128 runs on the tuned kernels (mma.sync
+ * fragments for the projection and the single-query pass, tcgen05 tiles for the prefill form); d_head = 64 runs the
+ * same arithmetic and cache format on plain kernels (one warp per head vector / per query head, fp32 attention), so
+ * its outputs meet the same bit-exact and tolerance statements but not the same speed.  Indices that live on the device (seq_ids,
  * positions, seq_lens) are checked by the kernels: an out-of-range entry is skipped (a sequence length is
  * clamped to the capacity) and RESQ_ERR_INDEX is reported by resq_device_status.
  */
@@ -63,12 +68,15 @@ extern "C" {
 typedef struct resq_kv_cache {
     int32_t n_seqs;     /* sequences the buffer has room for                     */
     int32_t n_kv_heads; /* KV heads per token                                    */
-    int32_t d_head;     /* 128                                                   */
+    int32_t d_head;     /* 128 or 64                                             */
     int32_t capacity;   /* positions per sequence, a multiple of RESQ_KV_BLOCK   */
     void* data;         /* resq_kv_cache_bytes() bytes, layout above             */
 } resq_kv_cache_t;
 
-/* n_seqs * n_kv_heads * (capacity / 32) * RESQ_KV_BLOCK_BYTES, or 0 for an invalid geometry. */
+/* Bytes of one cache block (32 positions of one KV head, keys and values): 5632 for d_head = 128, 3328 for 64, else 0. */
+size_t resq_kv_block_bytes(int d_head);
+
+/* n_seqs * n_kv_heads * (capacity / 32) * resq_kv_block_bytes(d_head), or 0 for an invalid geometry. */
 size_t resq_kv_cache_bytes(int n_seqs, int n_kv_heads, int d_head, int capacity);
 
 /* Section 5.1 ("U_C ... quantized to 8-bit"): INT8 codes wq [d_head][d_head] and scales s_u [d_head] of

@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libresq.so")
 SOURCES = ["api.cu", "quantize.cu", "quantize_asym.cu", "mixed_gemm.cu", "decode_stream.cu", "project.cu", "static_scratch.cu",
-           "kv_cache.cu", "kv_attention.cu", "kv_prefill.cu", "gptq.cu"]
+           "kv_cache.cu", "kv_attention.cu", "kv_prefill.cu", "kv_d64.cu", "gptq.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -544,9 +544,15 @@ int resq_selftest_wait_runs_out(void* stream) {
 }
 
 // ---- attention-block path (resq_kv.h) ----
+size_t resq_kv_block_bytes(int d_head) {
+    return d_head == 128 ? RESQ_KV_BLOCK_BYTES : d_head == 64 ? kv64_block_bytes() : 0;
+}
+
 size_t resq_kv_cache_bytes(int n_seqs, int n_kv_heads, int d_head, int capacity) {
-    if (n_seqs < 1 || n_kv_heads < 1 || d_head != 128 || capacity < RESQ_KV_BLOCK || capacity % RESQ_KV_BLOCK != 0) return 0;
-    return static_cast<size_t>(n_seqs) * n_kv_heads * (capacity / RESQ_KV_BLOCK) * RESQ_KV_BLOCK_BYTES;
+    if (n_seqs < 1 || n_kv_heads < 1 || (d_head != 128 && d_head != 64) || capacity < RESQ_KV_BLOCK ||
+        capacity % RESQ_KV_BLOCK != 0)
+        return 0;
+    return static_cast<size_t>(n_seqs) * n_kv_heads * (capacity / RESQ_KV_BLOCK) * resq_kv_block_bytes(d_head);
 }
 
 static int check_cache(const resq_kv_cache_t* c) {
@@ -557,20 +563,21 @@ static int check_cache(const resq_kv_cache_t* c) {
 }
 
 int resq_uc_quantize(const float* W_C, int d_head, int8_t* wq, float* s_u, void* stream) {
-    if (d_head != 128) return RESQ_ERR_SHAPE;
+    if (d_head != 128 && d_head != 64) return RESQ_ERR_SHAPE;
     if (!W_C || !wq || !s_u) return RESQ_ERR_NULL;
     if (!aligned16(W_C) || !aligned16(wq) || !aligned16(s_u)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
+    if (d_head == 64) return cuda_status(launch_uc_quantize64(W_C, wq, s_u, static_cast<cudaStream_t>(stream)));
     return cuda_status(launch_uc_quantize(W_C, wq, s_u, static_cast<cudaStream_t>(stream)));
 }
 
 int resq_query_project(const void* q, int64_t rows, int d_head, const int8_t* wq, const float* s_u, void* q_out,
                        void* stream) {
-    if (d_head != 128 || rows < 0) return RESQ_ERR_SHAPE;
+    if ((d_head != 128 && d_head != 64) || rows < 0) return RESQ_ERR_SHAPE;
     if (!q || !wq || !s_u || !q_out) return RESQ_ERR_NULL;
     if (!aligned16(q) || !aligned16(wq) || !aligned16(s_u) || !aligned16(q_out)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
-    return cuda_status(launch_qkv_project_append(nullptr, q, rows, q_out, nullptr, nullptr, 0, nullptr, nullptr, wq, s_u,
+    return cuda_status((d_head == 64 ? launch_qkv_project_append64 : launch_qkv_project_append)(nullptr, q, rows, q_out, nullptr, nullptr, 0, nullptr, nullptr, wq, s_u,
                                                  static_cast<cudaStream_t>(stream)));
 }
 
@@ -581,7 +588,7 @@ int resq_kv_append(const resq_kv_cache_t* cache, const void* k, const void* v, i
     if (!k || !v || !seq_ids || !positions || !wq || !s_u) return RESQ_ERR_NULL;
     if (!aligned16(k) || !aligned16(v) || !aligned16(wq) || !aligned16(s_u)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
-    return cuda_status(launch_qkv_project_append(cache, nullptr, 0, nullptr, k, v, T, seq_ids, positions, wq, s_u,
+    return cuda_status((cache->d_head == 64 ? launch_qkv_project_append64 : launch_qkv_project_append)(cache, nullptr, 0, nullptr, k, v, T, seq_ids, positions, wq, s_u,
                                                  static_cast<cudaStream_t>(stream)));
 }
 
@@ -594,14 +601,15 @@ int resq_qkv_project_append(const resq_kv_cache_t* cache, const void* q, int n_q
     if (!aligned16(q) || !aligned16(q_out) || !aligned16(k) || !aligned16(v) || !aligned16(wq) || !aligned16(s_u))
         return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
-    return cuda_status(launch_qkv_project_append(cache, q, T * n_q_heads, q_out, k, v, T, seq_ids, positions, wq, s_u,
+    return cuda_status((cache->d_head == 64 ? launch_qkv_project_append64 : launch_qkv_project_append)(cache, q, T * n_q_heads, q_out, k, v, T, seq_ids, positions, wq, s_u,
                                                  static_cast<cudaStream_t>(stream)));
 }
 
 size_t resq_attention_workspace_bytes(int n_seqs, int n_q_heads, int n_kv_heads, int d_head) {
-    if (n_seqs < 1 || n_kv_heads < 1 || d_head != 128 || n_q_heads < n_kv_heads || n_q_heads % n_kv_heads != 0 ||
-        n_q_heads / n_kv_heads > 8)
+    if (n_seqs < 1 || n_kv_heads < 1 || (d_head != 128 && d_head != 64) || n_q_heads < n_kv_heads ||
+        n_q_heads % n_kv_heads != 0 || n_q_heads / n_kv_heads > 8)
         return 0;
+    if (d_head == 64) return 256;  // the d_head = 64 kernel keeps its state in registers; a token amount keeps the contract
     return attention_scratch_bytes(n_seqs, n_kv_heads);
 }
 
@@ -614,6 +622,9 @@ int resq_attention_decode(const resq_kv_cache_t* cache, const void* q16, int n_q
     if (!workspace || workspace_bytes < need) return RESQ_ERR_WORKSPACE;
     if (!aligned16(q16) || !aligned16(out) || !aligned16(workspace)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
+    if (cache->d_head == 64)
+        return cuda_status(launch_attention64(*cache, q16, n_q_heads, cache->n_seqs, nullptr, seq_lens, -1, 0, out,
+                                              static_cast<cudaStream_t>(stream)));
     return cuda_status(launch_attention_decode(*cache, q16, n_q_heads, seq_lens, out, workspace,
                                                static_cast<cudaStream_t>(stream)));
 }
@@ -634,6 +645,9 @@ int resq_attention_queries(const resq_kv_cache_t* cache, const void* q16, int n_
     if (!workspace || workspace_bytes < need) return RESQ_ERR_WORKSPACE;
     if (!aligned16(q16) || !aligned16(out) || !aligned16(workspace)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
+    if (cache->d_head == 64)
+        return cuda_status(launch_attention64(*cache, q16, n_q_heads, n_queries, q_seq, q_len, -1, 0, out,
+                                              static_cast<cudaStream_t>(stream)));
     return cuda_status(launch_attention_decode(*cache, q16, n_q_heads, q_len, out, workspace,
                                                static_cast<cudaStream_t>(stream), n_queries, q_seq));
 }
@@ -646,6 +660,9 @@ int resq_attention_prefill(const resq_kv_cache_t* cache, const void* q16, int n_
     if (!q16 || !out) return RESQ_ERR_NULL;
     if (!aligned16(q16) || !aligned16(out)) return RESQ_ERR_ALIGN;
     if (int e = check_arch()) return e;
+    if (cache->d_head == 64)
+        return cuda_status(launch_attention64(*cache, q16, n_q_heads, T, nullptr, nullptr, seq, pos0, out,
+                                              static_cast<cudaStream_t>(stream)));
     return cuda_status(launch_attention_prefill(*cache, q16, n_q_heads, seq, pos0, T, out, static_cast<cudaStream_t>(stream)));
 }
 

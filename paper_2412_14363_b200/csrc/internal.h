@@ -96,6 +96,18 @@ cudaError_t launch_attention_decode(const resq_kv_cache_t& cache, const void* q1
 cudaError_t launch_attention_prefill(const resq_kv_cache_t& cache, const void* q16, int n_q_heads, int seq, int pos0,
                                      int T, float* out, cudaStream_t st);
 
+// d_head = 64 (plain kernels, same arithmetic and cache format with every code array halved).
+size_t kv64_block_bytes();
+cudaError_t launch_uc_quantize64(const float* W_C, int8_t* wq, float* s_u, cudaStream_t st);
+cudaError_t launch_qkv_project_append64(const resq_kv_cache_t* cache, const void* q, long long q_rows, void* q_out,
+                                        const void* k, const void* v, long long T, const int32_t* seq_ids,
+                                        const int32_t* positions, const int8_t* wq, const float* s_u, cudaStream_t st);
+// Row i of q16 / out attends the first len_of_row[i] (null: len0 + i + 1) positions of sequence seq_of_row[i] (null:
+// seq_const if >= 0, else i).
+cudaError_t launch_attention64(const resq_kv_cache_t& cache, const void* q16, int n_q_heads, int rows,
+                               const int32_t* seq_of_row, const int32_t* len_of_row, int seq_const, int len0, float* out,
+                               cudaStream_t st);
+
 // Driver entry point for tensor-map encoding (resolved once, without linking libcuda).
 void* tensor_map_encode_fn();
 

@@ -6,7 +6,7 @@ import ctypes
 from . import ERR_CUDA, ERR_INDEX, OK, ResqError, _check, _ptr, _stream, lib  # noqa: F401
 
 KV_BLOCK, KV_BLOCK_BYTES = 32, 5632
-KV_EXPORTS = ["resq_kv_cache_bytes", "resq_uc_quantize", "resq_query_project", "resq_kv_append", "resq_qkv_project_append",
+KV_EXPORTS = ["resq_kv_block_bytes", "resq_kv_cache_bytes", "resq_uc_quantize", "resq_query_project", "resq_kv_append", "resq_qkv_project_append",
               "resq_attention_workspace_bytes", "resq_attention_decode", "resq_attention_queries_workspace_bytes",
               "resq_attention_queries", "resq_attention_prefill"]
 
@@ -18,6 +18,8 @@ class KvCacheStruct(ctypes.Structure):
 
 _vp, _sz, _i, _i64 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_int64
 _cp = ctypes.POINTER(KvCacheStruct)
+lib.resq_kv_block_bytes.restype = _sz
+lib.resq_kv_block_bytes.argtypes = [_i]
 lib.resq_kv_cache_bytes.restype = _sz
 lib.resq_kv_cache_bytes.argtypes = [_i, _i, _i, _i]
 lib.resq_uc_quantize.argtypes = [_vp, _i, _vp, _vp, _vp]

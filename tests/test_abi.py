@@ -72,14 +72,16 @@ def test_kv_host_validation(resq):
     from paper_2412_14363_b200 import kv
     L = resq.lib
     assert L.resq_kv_cache_bytes(2, 8, 128, 64) == 2 * 8 * 2 * 5632
-    assert L.resq_kv_cache_bytes(2, 8, 64, 64) == 0 and L.resq_kv_cache_bytes(2, 8, 128, 48) == 0
+    assert L.resq_kv_cache_bytes(2, 8, 64, 64) == 2 * 8 * 2 * 3328    # d_head = 64: every code array halved
+    assert L.resq_kv_block_bytes(128) == 5632 and L.resq_kv_block_bytes(64) == 3328 and L.resq_kv_block_bytes(96) == 0
+    assert L.resq_kv_cache_bytes(2, 8, 96, 64) == 0 and L.resq_kv_cache_bytes(2, 8, 128, 48) == 0
     assert L.resq_kv_cache_bytes(0, 8, 128, 64) == 0
     assert L.resq_attention_workspace_bytes(4, 32, 8, 128) > 0
     assert L.resq_attention_workspace_bytes(4, 30, 8, 128) == 0      # not a multiple of the KV heads
     assert L.resq_attention_workspace_bytes(4, 72, 8, 128) == 0      # more than 8 query heads per KV head
     fake = 1 << 20
     c = kv.KvCacheStruct(2, 8, 128, 64, fake)
-    assert L.resq_uc_quantize(fake, 64, fake, fake, None) == resq.ERR_SHAPE
+    assert L.resq_uc_quantize(fake, 96, fake, fake, None) == resq.ERR_SHAPE
     assert L.resq_uc_quantize(None, 128, fake, fake, None) == resq.ERR_NULL
     assert L.resq_query_project(fake, 5, 128, fake, fake + 4, fake, None) == resq.ERR_ALIGN
     assert L.resq_query_project(fake, -1, 128, fake, fake, fake, None) == resq.ERR_SHAPE
