@@ -230,11 +230,11 @@ __device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint3
 template <bool F32>
 __global__ void __launch_bounds__(kThreads)
 split_quantize_fast_kernel(const void* __restrict__ in, size_t in_row_bytes, size_t rows, int K, int r,
-                           int rows_per_cta, int8_t* __restrict__ q8, uint8_t* __restrict__ q4,
+                           int rows_per_cta, int nstages, int8_t* __restrict__ q8, uint8_t* __restrict__ q4,
                            float* __restrict__ s8_out, float* __restrict__ s4_out, int8_t* __restrict__ q4e,
                            int* __restrict__ status) {
     extern __shared__ __align__(128) uint8_t stage[];
-    __shared__ uint64_t bar;
+    __shared__ uint64_t bar[2];
     __shared__ int abort_flag;
     __shared__ float red[2][kThreads / 32];
     // A kernel enqueued behind this one with programmatic stream serialization may start its own
@@ -244,129 +244,157 @@ split_quantize_fast_kernel(const void* __restrict__ in, size_t in_row_bytes, siz
     // scheduled before its input was complete: wait for the preceding grid (returns at once otherwise).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t row_bytes = static_cast<uint32_t>(K) * (F32 ? 4u : 2u);
-    const size_t row0 = static_cast<size_t>(blockIdx.x) * rows_per_cta;
-    const int nrows = static_cast<int>(rows - row0 < static_cast<size_t>(rows_per_cta) ? rows - row0 : rows_per_cta);
+    const size_t group_bytes = static_cast<size_t>(row_bytes) * rows_per_cta;
+    const size_t groups = (rows + rows_per_cta - 1) / rows_per_cta;
+    auto rows_of = [&](size_t g) {
+        const size_t row0 = g * rows_per_cta;
+        return static_cast<int>(rows - row0 < static_cast<size_t>(rows_per_cta) ? rows - row0 : rows_per_cta);
+    };
+    auto issue = [&](size_t g, int buf) {  // one thread: the rows of group g, one bulk copy each
+        const int n = rows_of(g);
+        mbar_arrive_expect_tx(&bar[buf], row_bytes * static_cast<uint32_t>(n));
+        for (int i = 0; i < n; ++i)
+            bulk_load(stage + buf * group_bytes + static_cast<size_t>(i) * row_bytes,
+                      reinterpret_cast<const char*>(in) + (g * rows_per_cta + i) * in_row_bytes, row_bytes, &bar[buf]);
+    };
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        mbar_init(&bar, 1);
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
         fence_mbar_init();
-        mbar_arrive_expect_tx(&bar, row_bytes * static_cast<uint32_t>(nrows));
-        for (int i = 0; i < nrows; ++i)
-            bulk_load(stage + static_cast<size_t>(i) * row_bytes,
-                      reinterpret_cast<const char*>(in) + (row0 + i) * in_row_bytes, row_bytes, &bar);
+        if (blockIdx.x < groups) issue(blockIdx.x, 0);
     }
     __syncthreads();
-    const bool landed = mbar_wait(&bar, 0, &abort_flag, status);
-    if (__syncthreads_or(!landed)) {
-        // The copy did not land in time: report it and leave the outputs of this group unwritten.
-        if (threadIdx.x == 0) atomicOr(status, kStatusBitTimeout);
-        return;
-    }
 
     const int tpr = kThreads / rows_per_cta;  // threads per row, a multiple of 32
     const int grp = threadIdx.x / tpr, j = threadIdx.x - grp * tpr;
     const int nchunks = K >> 3, rchunks = r >> 3;
     const int K4 = K - r;
-    const bool live = grp < nrows;
-    const uint8_t* srow = stage + static_cast<size_t>(live ? grp : 0) * row_bytes;
 
-    float a8 = 0.f, a4 = 0.f;
-    if (live) {
-        if constexpr (F32) {
-            for (int c = j; c < rchunks; c += tpr) a8 = fmaxf(a8, chunk_absmax(lds_chunk<F32>(srow, c)));
-            float m0 = 0.f, m1 = 0.f;  // two chains: the INT4 segment is 7/8 of the row
-            int c = rchunks + j;
-            for (; c + tpr < nchunks; c += 2 * tpr) {
-                m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
-                m1 = fmaxf(m1, chunk_absmax(lds_chunk<F32>(srow, c + tpr)));
+    // The CTA walks its groups (grid-stride); with two stages the rows of the next group are in flight while this
+    // one is quantized, so the copy engine never waits for the arithmetic of the same CTA.
+    int it = 0;
+    for (size_t g = blockIdx.x; g < groups; g += gridDim.x, ++it) {
+        const int buf = nstages == 2 ? (it & 1) : 0;
+        const uint32_t parity = nstages == 2 ? (it >> 1) & 1 : it & 1;
+        const bool more = g + gridDim.x < groups;
+        if (nstages == 2 && more && threadIdx.x == 0) issue(g + gridDim.x, buf ^ 1);
+        const bool landed = mbar_wait(&bar[buf], parity, &abort_flag, status);
+        if (__syncthreads_or(!landed)) {
+            // The copy did not land in time: report it and leave the outputs of the remaining groups unwritten.
+            if (threadIdx.x == 0) {
+                atomicOr(status, kStatusBitTimeout);
+                if (nstages == 2 && more) {  // the copies of the next group are still this CTA's to wait for
+                    int keep_waiting = 0;
+                    (void)mbar_wait(&bar[buf ^ 1], ((it + 1) >> 1) & 1, &keep_waiting, status);
+                }
             }
-            if (c < nchunks) m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
-            a4 = fmaxf(m0, m1);
-        } else {
-            // bf16 rows: sign bits cleared, maxima kept as packed pairs until the end (two operations per pair)
-            const uint4* v = reinterpret_cast<const uint4*>(srow);
-            uint32_t m8 = 0, m4a = 0, m4b = 0;
-            auto acc = [](uint32_t& m, const uint4 u) {
-                const uint32_t w[4] = {u.x & 0x7FFF7FFFu, u.y & 0x7FFF7FFFu, u.z & 0x7FFF7FFFu, u.w & 0x7FFF7FFFu};
-                __nv_bfloat162 mm = *reinterpret_cast<const __nv_bfloat162*>(&m);
+            return;
+        }
+        const int nrows = rows_of(g);
+        const size_t row0 = g * rows_per_cta;
+        const bool live = grp < nrows;
+        const uint8_t* srow = stage + buf * group_bytes + static_cast<size_t>(live ? grp : 0) * row_bytes;
+
+        float a8 = 0.f, a4 = 0.f;
+        if (live) {
+            if constexpr (F32) {
+                for (int c = j; c < rchunks; c += tpr) a8 = fmaxf(a8, chunk_absmax(lds_chunk<F32>(srow, c)));
+                float m0 = 0.f, m1 = 0.f;  // two chains: the INT4 segment is 7/8 of the row
+                int c = rchunks + j;
+                for (; c + tpr < nchunks; c += 2 * tpr) {
+                    m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
+                    m1 = fmaxf(m1, chunk_absmax(lds_chunk<F32>(srow, c + tpr)));
+                }
+                if (c < nchunks) m0 = fmaxf(m0, chunk_absmax(lds_chunk<F32>(srow, c)));
+                a4 = fmaxf(m0, m1);
+            } else {
+                // bf16 rows: sign bits cleared, maxima kept as packed pairs until the end (two operations per pair)
+                const uint4* v = reinterpret_cast<const uint4*>(srow);
+                uint32_t m8 = 0, m4a = 0, m4b = 0;
+                auto acc = [](uint32_t& m, const uint4 u) {
+                    const uint32_t w[4] = {u.x & 0x7FFF7FFFu, u.y & 0x7FFF7FFFu, u.z & 0x7FFF7FFFu, u.w & 0x7FFF7FFFu};
+                    __nv_bfloat162 mm = *reinterpret_cast<const __nv_bfloat162*>(&m);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) mm = __hmax2(mm, *reinterpret_cast<const __nv_bfloat162*>(&w[i]));
-                m = *reinterpret_cast<const uint32_t*>(&mm);
-            };
-            for (int c = j; c < rchunks; c += tpr) acc(m8, v[c]);
-            int c = rchunks + j;
+                    for (int i = 0; i < 4; ++i) mm = __hmax2(mm, *reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+                    m = *reinterpret_cast<const uint32_t*>(&mm);
+                };
+                for (int c = j; c < rchunks; c += tpr) acc(m8, v[c]);
+                int c = rchunks + j;
 #pragma unroll 2
-            for (; c + tpr < nchunks; c += 2 * tpr) {
-                acc(m4a, v[c]);
-                acc(m4b, v[c + tpr]);
+                for (; c + tpr < nchunks; c += 2 * tpr) {
+                    acc(m4a, v[c]);
+                    acc(m4b, v[c + tpr]);
+                }
+                if (c < nchunks) acc(m4a, v[c]);
+                auto unpack = [](uint32_t m) { return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u)); };
+                a8 = unpack(m8);
+                a4 = fmaxf(unpack(m4a), unpack(m4b));
             }
-            if (c < nchunks) acc(m4a, v[c]);
-            auto unpack = [](uint32_t m) { return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u)); };
-            a8 = unpack(m8);
-            a4 = fmaxf(unpack(m4a), unpack(m4b));
         }
-    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        a8 = fmaxf(a8, __shfl_xor_sync(0xffffffffu, a8, o));
-        a4 = fmaxf(a4, __shfl_xor_sync(0xffffffffu, a4, o));
-    }
-    if (tpr > 32) {
-        const int warp = threadIdx.x >> 5, wpr = tpr >> 5;
-        if ((threadIdx.x & 31) == 0) {
-            red[0][warp] = a8;
-            red[1][warp] = a4;
+        for (int o = 16; o > 0; o >>= 1) {
+            a8 = fmaxf(a8, __shfl_xor_sync(0xffffffffu, a8, o));
+            a4 = fmaxf(a4, __shfl_xor_sync(0xffffffffu, a4, o));
         }
-        __syncthreads();
-        for (int w = 0; w < wpr; ++w) {
-            a8 = fmaxf(a8, red[0][grp * wpr + w]);
-            a4 = fmaxf(a4, red[1][grp * wpr + w]);
+        if (tpr > 32) {
+            const int warp = threadIdx.x >> 5, wpr = tpr >> 5;
+            if ((threadIdx.x & 31) == 0) {
+                red[0][warp] = a8;
+                red[1][warp] = a4;
+            }
+            __syncthreads();
+            for (int w = 0; w < wpr; ++w) {
+                a8 = fmaxf(a8, red[0][grp * wpr + w]);
+                a4 = fmaxf(a4, red[1][grp * wpr + w]);
+            }
         }
-    }
-    if (!live) return;
+        if (live) {
+            const size_t row = row0 + grp;
+            const float s8 = __fdiv_rn(a8, 127.f), s4 = __fdiv_rn(a4, 7.f);
+            const float inv8 = s8 > 0.f ? __frcp_rn(s8) : 0.f, inv4 = s4 > 0.f ? __frcp_rn(s4) : 0.f;
+            // The product form needs a finite, normal reciprocal; otherwise every chunk takes the division.
+            const bool exact8 = s8 > 0.f && !(inv8 >= 1.1754944e-38f && inv8 <= 3.0e38f);
+            const bool exact4 = s4 > 0.f && !(inv4 >= 1.1754944e-38f && inv4 <= 3.0e38f);
+            if (j == 0) {
+                s8_out[row] = s8;
+                s4_out[row] = s4;
+            }
+            int8_t* q8row = q8 + row * static_cast<size_t>(r);
+            uint8_t* q4row = q4 ? q4 + row * static_cast<size_t>(K4 >> 1) : nullptr;
+            int8_t* q4e_row = q4e ? q4e + row * static_cast<size_t>(K4) : nullptr;
 
-    const size_t row = row0 + grp;
-    const float s8 = __fdiv_rn(a8, 127.f), s4 = __fdiv_rn(a4, 7.f);
-    const float inv8 = s8 > 0.f ? __frcp_rn(s8) : 0.f, inv4 = s4 > 0.f ? __frcp_rn(s4) : 0.f;
-    // The product form needs a finite, normal reciprocal; otherwise every chunk takes the division.
-    const bool exact8 = s8 > 0.f && !(inv8 >= 1.1754944e-38f && inv8 <= 3.0e38f);
-    const bool exact4 = s4 > 0.f && !(inv4 >= 1.1754944e-38f && inv4 <= 3.0e38f);
-    if (j == 0) {
-        s8_out[row] = s8;
-        s4_out[row] = s4;
-    }
-    int8_t* q8row = q8 + row * static_cast<size_t>(r);
-    uint8_t* q4row = q4 ? q4 + row * static_cast<size_t>(K4 >> 1) : nullptr;
-    int8_t* q4e_row = q4e ? q4e + row * static_cast<size_t>(K4) : nullptr;
-
-    for (int c = j; c < rchunks; c += tpr) {
-        uint32_t t[8];
-        if (s8 > 0.f) fast_codes(lds_chunk<F32>(srow, c), s8, inv8, exact8, t);
-        else {
+            for (int c = j; c < rchunks; c += tpr) {
+                uint32_t t[8];
+                if (s8 > 0.f) fast_codes(lds_chunk<F32>(srow, c), s8, inv8, exact8, t);
+                else {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) t[k] = 0;
-        }
-        *reinterpret_cast<uint2*>(q8row + c * 8) =
-            make_uint2(pack_low_bytes(t[0], t[1], t[2], t[3]), pack_low_bytes(t[4], t[5], t[6], t[7]));
-    }
+                    for (int k = 0; k < 8; ++k) t[k] = 0;
+                }
+                *reinterpret_cast<uint2*>(q8row + c * 8) =
+                    make_uint2(pack_low_bytes(t[0], t[1], t[2], t[3]), pack_low_bytes(t[4], t[5], t[6], t[7]));
+            }
 #pragma unroll 2
-    for (int c = rchunks + j; c < nchunks; c += tpr) {
-        uint32_t t[8];
-        if (s4 > 0.f) fast_codes(lds_chunk<F32>(srow, c), s4, inv4, exact4, t);
-        else {
+            for (int c = rchunks + j; c < nchunks; c += tpr) {
+                uint32_t t[8];
+                if (s4 > 0.f) fast_codes(lds_chunk<F32>(srow, c), s4, inv4, exact4, t);
+                else {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) t[k] = 0;
+                    for (int k = 0; k < 8; ++k) t[k] = 0;
+                }
+                const int jj = (c - rchunks) * 8;
+                const uint32_t lo = pack_low_bytes(t[0], t[1], t[2], t[3]), hi = pack_low_bytes(t[4], t[5], t[6], t[7]);
+                if (q4e_row) *reinterpret_cast<uint2*>(q4e_row + jj) = make_uint2(lo, hi);
+                if (q4row) {
+                    // two's-complement nibbles of the eight bytes: byte pairs (b0 | b1 << 4) sit in bytes 0 and 2 of
+                    // x | x >> 4 once the high nibbles are cleared
+                    const uint32_t xl = lo & 0x0F0F0F0Fu, xh = hi & 0x0F0F0F0Fu;
+                    *reinterpret_cast<uint32_t*>(q4row + (jj >> 1)) = __byte_perm(xl | (xl >> 4), xh | (xh >> 4), 0x6420);
+                }
+            }
         }
-        const int jj = (c - rchunks) * 8;
-        if (q4e_row)
-            *reinterpret_cast<uint2*>(q4e_row + jj) =
-                make_uint2(pack_low_bytes(t[0], t[1], t[2], t[3]), pack_low_bytes(t[4], t[5], t[6], t[7]));
-        if (q4row) {
-            uint32_t packed = 0;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) packed |= (t[k] & 0xFu) << (4 * k);
-            *reinterpret_cast<uint32_t*>(q4row + (jj >> 1)) = packed;
-        }
+        __syncthreads();  // every thread is done with this stage (and with `red`) before it is refilled
+        if (nstages == 1 && more && threadIdx.x == 0) issue(g + gridDim.x, 0);
     }
 }
 
@@ -632,10 +660,12 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
     if (rows == 0) return cudaSuccess;
     const size_t row_bytes = static_cast<size_t>(K) * (in_is_f32 ? 4 : 2);
     if (!scale_fp16 && row_bytes <= static_cast<size_t>(kFastMaxRowBytes) && in_row_stride_bytes % 16 == 0) {
-        int rpc = 1;  // rows per CTA: 1, 2, 4 or 8, about kFastGroupBytes of staging
+        int rpc = 1;  // rows per CTA and step: 1, 2, 4 or 8, about half of kFastGroupBytes of staging
         while (rpc < 8 && row_bytes * rpc * 2 <= static_cast<size_t>(kFastGroupBytes)) rpc *= 2;
         while (rpc > 1 && rows / rpc < 148) rpc /= 2;  // few rows (a generation step): all threads of a CTA on one row
-        const size_t smem = row_bytes * rpc;
+        const size_t groups = (rows + rpc - 1) / rpc;
+        const size_t group_bytes = row_bytes * rpc;
+        // Two stages when they are cheap (several CTAs per SM still fit) and a CTA has more than one group to do.
         auto kern = in_is_f32 ? split_quantize_fast_kernel<true> : split_quantize_fast_kernel<false>;
         static bool attr_set[2][64] = {};
         int dev = 0;
@@ -646,12 +676,22 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
             if (e != cudaSuccess) return e;
             attr_set[in_is_f32][dev] = true;
         }
-        const size_t groups = (rows + rpc - 1) / rpc;
-        if (groups <= 0x7fffffffu) {
+        auto ctas_per_sm = [](size_t smem) {  // shared memory and the 2048-thread limit; registers allow 8 CTAs of 256
+            const size_t by_smem = (227u * 1024u) / (smem + 1024u);
+            return by_smem < 1 ? size_t(1) : (by_smem > 8 ? size_t(8) : by_smem);
+        };
+        int nstages = 1;
+        size_t grid = 148 * ctas_per_sm(group_bytes);
+        if (groups > grid && 2 * group_bytes <= 64u * 1024u) {
+            nstages = 2;
+            grid = 148 * ctas_per_sm(2 * group_bytes);
+        }
+        if (grid > groups) grid = groups;
+        {
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(static_cast<unsigned>(groups), 1, 1);
+            cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
             cfg.blockDim = dim3(kThreads, 1, 1);
-            cfg.dynamicSmemBytes = smem;
+            cfg.dynamicSmemBytes = group_bytes * nstages;
             cfg.stream = st;
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -662,7 +702,7 @@ cudaError_t launch_split_quantize(const void* in, bool in_is_f32, size_t rows, i
             (void)programmatic;
             cfg.numAttrs = 1;
             count_launch();
-            return cudaLaunchKernelEx(&cfg, kern, in, in_row_stride_bytes, rows, K, r, rpc, q8, q4,
+            return cudaLaunchKernelEx(&cfg, kern, in, in_row_stride_bytes, rows, K, r, rpc, nstages, q8, q4,
                                       static_cast<float*>(s8), static_cast<float*>(s4), q4_i8, device_status_ptr());
         }
     }

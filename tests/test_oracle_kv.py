@@ -71,22 +71,24 @@ def test_query_kept_in_half_precision():
     assert float(h[0, 0]) == 1.0 and float(h[0, 1]) == 1.0 + 2.0 ** -9 and float(h[0, 2]) == 65504.0  # ties to even
 
 
-def test_kv_quantize_layout_and_bounds():
+@pytest.mark.parametrize("d", [128, 64])
+def test_kv_quantize_layout_and_bounds(d):
+    """The first d/8 coefficients in 8 bits, the rest in 4 (d = 128 and the 64-wide heads of the small model)."""
     rng = np.random.default_rng(6)
-    d, rows = 128, 11
-    Y = (rng.standard_normal((rows, d)) * np.r_[np.full(16, 8.0), np.ones(112)] + 0.7).astype(np.float32)
+    rows, r = 11, d // 8
+    Y = (rng.standard_normal((rows, d)) * np.r_[np.full(r, 8.0), np.ones(d - r)] + 0.7).astype(np.float32)
     h = kv.kv_quantize(Y)
-    assert h.c8.shape == (rows, 16) and h.u4.shape == (rows, 112) and h.c4.shape == (rows, 56) and h.meta.shape == (rows, 4)
+    assert h.c8.shape == (rows, r) and h.u4.shape == (rows, d - r) and h.c4.shape == (rows, (d - r) // 2) and h.meta.shape == (rows, 4)
     assert h.u4.max() == 15 and h.c8.max() == 255 and h.c8.min() == 0 and h.u4.min() == 0
     for t in range(rows):
         s8, z8, s4, z4 = (np.float32(v) for v in h.meta[t])
-        assert z8 == Y[t, :16].min() and z4 == Y[t, 16:].min()
-        assert s8 == (Y[t, :16].max() - Y[t, :16].min()) / np.float32(255)
-        assert s4 == (Y[t, 16:].max() - Y[t, 16:].min()) / np.float32(15)
-        assert h.c8[t, Y[t, :16].argmax()] == 255 and h.u4[t, Y[t, 16:].argmin()] == 0
+        assert z8 == Y[t, :r].min() and z4 == Y[t, r:].min()
+        assert s8 == (Y[t, :r].max() - Y[t, :r].min()) / np.float32(255)
+        assert s4 == (Y[t, r:].max() - Y[t, r:].min()) / np.float32(15)
+        assert h.c8[t, Y[t, :r].argmax()] == 255 and h.u4[t, Y[t, r:].argmin()] == 0
     xh = kv.kv_dequantize(h)
     err = np.abs(xh - Y)
-    assert (err[:, :16] <= h.meta[:, 0:1] / 2 * (1 + 1e-4)).all() and (err[:, 16:] <= h.meta[:, 2:3] / 2 * (1 + 1e-4)).all()
+    assert (err[:, :r] <= h.meta[:, 0:1] / 2 * (1 + 1e-4)).all() and (err[:, r:] <= h.meta[:, 2:3] / 2 * (1 + 1e-4)).all()
     # two codes per byte, code 2i in the low nibble
     assert (h.c4 == (h.u4[:, 0::2] | (h.u4[:, 1::2] << 4))).all()
 
