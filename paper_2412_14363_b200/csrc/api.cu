@@ -420,6 +420,28 @@ static int mixed_gemm_asym_impl(const resq_layer_desc_t* d, int T, const uint8_t
                                                        d->w_scale_dtype == RESQ_SCALE_FP16, Y, y_dtype, dbg8, dbg4, st,
                                                        z_x8, z_x4, wsum8, wsum4);
         if (e != cudaErrorNotSupported) return cuda_status(e);
+        if (T > 8) {
+            // Rows too wide to stage 9-16 tokens beside the weight rings: two launches of at most 8 tokens, as in the
+            // symmetric path (the tile kernel below would read one byte per INT4 weight for these few rows).
+            const size_t ysz = y_dtype == RESQ_Y_BF16 ? 2 : 4;
+            bool done = true;
+            for (int t0 = 0; t0 < T && done; t0 += 8) {
+                const int rows = T - t0 < 8 ? T - t0 : 8;
+                const cudaError_t e2 = launch_mixed_gemm_stream(
+                    rows, d->n_out, d->K, d->r, u8 ? reinterpret_cast<const int8_t*>(u8) + static_cast<size_t>(t0) * d->r : nullptr,
+                    u4 + static_cast<size_t>(t0) * (K4 / 2), s_x8 + t0, s_x4 + t0, W->w8, W->w4, W->s_w8, W->s_w4,
+                    d->w_scale_dtype == RESQ_SCALE_FP16, static_cast<char*>(Y) + static_cast<size_t>(t0) * d->n_out * ysz,
+                    y_dtype, dbg8 ? dbg8 + static_cast<size_t>(t0) * d->n_out : nullptr,
+                    dbg4 ? dbg4 + static_cast<size_t>(t0) * d->n_out : nullptr, st, z_x8 + t0, z_x4 + t0, wsum8, wsum4);
+                if (e2 == cudaErrorNotSupported) {
+                    if (t0 > 0) return RESQ_ERR_SHAPE;  // cannot happen: the plan does not depend on the row offset
+                    done = false;
+                } else if (e2 != cudaSuccess) {
+                    return cuda_status(e2);
+                }
+            }
+            if (done) return RESQ_OK;
+        }
     }
     const int8_t* x4e = reinterpret_cast<const int8_t*>(u4e_ready);
     if (!x4e) {

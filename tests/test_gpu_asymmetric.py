@@ -189,6 +189,8 @@ def test_asym_online_projection(resq):
     (3, 1056, 72, 96, False),        # segment lengths that are not multiples of a step
     (16, 14336, 256, 1792, True),    # down_proj reduction length
     (2, 4096, 8, 512, False),        # a single unit
+    (16, 28672, 64, 3584, False),    # rows too wide to stage 9-16 tokens: two launches of 8 tokens
+    (11, 28672, 72, 0, False),       # ... 8 + 3 tokens, uniform INT4, ragged channel block
 ])
 def test_asym_decode_bit_exact(resq, T, K, N, r, fp16):
     """T <= 16 with packed codes: the weight-streaming kernel with unsigned activation codes."""
