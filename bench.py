@@ -303,6 +303,28 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
         l1 = ev()
         torch.cuda.synchronize()
         total_linear = l0.elapsed_time(l1) / steps
+        # The same calls recorded once into a CUDA graph (one graph = DECODE_COPIES steps, so that the weight copies
+        # still cycle) and replayed: the library allocates nothing and never synchronises, so its calls can be captured.
+        total_graph = None
+        try:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(DECODE_COPIES):
+                    linear_chain(i)
+            reps = max(1, steps // DECODE_COPIES)
+            for _ in range(2):
+                g.replay()
+            torch.cuda.synchronize()
+            torch.cuda._sleep(HOST_LEAD_CYCLES)
+            g0 = ev()
+            for _ in range(reps):
+                g.replay()
+            g1 = ev()
+            torch.cuda.synchronize()
+            total_graph = g0.elapsed_time(g1) / (reps * DECODE_COPIES)
+        except RuntimeError as e:
+            print(f"[bench] graph capture of the few-token block failed: {e}", file=sys.stderr)
+            torch.cuda.synchronize()
         # The same block with the Hadamard form of the online layer(s).
         hb = {}
         for (L, desc, _), b in zip(sets, bufs):
@@ -378,6 +400,7 @@ def decode_leg(resq, torch, dev, peaks, layers, steps):
                         "block_split_calls_us": round(total * 1e3, 2),
                         "block_linears_us": round(total_linear * 1e3, 2),
                         "tokens_per_s": round(T / (total_linear * 1e-3), 1),
+                        "block_linears_cuda_graph_us": round(total_graph * 1e3, 2) if total_graph else None,
                         "block_linears_hadamard_down_us": round(total_hadamard * 1e3, 2) if total_hadamard else None,
                         "tokens_per_s_hadamard_down": round(T / (total_hadamard * 1e-3), 1) if total_hadamard else None}
     resq.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 0)

@@ -192,3 +192,46 @@ def test_decode_linear_with_online_projection(resq, T, K, N, r):
     e32, ebf = oracle.epilogue(acc8, acc4, gs8, gs4, pw.s8, pw.s4)
     res = oracle.LayerResult(None, g8.astype(np.int8), g4.astype(np.int8), None, gs8, gs4, acc8, acc4, e32, ebf)
     check_output(res, pw, host(y32), bf16_bits_from_dev(ybf))
+
+
+def test_decode_layers_replay_from_a_cuda_graph(resq):
+    """The library allocates nothing and never synchronises, so its calls can be recorded into a CUDA graph (the way a
+    generation loop removes its launch overhead): two layers of a step -- one folded, one with the online projection --
+    are captured once, the inputs are overwritten in place, and the replay gives, bit for bit, what direct calls give
+    on the new inputs (and differs from the captured run's outputs)."""
+    T, K, N, r = 4, 2304, 264, 288
+    desc = resq.layer_desc(K, N, r, resq.SCALE_FP16)
+    Wp = synth.projected_weights_direct(N, K, seed=1401)
+    W = resq.resq_pack_weights(desc, dev(Wp), with_w4_i8=False)
+    P = bf16_to_dev(synth.f32_to_bf16_bits(synth.kron_orthogonal_bf16(K, inner=32)))
+    ws_f, ws_p = resq.alloc_workspace(desc, T, False, False), resq.alloc_workspace(desc, T, True, False)
+    X = bf16_to_dev(synth.f32_to_bf16_bits(synth.activations(T, K, "t4", seed=1402)))
+    X2 = bf16_to_dev(synth.f32_to_bf16_bits(synth.activations(T, K, "t4", seed=1403)))
+    y_f = torch.zeros((T, N), dtype=torch.float32, device="cuda")
+    y_p = torch.zeros((T, N), dtype=torch.float32, device="cuda")
+    resq.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 1)
+    try:
+        for _ in range(2):                       # first calls set function attributes: not inside a capture
+            resq.resq_linear(W, X, None, y_f, ws_f)
+            resq.resq_linear(W, X, P, y_p, ws_p)
+        torch.cuda.synchronize()
+        first = host(y_f).copy(), host(y_p).copy()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            resq.resq_linear(W, X, None, y_f, ws_f)
+            resq.resq_linear(W, X, P, y_p, ws_p)
+        X.copy_(X2)
+        y_f.fill_(float("nan"))
+        y_p.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        got = host(y_f).copy(), host(y_p).copy()
+        resq.resq_linear(W, X2, None, y_f, ws_f)
+        resq.resq_linear(W, X2, P, y_p, ws_p)
+        assert resq.resq_device_status() == resq.OK
+        want = host(y_f), host(y_p)
+    finally:
+        resq.resq_set_option(resq.OPT_DECODE_EARLY_WEIGHTS, 0)
+    for a, b, c in zip(got, want, first):
+        assert np.isfinite(a).all() and (a.view(np.uint32) == b.view(np.uint32)).all()
+        assert (a != c).any()
