@@ -152,3 +152,52 @@ def test_attention_full_size_sampled_heads():
             ref = okv.attention_decode(q16_h[b:b + 1, hq:hq + 1], [[dk[:, hk_i]]], [[dv[:, hk_i]]], [n], 1, 1)[0, 0]
             vmax = np.abs(dv[:n, hk_i]).max()
             assert np.abs(out_h[b, hq] - ref).max() <= 1e-3 * vmax, (b, hq)
+
+
+def test_prefill_attention_full_size_sampled_rows():
+    """Causal attention of new tokens at the benchmark's size and launch shapes (Llama-3-8B geometry, one sequence of
+    8192 positions): the whole sequence in one call (2048 tiles) and its last 1024 tokens (256 tiles).  Sampled
+    (token, query head) rows -- first and last rows of tiles, rows on both sides of a 64-position step boundary, the
+    very first and last tokens -- against the oracle's fp64 definition on the oracle's own codes, within 1e-3 of the
+    value magnitude; the two calls agree on the rows they share to the same bound."""
+    import paper_2412_14363_b200 as resq
+    from oracle import kv as okv
+    from paper_2412_14363_b200 import kv
+    from tests.gpu_util import dev as to_dev
+
+    S, Hq, Hkv, D, Tc = 8192, 32, 8, 128, 1024
+    device = torch.device("cuda")
+    W_C = np.ascontiguousarray(synth.haar_orthogonal(D).T.astype(np.float32))
+    wq, s_u = kv.resq_uc_quantize(to_dev(W_C))
+    cache = kv.KvCache(2, Hkv, S)
+    cache.data.fill_(0xFF)
+    k = synth.t_head_vectors(S, Hkv, D, device, stream=5000, lead=1.0, scale=1.5)
+    v = synth.t_head_vectors(S, Hkv, D, device, stream=5001, lead=4.0, shift=0.2)
+    kv.resq_kv_append(cache, k, v, torch.ones(S, dtype=torch.int32, device=device),
+                      torch.arange(S, dtype=torch.int32, device=device), wq, s_u)
+    q = synth.t_head_vectors(S, Hq, D, device, stream=5002, lead=1.0, scale=1.5)
+    q16 = torch.empty((S, Hq, D), dtype=torch.float16, device=device)
+    kv.resq_query_project(q, wq, s_u, q16)
+    out = torch.full((S, Hq, D), float("nan"), dtype=torch.float32, device=device)
+    kv.resq_attention_prefill(cache, q16, 1, 0, out)
+    tail = torch.full((Tc, Hq, D), float("nan"), dtype=torch.float32, device=device)
+    kv.resq_attention_prefill(cache, q16[S - Tc:].contiguous(), 1, S - Tc, tail)
+    assert resq.resq_device_status() == resq.OK
+    out_h, tail_h, q16_h = host(out), host(tail), host(q16)
+    assert np.isfinite(out_h).all() and np.isfinite(tail_h).all()
+    kf, vf = synth.bf16_bits_to_f32(_bits(k)), synth.bf16_bits_to_f32(_bits(v))
+    Yk, _, _ = okv.project_int8(kf.reshape(-1, D), *okv.quantize_uc(W_C))
+    dk = okv.kv_dequantize(okv.kv_quantize(Yk)).reshape(S, Hkv, D)
+    dv = okv.kv_dequantize(okv.kv_quantize(vf.reshape(-1, D))).reshape(S, Hkv, D)
+    g = Hq // Hkv
+    tokens = [0, 1, 31, 32, 63, 64, 65, 4095, 4096, 7168, 7199, 7200, 8160, 8191]
+    for t in tokens:
+        for hq in (0, 7, 22, 31):
+            h = hq // g
+            ref = okv.attention_queries(q16_h[t:t + 1, hq:hq + 1], [[dk[:, h]]], [[dv[:, h]]], [0], [t + 1], 1, 1)[0, 0]
+            vmax = np.abs(dv[:t + 1, h]).max()
+            assert np.abs(out_h[t, hq] - ref).max() <= 1e-3 * vmax, (t, hq)
+            if t >= S - Tc:
+                assert np.abs(tail_h[t - (S - Tc), hq] - ref).max() <= 1e-3 * vmax, (t, hq)
+    vall = np.abs(dv).max()
+    assert np.abs(out_h[S - Tc:] - tail_h).max() <= 1e-3 * vall
