@@ -206,6 +206,22 @@ HOST_LEAD_CYCLES = 60_000_000  # ~30 ms of device idling, enough for the host to
 DECODE_COPIES = 3  # distinct copies of the packed weights, cycled per step: one block's 123 MB would sit in the 126 MB L2
 
 
+def decode_leg_with_clocks(gpu_id, *a):
+    """decode_leg with the SM clock sampled over the leg (the timed chains last under a millisecond each, far below
+    the sampling period, so the record covers the leg as a whole): adds `clocks` and, per T, the chain's time x the
+    median clock in SM cycles, which is what to compare between boxes that settle at different clocks."""
+    sampler = ClockSampler(gpu_id)
+    sampler.start()
+    out = decode_leg(*a)
+    out["clocks"] = sampler.stop()
+    mhz = out["clocks"].get("sm_mhz")
+    if mhz:
+        for k, v in out.items():
+            if isinstance(v, dict) and "mixed_gemv_us" in v:
+                v["mixed_gemv_sm_kcycles"] = round(v["mixed_gemv_us"] * mhz / 1e3, 1)
+    return out
+
+
 def decode_leg(resq, torch, dev, peaks, layers, steps):
     """Few-token variant of the same block: packed INT8 + nibble-packed INT4 weights with fp16 scales,
     streamed once per step.  Reports the weight-stream rate of the mixed GEMV kernels against the HBM
@@ -780,12 +796,16 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    gpu_id = str(getattr(torch.cuda.get_device_properties(dev), "uuid", local_rank))
+    if not gpu_id.startswith("GPU-") and "-" in gpu_id:
+        gpu_id = "GPU-" + gpu_id
+
     if args.kv_only:  # profiling runs: the attention-block leg alone
         print(json.dumps({"kv_cache_path": kv_leg(resq, torch, dev, peaks, max(5, min(args.steps, 20)), args.kv_seqs,
                                                   args.kv_len)}))
         return
     if args.decode_only:  # profiling runs: the few-token leg alone
-        print(json.dumps({"decode": decode_leg(resq, torch, dev, peaks, layers, max(5, min(args.steps, 20)))}))
+        print(json.dumps({"decode": decode_leg_with_clocks(gpu_id, resq, torch, dev, peaks, layers, max(5, min(args.steps, 20)))}))
         return
 
     for _ in range(max(args.warmup, 3)):
@@ -794,9 +814,6 @@ def run_ours(args):
     if st != resq.OK:
         raise SystemExit(f"device status {st}: {resq.status_string(st)}")
 
-    gpu_id = str(getattr(torch.cuda.get_device_properties(dev), "uuid", local_rank))
-    if not gpu_id.startswith("GPU-") and "-" in gpu_id:
-        gpu_id = "GPU-" + gpu_id
     sampler = ClockSampler(gpu_id)
     sampler.start()
     events = []
@@ -960,7 +977,7 @@ def run_ours(args):
     # ---- decode variant of the same block (this rank only; reported by rank 0)
     decode = None
     if not args.no_decode and not only:
-        decode = decode_leg(resq, torch, dev, peaks, layers, max(5, min(args.steps, 20)))
+        decode = decode_leg_with_clocks(gpu_id, resq, torch, dev, peaks, layers, max(5, min(args.steps, 20)))
         k = decode["T1"]
         kernels["mixed_gemm_decode_T1"] = {"bound": "hbm", "dtype": "int8", "achieved": k["weight_stream_gbs"],
                                            "peak": peaks["hbm_gbs"], "unit": "GB/s",
